@@ -1,0 +1,413 @@
+#!/usr/bin/env python
+"""Benchmark of the tree-verify path: one step = graft_build_tree -> graft_tree_verify_attn ->
+graft_accept -> graft_compact_kv over one batch of synthetic input.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload cfg4-B4] [--impl ours|reference]
+
+Prints ONE JSON line.  `value` is algorithmic KV bytes per step / device time per step (GB/s, all
+ranks together); `roofline` times graft_tree_verify_attn alone with CUDA events inside the same
+timed region; `e2e` repeats the step with that step's inputs coming from pinned host memory and
+its results read back; `cpu_baseline` times the CPU oracle on a bounded sample.
+With --impl reference the oracle itself is the timed arm (host cores only).
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import subprocess
+import sys
+import tempfile
+import time
+
+import numpy as np
+import torch
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+from paper_2605_20104_b200 import workloads as W  # noqa: E402
+
+L2_BYTES = 126e6
+METRIC = "tree-verify attn HBM GB/s (KV bytes per verify step / step time)"
+
+WORKLOADS = {
+    # name: (config id, B, L)
+    "cfg1": ("1", None, None),
+    "cfg2": ("2", None, None),
+    "cfg3": ("3", None, None),
+    "cfg4-B1": ("4", 1, 65536),
+    "cfg4-B1-32k": ("4", 1, 32768),
+    "cfg4-B4": ("4", 4, 65536),
+    "cfg5": ("5", None, None),
+}
+DEFAULT_WORKLOAD = "cfg4-B4"          # the 64K-context point the metric's target is stated on
+EXTRA_WORKLOADS = ["cfg2", "cfg3", "cfg4-B1-32k", "cfg4-B1", "cfg5"]
+
+
+def measured_peaks():
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(p):
+        d = json.load(open(p))
+        return float(d["hbm_gbs"]), "measured"
+    return 6650.0, "fallback"
+
+
+def kv_bytes(w, tree_size):
+    """Algorithmic bytes of one attention call: every visible K and V row once, plus Q and O."""
+    kv = sum(w.Hkv * (int(w.seq_len[b]) + int(tree_size[b])) * w.d * 2 * 2 for b in range(w.B))
+    qo = sum(2 * int(tree_size[b]) * w.Hq * w.d * 2 for b in range(w.B))
+    return kv, qo
+
+
+class ClockSampler:
+    QUERY = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,clocks_event_reasons.hw_slowdown,"
+             "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+             "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.f = tempfile.NamedTemporaryFile("w+", suffix=".csv", delete=False)
+        try:
+            self.p = subprocess.Popen(["nvidia-smi", "-i", str(index), "--query-gpu=" + self.QUERY,
+                                       "--format=csv,noheader,nounits", "-lms", "100"], stdout=self.f,
+                                      stderr=subprocess.DEVNULL)
+        except OSError:
+            self.p = None
+
+    def stop(self):
+        out = {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
+        if self.p is None:
+            return out
+        self.p.terminate()
+        try:
+            self.p.wait(timeout=5)
+        except subprocess.TimeoutExpired:
+            self.p.kill()
+        self.f.flush()
+        rows = [r.split(",") for r in open(self.f.name).read().strip().splitlines() if r.count(",") >= 8]
+        os.unlink(self.f.name)
+        if not rows:
+            return out
+        sm = [float(r[1]) for r in rows if r[1].strip().replace(".", "").isdigit()]
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        reasons = [n for i, n in enumerate(names) if any("Active" == r[5 + i].strip() for r in rows)]
+        out.update(sm_mhz=float(np.median(sm)) if sm else None, sm_max_mhz=float(rows[0][2]), reasons=reasons,
+                   samples=len(rows), power_w_max=max(float(r[3]) for r in rows))
+        return out
+
+
+def make_step(w, n_rot, device):
+    """Device state with n_rot distinct K/V caches (rotated per step when one cache fits in L2)."""
+    from paper_2605_20104_b200.step import VerifyStep
+    vs = VerifyStep(w, device=device, upload_qkv=False)
+    g = torch.Generator(device="cuda")
+    g.manual_seed(1234 + w.seed)
+    dev = "cuda:%d" % device
+    vs.Q = (torch.randn(w.B, w.T_max, w.Hq, w.d, generator=g, device=dev) * w.std).to(torch.bfloat16)
+    caches = []
+    for _ in range(n_rot):
+        K = (torch.randn(w.B, w.Hkv, w.S_cap, w.d, generator=g, device=dev) * w.std).to(torch.bfloat16)
+        V = (torch.randn(w.B, w.Hkv, w.S_cap, w.d, generator=g, device=dev) * w.std).to(torch.bfloat16)
+        caches.append((K, V))
+    vs.Kc, vs.Vc = caches[0]
+    return vs, caches
+
+
+def set_target_next(vs, w):
+    """The target's greedy ids for the tree the device built (input generation, untimed)."""
+    t = vs.tree_host()
+    nxt = W.draw_target_next(t["tree_token"], t["tree_parent"], t["tree_size"], t["tree_src"], w.V, w.p_draft,
+                             w.p_graft, w.seed)
+    vs.target_next.copy_(torch.from_numpy(nxt))
+    return t
+
+
+def time_workload(name, steps, warmup, device, variant, do_e2e=True):
+    from paper_2605_20104_b200 import binding as G
+    cfg, B, L = WORKLOADS[name]
+    w = W.config(cfg, B=B, L=L)
+    # build once to learn the tree sizes (they define the algorithmic bytes)
+    kv_guess = w.B * w.Hkv * w.S_cap * w.d * 4
+    n_rot = 1 if kv_guess > 2 * L2_BYTES else int(min(16, np.ceil(3 * L2_BYTES / kv_guess)))
+    vs, caches = make_step(w, n_rot, device)
+    vs.build()
+    tree = set_target_next(vs, w)
+    kvb, qob = kv_bytes(w, tree["tree_size"])
+
+    def one(i):
+        vs.Kc, vs.Vc = caches[i % n_rot]
+        vs.build()
+        ea[i % len(ea)].record()
+        vs.attn(variant)
+        eb[i % len(eb)].record()
+        vs.accept()
+        vs.compact()
+
+    ea = [torch.cuda.Event(enable_timing=True) for _ in range(steps)]
+    eb = [torch.cuda.Event(enable_timing=True) for _ in range(steps)]
+    for i in range(warmup):
+        one(i)
+    torch.cuda.synchronize()
+    flags = vs.ctx.device_status()
+    t0, t1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    return dict(w=w, vs=vs, caches=caches, one=one, ea=ea, eb=eb, t0=t0, t1=t1, kvb=kvb, qob=qob, n_rot=n_rot,
+                flags=flags, tree=tree)
+
+
+def run_timed(st, steps):
+    st["t0"].record()
+    for i in range(steps):
+        st["one"](i)
+    st["t1"].record()
+    torch.cuda.synchronize()
+    total_ms = st["t0"].elapsed_time(st["t1"])
+    attn_ms = [a.elapsed_time(b) for a, b in zip(st["ea"], st["eb"])]
+    return total_ms / steps, float(np.mean(attn_ms)), float(np.min(attn_ms))
+
+
+def run_e2e(st, steps, warmup, variant):
+    """The same step with its inputs arriving from pinned host memory and its results read back.
+    The cached prefix is resident state (it was produced by earlier steps); the step's own inputs
+    are the draft arrays, Q, the tree tokens' K/V rows and the target's ids."""
+    w, vs = st["w"], st["vs"]
+    pin = lambda t: t.cpu().pin_memory()
+    B, T = w.B, w.T_max
+    h_in = dict(draft_token=pin(vs.draft_token), draft_parent=pin(vs.draft_parent), draft_score=pin(vs.draft_score),
+                n_draft=pin(vs.n_draft), seq_len=pin(vs.seq_len), Q=pin(vs.Q), target_next=pin(vs.target_next))
+    L0 = int(w.seq_len.min())
+    h_k = torch.randn(B, w.Hkv, T, w.d).to(torch.bfloat16).pin_memory()
+    h_v = torch.randn(B, w.Hkv, T, w.d).to(torch.bfloat16).pin_memory()
+    d_k, d_v = torch.empty_like(h_k, device=vs.dev), torch.empty_like(h_v, device=vs.dev)
+    seq = [int(x) for x in w.seq_len]
+    h_out = dict(O=torch.empty_like(vs.O, device="cpu").pin_memory(), n_acc=pin(vs.n_acc), path=pin(vs.path),
+                 bonus=pin(vs.bonus), new_seq_len=pin(vs.new_seq_len))
+    h2d = sum(t.numel() * t.element_size() for t in h_in.values()) + h_k.numel() * 2 * 2
+    d2h = sum(t.numel() * t.element_size() for t in h_out.values())
+
+    def one(i):
+        vs.Kc, vs.Vc = st["caches"][i % st["n_rot"]]
+        for k, t in h_in.items():
+            getattr(vs, k).copy_(t, non_blocking=True)
+        d_k.copy_(h_k, non_blocking=True)
+        d_v.copy_(h_v, non_blocking=True)
+        for b in range(B):                                   # the projection's write of the tree K/V rows
+            vs.Kc[b, :, seq[b]:seq[b] + T].copy_(d_k[b])
+            vs.Vc[b, :, seq[b]:seq[b] + T].copy_(d_v[b])
+        vs.build()
+        vs.attn(variant)
+        vs.accept()
+        vs.compact()
+        for k, t in h_out.items():
+            t.copy_(getattr(vs, k), non_blocking=True)
+        torch.cuda.synchronize()                             # the caller reads the result every step
+
+    for i in range(warmup):
+        one(i)
+    t0, t1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    torch.cuda.synchronize()
+    t0.record()
+    for i in range(steps):
+        one(i)
+    t1.record()
+    torch.cuda.synchronize()
+    return t0.elapsed_time(t1) / steps, h2d, d2h
+
+
+class OracleTimer:
+    """Times the CPU oracle, as it stands, on bounded samples of one step of workload `w`: tree
+    assembly and acceptance in full, attention on sampled rows, compaction on one sequence; the
+    sampled parts are scaled to the full step."""
+
+    def __init__(self, w):
+        import oracle
+        oracle.build()
+        self.o, self.w = oracle, w
+        self.tree = oracle.build_tree(w)
+        W.make_qkv(w)                                    # the workload's tensors, drawn once (untimed)
+        self.bits = (W.bf16_bits(w.Q), W.bf16_bits(w.Kc), W.bf16_bits(w.Vc))
+        self.nxt = W.draw_target_next(self.tree["tree_token"], self.tree["tree_parent"], self.tree["tree_size"],
+                                      self.tree["tree_src"], w.V, w.p_draft, w.p_graft, w.seed)
+        self.total_rows = int(self.tree["tree_size"].sum()) * w.Hq
+        self.threads = 1
+
+    def attn_rows(self, n, rng):
+        w, tree = self.w, self.tree
+        rows = np.array([(b, int(rng.integers(0, tree["tree_size"][b])), int(rng.integers(0, w.Hq)))
+                         for b in rng.integers(0, w.B, size=n)], np.int32)
+        t = time.perf_counter()
+        out = self.o.tree_attn(*self.bits, w.seq_len, tree["tree_size"], tree["tree_anc"], w.scale, rows=rows)
+        self.threads = out["threads"]
+        return time.perf_counter() - t
+
+    def rows_for(self, seconds, rng):
+        t = self.attn_rows(32, rng)
+        return int(min(1 << 16, max(32, 32 * seconds / max(t, 1e-4))))
+
+    def step_seconds(self, n_rows, rng):
+        """Estimated seconds of one full step from a sample with n_rows attention rows."""
+        w, tree, o = self.w, self.tree, self.o
+        t = time.perf_counter()
+        o.build_tree(w)
+        t_build = time.perf_counter() - t
+        t_rows = self.attn_rows(n_rows, rng)
+        t = time.perf_counter()
+        acc = o.accept(tree["tree_token"], tree["tree_parent"], tree["tree_size"], self.nxt)
+        t_acc = time.perf_counter() - t
+        t = time.perf_counter()
+        o.compact_kv(self.bits[1][:1], self.bits[2][:1], w.seq_len[:1], acc["n_acc"][:1], acc["path"][:1])
+        t_comp = (time.perf_counter() - t) * w.B
+        return t_build + t_rows * self.total_rows / n_rows + t_acc + t_comp
+
+    def describe(self, n_rows):
+        return ("tree assembly and acceptance in full; attention on %d of %d rows (uniform over (b,t,h)), scaled; "
+                "compaction on 1 of %d sequences, scaled" % (n_rows, self.total_rows, self.w.B))
+
+
+def reference_arm(args):
+    """--impl reference: the CPU oracle as it stands, on the host cores, same metric and workload.
+    Each step is a bounded sample (about two seconds of attention rows) scaled to a full step."""
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    cfg, B, L = WORKLOADS[args.workload]
+    w = W.config(cfg, B=B, L=L)
+    ot = OracleTimer(w)
+    rng = np.random.default_rng(0)
+    n_rows = ot.rows_for(2.0, rng)
+    vals = []
+    for i in range(args.warmup + args.steps):
+        est = ot.step_seconds(n_rows, rng)
+        if i >= args.warmup:
+            vals.append(est)
+    kvb, _ = kv_bytes(w, ot.tree["tree_size"])
+    sec = float(np.mean(vals))
+    value = kvb / sec / 1e9
+    line = {"impl": "reference", "metric": METRIC, "value": value, "unit": "GB/s", "n_gpus": args.gpus,
+            "steps": args.steps, "warmup": args.warmup, "ms_per_step": sec * 1e3, "higher_is_better": True,
+            "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+            "config": {"workload": args.workload, "B": w.B, "Hq": w.Hq, "Hkv": w.Hkv, "d": w.d,
+                       "L": int(w.seq_len.max()), "T_max": w.T_max},
+            "cpu_baseline": {"value": value, "unit": "GB/s", "cores": ot.threads, "kind": "oracle",
+                             "sample": ot.describe(n_rows)},
+            "e2e": {"value": value, "unit": "GB/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+            "gpu_launches": 0}
+    print(json.dumps(line))
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=30)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default=DEFAULT_WORKLOAD, choices=sorted(WORKLOADS))
+    ap.add_argument("--variant", default="auto", choices=["auto", "mma", "tc"])
+    ap.add_argument("--no-extra", action="store_true", help="skip the other configurations' lines")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    args.warmup = max(args.warmup, 3)
+    if args.impl == "reference":
+        reference_arm(args)
+        return
+
+    from paper_2605_20104_b200 import binding as G
+    variant = {"auto": G.ATTN_AUTO, "mma": G.ATTN_MMA_SYNC, "tc": G.ATTN_TCGEN05}[args.variant]
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    torch.cuda.set_device(local)
+    dist = None
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+
+    def barrier():
+        if dist is not None:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    def max_over_ranks(x):
+        if dist is None:
+            return x
+        t = torch.tensor([x], dtype=torch.float64, device="cuda")
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        return float(t.item())
+
+    # every rank verifies its own batch (sequences are independent: no data-path collective)
+    st = time_workload(args.workload, args.steps, args.warmup, local, variant)
+    sampler = ClockSampler(local) if rank == 0 else None
+    barrier()
+    ms_step, attn_ms, attn_ms_min = run_timed(st, args.steps)
+    barrier()
+    clocks = sampler.stop() if sampler else None
+    ms_step = max_over_ranks(ms_step)
+    attn_ms = max_over_ranks(attn_ms)
+    e2e_ms, h2d, d2h = run_e2e(st, max(3, args.steps // 3), 3, variant)
+    e2e_ms = max_over_ranks(e2e_ms)
+    flags = st["vs"].ctx.device_status()
+
+    if rank != 0:
+        if dist is not None:
+            dist.barrier()
+            dist.destroy_process_group()
+        return
+
+    w = st["w"]
+    peak, peak_kind = measured_peaks()
+    kvb, qob = st["kvb"], st["qob"]
+    value = kvb * world / (ms_step * 1e-3) / 1e9
+    achieved = (kvb + qob) / (attn_ms * 1e-3) / 1e9
+    line = {
+        "metric": METRIC, "value": value, "unit": "GB/s", "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
+        "ms_per_step": ms_step, "us_per_step": ms_step * 1e3, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+        "config": {"workload": args.workload, "B": w.B, "Hq": w.Hq, "Hkv": w.Hkv, "d": w.d, "L": int(w.seq_len.max()),
+                   "T": [int(x) for x in st["tree"]["tree_size"]][:4], "T_max": w.T_max, "attn_variant": args.variant,
+                   "l2": "inputs larger than L2" if st["n_rot"] == 1 else "rotating %d KV caches (> 3x L2)" % st["n_rot"],
+                   "kv_bytes_per_step": kvb},
+        "roofline": {"bound": "hbm", "kernel": "graft_tree_verify_attn (split kernel + merge)",
+                     "achieved": achieved, "peak": peak, "peak_kind": "of " + peak_kind, "unit": "GB/s",
+                     "frac": achieved / peak, "frac_of_8TBps_nominal": achieved / 8000.0,
+                     "us_per_call": attn_ms * 1e3, "us_per_call_min": attn_ms_min * 1e3,
+                     "algorithmic_bytes": kvb + qob, "traffic": TRAFFIC.get(args.workload)},
+        "e2e": {"value": kvb * world / (e2e_ms * 1e-3) / 1e9, "unit": "GB/s", "ms_per_step": e2e_ms,
+                "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
+                "note": "cached prefix resident; step inputs (draft arrays, Q, tree K/V rows, target ids) from pinned host"},
+        "gpu_launches": 5 * args.steps,
+        "clocks": clocks, "device_flags": flags,
+    }
+    if not args.no_extra and world == 1:
+        extra = []
+        del st
+        torch.cuda.empty_cache()
+        for name in EXTRA_WORKLOADS:
+            s2 = time_workload(name, args.steps, args.warmup, local, variant)
+            ms2, a2, a2min = run_timed(s2, args.steps)
+            kv2, qo2 = s2["kvb"], s2["qob"]
+            extra.append({"workload": name, "us_per_step": ms2 * 1e3, "attn_us": a2 * 1e3, "attn_us_min": a2min * 1e3,
+                          "attn_GBps": (kv2 + qo2) / (a2 * 1e-3) / 1e9,
+                          "attn_frac_of_" + peak_kind: (kv2 + qo2) / (a2 * 1e-3) / 1e9 / peak,
+                          "kv_bytes": kv2, "l2": "larger than L2" if s2["n_rot"] == 1 else "rotating %d caches" % s2["n_rot"]})
+            del s2
+            torch.cuda.empty_cache()
+        line["other_configs"] = extra
+    if not args.no_cpu_baseline:
+        cfg, B, L = WORKLOADS[args.workload]
+        ot = OracleTimer(W.config(cfg, B=B, L=L))
+        rng = np.random.default_rng(0)
+        n_rows = ot.rows_for(12.0, rng)
+        est = ot.step_seconds(n_rows, rng)
+        line["cpu_baseline"] = {"value": kvb / est / 1e9, "unit": "GB/s", "seconds_per_step_est": est,
+                                "cores": ot.threads, "kind": "oracle", "sample": ot.describe(n_rows)}
+    print(json.dumps(line))
+    if dist is not None:
+        dist.barrier()
+        dist.destroy_process_group()
+
+
+# dram__bytes_read.sum + dram__bytes_write.sum of the attention kernel per launch, from the ncu
+# captures summarised under profiles/ (None until a capture of that workload exists)
+TRAFFIC = {}
+
+if __name__ == "__main__":
+    main()

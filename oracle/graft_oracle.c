@@ -194,6 +194,7 @@ unsigned orc_build_tree(const orc_build_args *a) {
         if (graft) {
             int K_ret = t_hi - t_lo;
             if (K_ret > budget - K_kept) K_ret = budget - K_kept;
+            if (K_ret < 0) K_ret = 0;
             for (int u = 0; u < K_ret; ++u) {
                 int tp = a->tmpl_parent[t_lo + u], r = a->tmpl_rank[t_lo + u];
                 int j = K_kept + u, ok = 1;

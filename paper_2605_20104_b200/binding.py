@@ -1,0 +1,210 @@
+"""ctypes binding of libgraft.so: the same entry points as include/graft.h, taking torch CUDA
+tensors.  Argument marshalling only; every step of the path runs in the library's kernels.
+PyTorch supplies device memory and the stream, nothing else.
+
+Importing this module loads the library and raises if it has not been built
+(`python -m paper_2605_20104_b200.build`): there is no fallback path.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+from typing import Optional
+
+import torch
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libgraft.so")
+
+if not os.path.exists(LIB_PATH):
+    raise ImportError("libgraft.so is not built; run `python -m paper_2605_20104_b200.build` "
+                      "(the CUDA library is the only implementation, there is no fallback)")
+_lib = C.CDLL(LIB_PATH)
+
+OK, ERR_INVALID_ARG, ERR_UNSUPPORTED, ERR_WORKSPACE_TOO_SMALL, ERR_CUDA = 0, -1, -2, -3, -4
+FLAG_BAD_SIZE, FLAG_BAD_PARENT, FLAG_BAD_TOKEN, FLAG_ORPHAN = 1, 2, 4, 8
+FLAG_BUDGET, FLAG_BAD_TEMPLATE, FLAG_NAN_SCORE, FLAG_BAD_PATH, FLAG_WAIT_TIMEOUT = 16, 32, 64, 128, 256
+PRUNE_NONE, PRUNE_TOPK, PRUNE_GATED, PRUNE_NODE = 0, 1, 2, 3
+ATTN_AUTO, ATTN_MMA_SYNC, ATTN_TCGEN05 = 0, 1, 2
+
+EXPORTS = ("graft_workspace_bytes", "graft_create", "graft_destroy", "graft_status_string", "graft_device_status",
+           "graft_build_tree", "graft_tree_verify_attn", "graft_accept", "graft_compact_kv")
+
+_vp = C.c_void_p
+
+
+class BuildParams(C.Structure):
+    _fields_ = ([(n, C.c_int) for n in ("B", "N_max", "T_max", "K_max", "V", "k", "S_cap", "mode", "gate_depth")] +
+                [("node_threshold", C.c_float), ("n_ckpt", C.c_int), ("N_tmpl", C.c_int)] +
+                [(n, _vp) for n in ("draft_token", "draft_parent", "draft_score", "n_draft", "seq_len", "M", "keep_count",
+                                    "k_max", "ckpt_depth", "ckpt_keep", "ckpt_log_tau", "tmpl_offset", "tmpl_parent",
+                                    "tmpl_rank", "tree_token", "tree_parent", "tree_pos", "tree_src", "tree_anc",
+                                    "tree_size")])
+
+
+class AttnParams(C.Structure):
+    _fields_ = ([(n, C.c_int) for n in ("B", "T_max", "Hq", "Hkv", "d", "S_cap")] +
+                [("scale", C.c_float), ("variant", C.c_int),
+                 ("Q", _vp), ("q_stride_b", C.c_int64), ("q_stride_t", C.c_int64), ("q_stride_h", C.c_int64),
+                 ("Kc", _vp), ("Vc", _vp),
+                 ("kv_stride_b", C.c_int64), ("kv_stride_h", C.c_int64), ("kv_stride_s", C.c_int64),
+                 ("O", _vp), ("o_stride_b", C.c_int64), ("o_stride_t", C.c_int64), ("o_stride_h", C.c_int64),
+                 ("LSE", _vp), ("seq_len", _vp), ("tree_size", _vp), ("tree_anc", _vp)])
+
+
+class AcceptParams(C.Structure):
+    _fields_ = ([("B", C.c_int), ("T_max", C.c_int)] +
+                [(n, _vp) for n in ("tree_token", "tree_parent", "tree_anc", "tree_size", "target_next", "n_acc", "path",
+                                    "best_node", "bonus")])
+
+
+class CompactParams(C.Structure):
+    _fields_ = ([(n, C.c_int) for n in ("B", "Hkv", "d", "S_cap", "T_max", "n_layers")] +
+                [(n, C.c_int64) for n in ("layer_stride", "kv_stride_b", "kv_stride_h", "kv_stride_s")] +
+                [(n, _vp) for n in ("Kc", "Vc", "seq_len", "n_acc", "path", "new_seq_len")])
+
+
+_lib.graft_workspace_bytes.restype = C.c_size_t
+_lib.graft_workspace_bytes.argtypes = [C.c_int] * 6
+_lib.graft_create.restype = C.c_int
+_lib.graft_create.argtypes = [C.POINTER(_vp), C.c_int, _vp, C.c_size_t]
+_lib.graft_destroy.restype = C.c_int
+_lib.graft_destroy.argtypes = [_vp]
+_lib.graft_status_string.restype = C.c_char_p
+_lib.graft_status_string.argtypes = [C.c_int]
+_lib.graft_device_status.restype = C.c_int
+_lib.graft_device_status.argtypes = [_vp, _vp, C.POINTER(C.c_uint), C.c_int]
+for _name, _typ in (("graft_build_tree", BuildParams), ("graft_tree_verify_attn", AttnParams),
+                    ("graft_accept", AcceptParams), ("graft_compact_kv", CompactParams)):
+    getattr(_lib, _name).restype = C.c_int
+    getattr(_lib, _name).argtypes = [_vp, C.POINTER(_typ), _vp]
+
+
+class GraftError(RuntimeError):
+    def __init__(self, code: int, where: str):
+        self.code = code
+        super().__init__("%s: %s (%d)" % (where, _lib.graft_status_string(code).decode(), code))
+
+
+def _check(code: int, where: str) -> None:
+    if code != OK:
+        raise GraftError(code, where)
+
+
+def _ptr(t: Optional[torch.Tensor], dtype=None) -> Optional[int]:
+    if t is None:
+        return None
+    assert t.is_cuda, "device tensor expected"
+    if dtype is not None:
+        assert t.dtype == dtype, (t.dtype, dtype)
+    return t.data_ptr()
+
+
+def _stream() -> int:
+    return torch.cuda.current_stream().cuda_stream
+
+
+def graft_workspace_bytes(device: int, B: int, Hq: int, Hkv: int, d: int, T_max: int) -> int:
+    return int(_lib.graft_workspace_bytes(device, B, Hq, Hkv, d, T_max))
+
+
+class Context:
+    """graft_ctx plus the torch-allocated workspace it is bound to."""
+
+    def __init__(self, B: int, Hq: int, Hkv: int, d: int, T_max: int, device: Optional[int] = None,
+                 workspace: Optional[torch.Tensor] = None):
+        self.device = torch.cuda.current_device() if device is None else device
+        if workspace is None:
+            n = graft_workspace_bytes(self.device, B, Hq, Hkv, d, T_max)
+            if n == 0:
+                raise GraftError(ERR_UNSUPPORTED, "graft_workspace_bytes")
+            workspace = torch.empty(n, dtype=torch.uint8, device="cuda:%d" % self.device)
+        self.workspace = workspace
+        h = _vp()
+        _check(_lib.graft_create(C.byref(h), self.device, workspace.data_ptr(), workspace.numel()), "graft_create")
+        self.handle = h
+
+    def close(self) -> None:
+        if self.handle:
+            _lib.graft_destroy(self.handle)
+            self.handle = None
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+    def device_status(self, clear: bool = True) -> int:
+        """Synchronises the current stream and returns the accumulated GRAFT_FLAG_* bits."""
+        f = C.c_uint(0)
+        _check(_lib.graft_device_status(self.handle, _stream(), C.byref(f), int(clear)), "graft_device_status")
+        return int(f.value)
+
+
+def graft_build_tree(ctx: Context, *, mode: int, K_max: int, V: int, k: int, S_cap: int,
+                     draft_token, draft_parent, draft_score, n_draft, seq_len, M=None, keep_count=None, k_max=None,
+                     gate_depth: int = 0, node_threshold: float = 0.0, ckpt_depth=None, ckpt_keep=None,
+                     ckpt_log_tau=None, tmpl_offset=None, tmpl_parent=None, tmpl_rank=None,
+                     tree_token, tree_parent, tree_pos, tree_src, tree_anc, tree_size) -> None:
+    B, N_max = draft_token.shape
+    T_max = tree_token.shape[1]
+    i32, f32 = torch.int32, torch.float32
+    p = BuildParams(B=B, N_max=N_max, T_max=T_max, K_max=K_max, V=V, k=k, S_cap=S_cap, mode=mode, gate_depth=gate_depth,
+                    node_threshold=node_threshold, n_ckpt=0 if ckpt_depth is None else ckpt_depth.numel(),
+                    N_tmpl=0 if tmpl_parent is None else tmpl_parent.numel(),
+                    draft_token=_ptr(draft_token, i32), draft_parent=_ptr(draft_parent, i32),
+                    draft_score=_ptr(draft_score, f32), n_draft=_ptr(n_draft, i32), seq_len=_ptr(seq_len, i32),
+                    M=_ptr(M, i32), keep_count=_ptr(keep_count, i32), k_max=_ptr(k_max, i32),
+                    ckpt_depth=_ptr(ckpt_depth, i32), ckpt_keep=_ptr(ckpt_keep, i32),
+                    ckpt_log_tau=_ptr(ckpt_log_tau, f32), tmpl_offset=_ptr(tmpl_offset, i32),
+                    tmpl_parent=_ptr(tmpl_parent, i32), tmpl_rank=_ptr(tmpl_rank, i32),
+                    tree_token=_ptr(tree_token, i32), tree_parent=_ptr(tree_parent, i32), tree_pos=_ptr(tree_pos, i32),
+                    tree_src=_ptr(tree_src, i32), tree_anc=_ptr(tree_anc, torch.int64), tree_size=_ptr(tree_size, i32))
+    _check(_lib.graft_build_tree(ctx.handle, C.byref(p), _stream()), "graft_build_tree")
+
+
+def graft_tree_verify_attn(ctx: Context, *, Q, Kc, Vc, O, seq_len, tree_size, tree_anc, scale: float,
+                           LSE=None, variant: int = ATTN_AUTO) -> None:
+    """Q, O: bf16 [B, T_max, Hq, d]; Kc, Vc: bf16 [B, Hkv, S_cap, d] (any strides with a contiguous
+    last axis); tree_anc: int64 [B, T_max] holding the 64-bit masks."""
+    bf = torch.bfloat16
+    B, T_max, Hq, d = Q.shape
+    _, Hkv, S_cap, _ = Kc.shape
+    assert Q.stride(3) == 1 and Kc.stride(3) == 1 and Vc.stride(3) == 1 and O.stride(3) == 1
+    assert Kc.stride() == Vc.stride() and Kc.shape == Vc.shape and O.shape == Q.shape
+    p = AttnParams(B=B, T_max=T_max, Hq=Hq, Hkv=Hkv, d=d, S_cap=S_cap, scale=scale, variant=variant,
+                   Q=_ptr(Q, bf), q_stride_b=Q.stride(0), q_stride_t=Q.stride(1), q_stride_h=Q.stride(2),
+                   Kc=_ptr(Kc, bf), Vc=_ptr(Vc, bf), kv_stride_b=Kc.stride(0), kv_stride_h=Kc.stride(1),
+                   kv_stride_s=Kc.stride(2),
+                   O=_ptr(O, bf), o_stride_b=O.stride(0), o_stride_t=O.stride(1), o_stride_h=O.stride(2),
+                   LSE=_ptr(LSE, torch.float32), seq_len=_ptr(seq_len, torch.int32),
+                   tree_size=_ptr(tree_size, torch.int32), tree_anc=_ptr(tree_anc, torch.int64))
+    _check(_lib.graft_tree_verify_attn(ctx.handle, C.byref(p), _stream()), "graft_tree_verify_attn")
+
+
+def graft_accept(ctx: Context, *, tree_token, tree_parent, tree_anc, tree_size, target_next, n_acc, path, best_node,
+                 bonus) -> None:
+    i32 = torch.int32
+    B, T_max = tree_token.shape
+    p = AcceptParams(B=B, T_max=T_max, tree_token=_ptr(tree_token, i32), tree_parent=_ptr(tree_parent, i32),
+                     tree_anc=_ptr(tree_anc, torch.int64), tree_size=_ptr(tree_size, i32),
+                     target_next=_ptr(target_next, i32), n_acc=_ptr(n_acc, i32), path=_ptr(path, i32),
+                     best_node=_ptr(best_node, i32), bonus=_ptr(bonus, i32))
+    _check(_lib.graft_accept(ctx.handle, C.byref(p), _stream()), "graft_accept")
+
+
+def graft_compact_kv(ctx: Context, *, Kc, Vc, seq_len, n_acc, path, new_seq_len) -> None:
+    """Kc, Vc: bf16 [B, Hkv, S_cap, d] or [n_layers, B, Hkv, S_cap, d], compacted in place."""
+    bf, i32 = torch.bfloat16, torch.int32
+    if Kc.dim() == 4:
+        n_layers, layer_stride, off = 1, 0, 0
+    else:
+        n_layers, layer_stride, off = Kc.shape[0], Kc.stride(0), 1
+    B, Hkv, S_cap, d = Kc.shape[off:]
+    assert Kc.stride() == Vc.stride() and Kc.stride(-1) == 1
+    p = CompactParams(B=B, Hkv=Hkv, d=d, S_cap=S_cap, T_max=path.shape[1], n_layers=n_layers, layer_stride=layer_stride,
+                      kv_stride_b=Kc.stride(off), kv_stride_h=Kc.stride(off + 1), kv_stride_s=Kc.stride(off + 2),
+                      Kc=_ptr(Kc, bf), Vc=_ptr(Vc, bf), seq_len=_ptr(seq_len, i32), n_acc=_ptr(n_acc, i32),
+                      path=_ptr(path, i32), new_seq_len=_ptr(new_seq_len, i32))
+    _check(_lib.graft_compact_kv(ctx.handle, C.byref(p), _stream()), "graft_compact_kv")

@@ -1,0 +1,33 @@
+// Internal declarations shared by the library's translation units (not part of the C ABI).
+#pragma once
+#include <cuda_runtime.h>
+#include <stdint.h>
+#include "graft.h"
+
+struct graft_ctx {
+    int device;
+    int num_sms;
+    void* ws;           // caller-owned device workspace
+    size_t ws_bytes;
+    unsigned* status;   // device status word = first word of the workspace
+};
+
+// the first GRAFT_WS_HEADER bytes of the workspace are reserved (status word)
+#define GRAFT_WS_HEADER 256
+
+#define GRAFT_CHECK_CUDA(expr)                          \
+    do {                                                \
+        cudaError_t e_ = (expr);                        \
+        if (e_ != cudaSuccess) return GRAFT_ERR_CUDA;   \
+    } while (0)
+
+static inline bool graft_aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+// attention launchers (one per kernel family); both return GRAFT_OK or an error code
+int graft_attn_mma_init();   // per device, called by graft_create with the device current
+int graft_attn_tc_init();
+int graft_attn_mma_launch(graft_ctx* ctx, const graft_attn_params* p, cudaStream_t stream);
+int graft_attn_tc_launch(graft_ctx* ctx, const graft_attn_params* p, cudaStream_t stream);
+bool graft_attn_tc_supported(const graft_ctx* ctx, const graft_attn_params* p);
+size_t graft_attn_mma_ws_bytes(int num_sms, int B, int Hq, int Hkv, int d, int T_max);
+size_t graft_attn_tc_ws_bytes(int num_sms, int B, int Hq, int Hkv, int d, int T_max);
