@@ -61,7 +61,7 @@ def kv_bytes(w, tree_size):
 
 
 class ClockSampler:
-    QUERY = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,clocks_event_reasons.hw_slowdown,"
+    QUERY = ("timestamp,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,clocks_event_reasons.hw_slowdown,"
              "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
              "clocks_event_reasons.sw_power_cap")
 
@@ -74,7 +74,10 @@ class ClockSampler:
         except OSError:
             self.p = None
 
-    def stop(self):
+    def stop(self, t_begin=None, t_end=None):
+        """Median SM clock and active throttle reasons over the samples taken inside the wall-clock
+        window [t_begin, t_end] (the timed region); all samples if the window caught fewer than two."""
+        import datetime
         out = {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
         if self.p is None:
             return out
@@ -88,6 +91,16 @@ class ClockSampler:
         os.unlink(self.f.name)
         if not rows:
             return out
+        if t_begin is not None:
+            def ts(r):
+                try:
+                    return datetime.datetime.strptime(r[0].strip(), "%Y/%m/%d %H:%M:%S.%f").timestamp()
+                except ValueError:
+                    return None
+            inside = [r for r in rows if ts(r) is not None and t_begin - 0.05 <= ts(r) <= t_end + 0.05]
+            out["window"] = "timed region" if len(inside) >= 2 else "warm-up + timed region"
+            if len(inside) >= 2:
+                rows = inside
         sm = [float(r[1]) for r in rows if r[1].strip().replace(".", "").isdigit()]
         names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
         reasons = [n for i, n in enumerate(names) if any("Active" == r[5 + i].strip() for r in rows)]
@@ -241,7 +254,7 @@ class OracleTimer:
 
     def rows_for(self, seconds, rng):
         t = self.attn_rows(32, rng)
-        return int(min(1 << 16, max(32, 32 * seconds / max(t, 1e-4))))
+        return int(min(self.total_rows, max(32, 32 * seconds / max(t, 1e-4))))
 
     def step_seconds(self, n_rows, rng):
         """Estimated seconds of one full step from a sample with n_rows attention rows."""
@@ -297,8 +310,8 @@ def reference_arm(args):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=30)
-    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--steps", type=int, default=200)
+    ap.add_argument("--warmup", type=int, default=10)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default=DEFAULT_WORKLOAD, choices=sorted(WORKLOADS))
     ap.add_argument("--variant", default="auto", choices=["auto", "mma", "tc"])
@@ -334,12 +347,14 @@ def main():
         return float(t.item())
 
     # every rank verifies its own batch (sequences are independent: no data-path collective)
-    st = time_workload(args.workload, args.steps, args.warmup, local, variant)
     sampler = ClockSampler(local) if rank == 0 else None
+    st = time_workload(args.workload, args.steps, args.warmup, local, variant)
     barrier()
+    wall0 = time.time()
     ms_step, attn_ms, attn_ms_min = run_timed(st, args.steps)
     barrier()
-    clocks = sampler.stop() if sampler else None
+    wall1 = time.time()
+    clocks = sampler.stop(wall0, wall1) if sampler else None
     ms_step = max_over_ranks(ms_step)
     attn_ms = max_over_ranks(attn_ms)
     e2e_ms, h2d, d2h = run_e2e(st, max(3, args.steps // 3), 3, variant)
@@ -381,8 +396,9 @@ def main():
         del st
         torch.cuda.empty_cache()
         for name in EXTRA_WORKLOADS:
-            s2 = time_workload(name, args.steps, args.warmup, local, variant)
-            ms2, a2, a2min = run_timed(s2, args.steps)
+            k2 = min(args.steps, 50)
+            s2 = time_workload(name, k2, args.warmup, local, variant)
+            ms2, a2, a2min = run_timed(s2, k2)
             kv2, qo2 = s2["kvb"], s2["qob"]
             extra.append({"workload": name, "us_per_step": ms2 * 1e3, "attn_us": a2 * 1e3, "attn_us_min": a2min * 1e3,
                           "attn_GBps": (kv2 + qo2) / (a2 * 1e-3) / 1e9,

@@ -9,6 +9,7 @@
 #include <cuda_bf16.h>
 #include <math_constants.h>
 #include "attn_schedule.cuh"
+#include "attn_merge.cuh"
 #include "graft_internal.cuh"
 
 namespace {
@@ -17,7 +18,6 @@ constexpr int BR = 128;       // rows per CTA
 constexpr int BN = 64;        // keys per tile
 constexpr int NTHREADS = 256;
 constexpr float kLog2e = 1.4426950408889634f;
-constexpr float kLn2 = 0.6931471805599453f;
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
 
@@ -53,12 +53,7 @@ __device__ __forceinline__ uint32_t swz(int row, int chunk) {
     return (uint32_t)(row * (D * 2) + ((chunk ^ (row & 7)) << 4));
 }
 
-struct MmaArgs {
-    graft_attn_params p;
-    float* partial;     // workspace after the header: per slot BR*D floats of O, then BR of m2, BR of l
-    int target;         // CTAs the schedule aims for
-    int G;
-};
+using MmaArgs = graft_merge::AttnArgs;
 
 template <int D>
 __device__ __forceinline__ void load_kv_tile(uint32_t sK, uint32_t sV, const __nv_bfloat16* Kg, const __nv_bfloat16* Vg,
@@ -251,7 +246,7 @@ __global__ void __launch_bounds__(NTHREADS, 2) attn_mma_kernel(MmaArgs a) {
                 *reinterpret_cast<uint32_t*>(orow + i * 8 + (lane & 3) * 2) = v;
             }
             if (p.LSE && (lane & 3) == 0)
-                p.LSE[((size_t)w.b * p.Hq + w.h * G + g) * p.T_max + t] = l > 0.f ? (m * sl2 + log2f(l)) * kLn2 : -CUDART_INF_F;
+                p.LSE[((size_t)w.b * p.Hq + w.h * G + g) * p.T_max + t] = l > 0.f ? (m * sl2 + log2f(l)) * graft_merge::kLn2 : -CUDART_INF_F;
         }
     } else {
         const int slot = graft_sched::slot_of(w, w.h, w.split, w.rb);
@@ -269,83 +264,6 @@ __global__ void __launch_bounds__(NTHREADS, 2) attn_mma_kernel(MmaArgs a) {
                 base[BR * D + BR + lr] = half ? lB : lA;
             }
         }
-    }
-}
-
-// Merge kernel: one CTA per (b, h_kv, block of BR rows of the padded T_max*G row space); one warp
-// per row.  Rows of real nodes whose sequence was split are merged with the online-softmax rule
-// M = max m_i, w_i = 2^(m_i - M), O = sum w_i O_i / sum w_i l_i; rows of padding nodes are zeroed.
-template <int D>
-__global__ void __launch_bounds__(NTHREADS) attn_merge_kernel(MmaArgs a, unsigned* status) {
-    const graft_attn_params& p = a.p;
-    const int G = a.G;
-    const int nrb_max = (p.T_max * G + BR - 1) / BR;
-    int idx = blockIdx.x;
-    const int rbm = idx % nrb_max; idx /= nrb_max;
-    const int h = idx % p.Hkv;
-    const int b = idx / p.Hkv;
-    __shared__ graft_sched::Work s_work;
-    if (threadIdx.x < 32) {
-        graft_sched::Work w = graft_sched::find_work<BR, BN>(p.seq_len, p.tree_size, p.B, p.Hkv, G, p.T_max, p.S_cap,
-                                                             a.target, 0, b);
-        if (threadIdx.x == 0) {
-            s_work = w;
-            const int T = p.tree_size[b], L = p.seq_len[b];
-            if (rbm == 0 && h == 0 && (T < 0 || T > p.T_max || L < 0 || (long long)L + T > p.S_cap))
-                atomicOr(status, (unsigned)GRAFT_FLAG_BAD_SIZE);
-        }
-    }
-    __syncthreads();
-    const graft_sched::Work w = s_work;
-    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    constexpr int VPL = D / 32;      // floats per lane
-    __nv_bfloat16* Og = reinterpret_cast<__nv_bfloat16*>(p.O) + (size_t)b * p.o_stride_b + (size_t)h * G * p.o_stride_h;
-    for (int lr = warp; lr < BR; lr += NTHREADS / 32) {
-        const int r = rbm * BR + lr;
-        if (r >= p.T_max * G) break;
-        const int t = r / G, g = r % G;
-        __nv_bfloat16* orow = Og + (size_t)t * p.o_stride_t + (size_t)g * p.o_stride_h + lane * VPL;
-        float* lse = p.LSE ? p.LSE + ((size_t)b * p.Hq + h * G + g) * p.T_max + t : nullptr;
-        if (t >= w.T) {                       // padding node: zero row
-            if constexpr (VPL == 4) *reinterpret_cast<uint2*>(orow) = make_uint2(0u, 0u);
-            else *reinterpret_cast<uint32_t*>(orow) = 0u;
-            if (lse && lane == 0) *lse = -CUDART_INF_F;
-            continue;
-        }
-        if (w.nsplit <= 1) continue;          // written by the attention kernel itself
-        const int rb = r / BR, rl = r % BR;
-        float M = -CUDART_INF_F;
-        for (int s = 0; s < w.nsplit; ++s) {
-            const float* base = a.partial + (size_t)graft_sched::slot_of(w, h, s, rb) * (BR * (D + 2));
-            M = fmaxf(M, base[BR * D + rl]);
-        }
-        float acc[VPL];
-#pragma unroll
-        for (int v = 0; v < VPL; ++v) acc[v] = 0.f;
-        float den = 0.f;
-        for (int s = 0; s < w.nsplit; ++s) {
-            const float* base = a.partial + (size_t)graft_sched::slot_of(w, h, s, rb) * (BR * (D + 2));
-            const float m = base[BR * D + rl];
-            if (m == -CUDART_INF_F) continue;             // this split saw no visible key for the row
-            const float wgt = exp2f(m - M);
-            den += wgt * base[BR * D + BR + rl];
-            const float* orow_p = base + (size_t)rl * D + lane * VPL;
-            if constexpr (VPL == 4) {
-                const float4 x = *reinterpret_cast<const float4*>(orow_p);
-                acc[0] += wgt * x.x; acc[1] += wgt * x.y; acc[2] += wgt * x.z; acc[3] += wgt * x.w;
-            } else {
-                const float2 x = *reinterpret_cast<const float2*>(orow_p);
-                acc[0] += wgt * x.x; acc[1] += wgt * x.y;
-            }
-        }
-        const float inv = den > 0.f ? 1.f / den : 0.f;
-        if constexpr (VPL == 4) {
-            *reinterpret_cast<uint2*>(orow) = make_uint2(pack_bf16(acc[0] * inv, acc[1] * inv),
-                                                         pack_bf16(acc[2] * inv, acc[3] * inv));
-        } else {
-            *reinterpret_cast<uint32_t*>(orow) = pack_bf16(acc[0] * inv, acc[1] * inv);
-        }
-        if (lse && lane == 0) *lse = den > 0.f ? (M + log2f(den)) * kLn2 : -CUDART_INF_F;
     }
 }
 
@@ -374,10 +292,7 @@ static int launch(graft_ctx* ctx, const graft_attn_params* p, cudaStream_t strea
     const size_t smem = (size_t)BR * D * 2 + 4 * (size_t)BN * D * 2;
     attn_mma_kernel<D><<<grid, NTHREADS, smem, stream>>>(a);
     GRAFT_CHECK_CUDA(cudaGetLastError());
-    const int nrb_max = (p->T_max * a.G + BR - 1) / BR;
-    attn_merge_kernel<D><<<p->B * p->Hkv * nrb_max, NTHREADS, 0, stream>>>(a, ctx->status);
-    GRAFT_CHECK_CUDA(cudaGetLastError());
-    return GRAFT_OK;
+    return graft_merge::launch<D, BR, BN>(a, ctx->status, stream);
 }
 
 int graft_attn_mma_init() {

@@ -53,7 +53,8 @@ def check_attn(orc, w, vs, tree, rows=None):
         assert (O[~valid] == 0).all()                                                # padding rows are zero
         lse_valid = np.broadcast_to(valid[:, None, :], LSE.shape)
         assert np.isneginf(LSE[~lse_valid]).all()
-        lse_err = np.abs(LSE - out["LSE"])[lse_valid]
+        with np.errstate(invalid="ignore"):
+            lse_err = np.abs(LSE - out["LSE"])[lse_valid]
     else:
         err = np.stack([np.abs(O[b, t, h] - out["O"][b, t, h]) for b, t, h in rows])
         lse_err = np.array([abs(LSE[b, h, t] - out["LSE"][b, h, t]) for b, t, h in rows])
@@ -182,7 +183,7 @@ def test_mask_locality_on_device(orc, G, Step, variant):
     vs.Vc[0, :, 200 + u] += 2.0
     vs.Kc[0, :, 200 + u] *= -1.0
     vs.attn(variant_id(G, variant))
-    changed = (vs.O != base).flatten(2).any(-1).any(-1)[0].cpu().numpy()          # [T_max]
+    changed = (vs.O != base).flatten(2).any(-1)[0].cpu().numpy()          # [T_max]
     anc = tree["tree_anc"][0]
     for t in range(30):
         assert changed[t] == bool((int(anc[t]) >> u) & 1), t
