@@ -29,7 +29,7 @@ __device__ __forceinline__ uint32_t pack2(float lo, float hi) {
     return *reinterpret_cast<uint32_t*>(&v);
 }
 
-template <int D, int BR, int BN>
+template <int D, int BR, int BN, bool FLOOR>
 __global__ void __launch_bounds__(kRowsPerCta * 32) merge_kernel(AttnArgs a, unsigned* status) {
     const graft_attn_params& p = a.p;
     const int G = a.G;
@@ -41,7 +41,7 @@ __global__ void __launch_bounds__(kRowsPerCta * 32) merge_kernel(AttnArgs a, uns
     const int b = idx / p.Hkv;
     __shared__ graft_sched::Work s_work;
     if (threadIdx.x < 32) {
-        graft_sched::Work w = graft_sched::find_work<BR, BN>(p.seq_len, p.tree_size, p.B, p.Hkv, G, p.T_max, p.S_cap,
+        graft_sched::Work w = graft_sched::find_work<BR, BN, FLOOR>(p.seq_len, p.tree_size, p.B, p.Hkv, G, p.T_max, p.S_cap,
                                                              a.target, 0, b);
         if (threadIdx.x == 0) {
             s_work = w;
@@ -113,10 +113,10 @@ __global__ void __launch_bounds__(kRowsPerCta * 32) merge_kernel(AttnArgs a, uns
     if (lse && lane == 0) *lse = den > 0.f ? (M + log2f(den)) * kLn2 : -CUDART_INF_F;
 }
 
-template <int D, int BR, int BN>
+template <int D, int BR, int BN, bool FLOOR = false>
 static int launch(const AttnArgs& a, unsigned* status, cudaStream_t stream) {
     const int groups = (a.p.T_max * a.G + kRowsPerCta - 1) / kRowsPerCta;
-    merge_kernel<D, BR, BN><<<a.p.B * a.p.Hkv * groups, kRowsPerCta * 32, 0, stream>>>(a, status);
+    merge_kernel<D, BR, BN, FLOOR><<<a.p.B * a.p.Hkv * groups, kRowsPerCta * 32, 0, stream>>>(a, status);
     GRAFT_CHECK_CUDA(cudaGetLastError());
     return GRAFT_OK;
 }

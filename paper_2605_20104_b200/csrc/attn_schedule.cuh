@@ -30,7 +30,10 @@ __device__ __forceinline__ void seq_dims(const int32_t* seq_len, const int32_t* 
     if (T < 0 || T > T_max || L < 0 || (long long)L + T > (long long)S_cap) { L = 0; T = 0; }
 }
 
-template <int BR, int BN>
+// FLOOR = false: ceil(ntiles / chunk) pieces (a little over `target` CTAs, for kernels that run several
+// CTAs per SM in waves); FLOOR = true: floor(ntiles / chunk) pieces, so the grid stays within `target`
+// whenever no sequence is shorter than one chunk (for one-CTA-per-SM kernels that must fit one wave).
+template <int BR, int BN, bool FLOOR>
 __device__ __forceinline__ void seq_shape(int L, int T, int G, int chunk, int& ntiles, int& nrb, int& nsplit,
                                           int& per) {
     ntiles = T > 0 ? (L + T + BN - 1) / BN : 0;
@@ -38,7 +41,7 @@ __device__ __forceinline__ void seq_shape(int L, int T, int G, int chunk, int& n
     nsplit = 0;
     per = 0;
     if (ntiles > 0) {
-        const int want = (ntiles + chunk - 1) / chunk;
+        const int want = FLOOR ? max(1, ntiles / chunk) : (ntiles + chunk - 1) / chunk;
         per = (ntiles + want - 1) / want;
         nsplit = (ntiles + per - 1) / per;       // every split non-empty
     }
@@ -65,7 +68,7 @@ __device__ __forceinline__ int chunk_size(const int32_t* seq_len, const int32_t*
 // Maps CTA `cta` to its work.  Called by a full warp; every lane returns the same Work.
 // With want_b >= 0 the lookup is by sequence instead (used by the merge kernel): first_slot,
 // nsplit, nrb, L, T of sequence want_b.
-template <int BR, int BN>
+template <int BR, int BN, bool FLOOR = false>
 __device__ __forceinline__ Work find_work(const int32_t* seq_len, const int32_t* tree_size, int B, int Hkv, int G,
                                           int T_max, int S_cap, int target, int cta, int want_b) {
     const int lane = threadIdx.x & 31;
@@ -79,7 +82,7 @@ __device__ __forceinline__ Work find_work(const int32_t* seq_len, const int32_t*
         int L = 0, T = 0, ntiles = 0, nrb = 0, nsplit = 0, per = 0, cnt = 0;
         if (b < B) {
             seq_dims(seq_len, tree_size, b, T_max, S_cap, L, T);
-            seq_shape<BR, BN>(L, T, G, chunk, ntiles, nrb, nsplit, per);
+            seq_shape<BR, BN, FLOOR>(L, T, G, chunk, ntiles, nrb, nsplit, per);
             cnt = Hkv * nrb * nsplit;
         }
         int incl = cnt;
