@@ -142,7 +142,13 @@ class Context:
         return int(f.value)
 
 
-def graft_build_tree(ctx: Context, *, mode: int, K_max: int, V: int, k: int, S_cap: int,
+def launch(name: str, ctx: Context, params) -> None:
+    """Issues entry point `name` with an already marshalled params struct (see *_params below);
+    lets a caller that repeats a call with the same buffers skip the marshalling."""
+    _check(getattr(_lib, name)(ctx.handle, C.byref(params), _stream()), name)
+
+
+def build_tree_params(*, mode: int, K_max: int, V: int, k: int, S_cap: int,
                      draft_token, draft_parent, draft_score, n_draft, seq_len, M=None, keep_count=None, k_max=None,
                      gate_depth: int = 0, node_threshold: float = 0.0, ckpt_depth=None, ckpt_keep=None,
                      ckpt_log_tau=None, tmpl_offset=None, tmpl_parent=None, tmpl_rank=None,
@@ -161,11 +167,15 @@ def graft_build_tree(ctx: Context, *, mode: int, K_max: int, V: int, k: int, S_c
                     tmpl_parent=_ptr(tmpl_parent, i32), tmpl_rank=_ptr(tmpl_rank, i32),
                     tree_token=_ptr(tree_token, i32), tree_parent=_ptr(tree_parent, i32), tree_pos=_ptr(tree_pos, i32),
                     tree_src=_ptr(tree_src, i32), tree_anc=_ptr(tree_anc, torch.int64), tree_size=_ptr(tree_size, i32))
-    _check(_lib.graft_build_tree(ctx.handle, C.byref(p), _stream()), "graft_build_tree")
+    return p
 
 
-def graft_tree_verify_attn(ctx: Context, *, Q, Kc, Vc, O, seq_len, tree_size, tree_anc, scale: float,
-                           LSE=None, variant: int = ATTN_AUTO) -> None:
+def graft_build_tree(ctx: Context, **kw) -> None:
+    launch("graft_build_tree", ctx, build_tree_params(**kw))
+
+
+def tree_verify_attn_params(*, Q, Kc, Vc, O, seq_len, tree_size, tree_anc, scale: float,
+                            LSE=None, variant: int = ATTN_AUTO) -> AttnParams:
     """Q, O: bf16 [B, T_max, Hq, d]; Kc, Vc: bf16 [B, Hkv, S_cap, d] (any strides with a contiguous
     last axis); tree_anc: int64 [B, T_max] holding the 64-bit masks."""
     bf = torch.bfloat16
@@ -180,21 +190,29 @@ def graft_tree_verify_attn(ctx: Context, *, Q, Kc, Vc, O, seq_len, tree_size, tr
                    O=_ptr(O, bf), o_stride_b=O.stride(0), o_stride_t=O.stride(1), o_stride_h=O.stride(2),
                    LSE=_ptr(LSE, torch.float32), seq_len=_ptr(seq_len, torch.int32),
                    tree_size=_ptr(tree_size, torch.int32), tree_anc=_ptr(tree_anc, torch.int64))
-    _check(_lib.graft_tree_verify_attn(ctx.handle, C.byref(p), _stream()), "graft_tree_verify_attn")
+    return p
 
 
-def graft_accept(ctx: Context, *, tree_token, tree_parent, tree_anc, tree_size, target_next, n_acc, path, best_node,
-                 bonus) -> None:
+def graft_tree_verify_attn(ctx: Context, **kw) -> None:
+    launch("graft_tree_verify_attn", ctx, tree_verify_attn_params(**kw))
+
+
+def accept_params(*, tree_token, tree_parent, tree_anc, tree_size, target_next, n_acc, path, best_node,
+                  bonus) -> AcceptParams:
     i32 = torch.int32
     B, T_max = tree_token.shape
     p = AcceptParams(B=B, T_max=T_max, tree_token=_ptr(tree_token, i32), tree_parent=_ptr(tree_parent, i32),
                      tree_anc=_ptr(tree_anc, torch.int64), tree_size=_ptr(tree_size, i32),
                      target_next=_ptr(target_next, i32), n_acc=_ptr(n_acc, i32), path=_ptr(path, i32),
                      best_node=_ptr(best_node, i32), bonus=_ptr(bonus, i32))
-    _check(_lib.graft_accept(ctx.handle, C.byref(p), _stream()), "graft_accept")
+    return p
 
 
-def graft_compact_kv(ctx: Context, *, Kc, Vc, seq_len, n_acc, path, new_seq_len) -> None:
+def graft_accept(ctx: Context, **kw) -> None:
+    launch("graft_accept", ctx, accept_params(**kw))
+
+
+def compact_kv_params(*, Kc, Vc, seq_len, n_acc, path, new_seq_len) -> CompactParams:
     """Kc, Vc: bf16 [B, Hkv, S_cap, d] or [n_layers, B, Hkv, S_cap, d], compacted in place."""
     bf, i32 = torch.bfloat16, torch.int32
     if Kc.dim() == 4:
@@ -207,4 +225,8 @@ def graft_compact_kv(ctx: Context, *, Kc, Vc, seq_len, n_acc, path, new_seq_len)
                       kv_stride_b=Kc.stride(off), kv_stride_h=Kc.stride(off + 1), kv_stride_s=Kc.stride(off + 2),
                       Kc=_ptr(Kc, bf), Vc=_ptr(Vc, bf), seq_len=_ptr(seq_len, i32), n_acc=_ptr(n_acc, i32),
                       path=_ptr(path, i32), new_seq_len=_ptr(new_seq_len, i32))
-    _check(_lib.graft_compact_kv(ctx.handle, C.byref(p), _stream()), "graft_compact_kv")
+    return p
+
+
+def graft_compact_kv(ctx: Context, **kw) -> None:
+    launch("graft_compact_kv", ctx, compact_kv_params(**kw))

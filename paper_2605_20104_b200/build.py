@@ -23,6 +23,10 @@ def _newest_source() -> float:
 
 
 def build(force: bool = False, verbose: bool = False) -> str:
+    flags = list(NVCC_FLAGS)
+    if os.environ.get("GRAFT_TC_EXPERIMENTS"):      # ablation switches and phase timers of the tcgen05 kernel
+        flags.append("-DGRAFT_TC_EXPERIMENTS")
+        force = True
     if not force and os.path.exists(LIB) and os.path.getmtime(LIB) >= _newest_source():
         return LIB
     nvcc = os.environ.get("NVCC", "/usr/local/cuda/bin/nvcc")
@@ -30,7 +34,7 @@ def build(force: bool = False, verbose: bool = False) -> str:
     procs = []
     for src in SOURCES:
         obj = os.path.join(CSRC, src.replace(".cu", ".o"))
-        cmd = [nvcc, *NVCC_FLAGS, "-c", os.path.join(CSRC, src), "-o", obj]
+        cmd = [nvcc, *flags, "-c", os.path.join(CSRC, src), "-o", obj]
         if verbose:
             cmd.insert(1, "-Xptxas")
             cmd.insert(2, "-v")

@@ -22,6 +22,7 @@ struct AttnArgs {
     float* partial;     // workspace after the header
     int target;         // CTAs the schedule aims for
     int G;
+    int dbg;            // experiment switches (0 in production)
 };
 
 __device__ __forceinline__ uint32_t pack2(float lo, float hi) {

@@ -288,6 +288,7 @@ static int launch(graft_ctx* ctx, const graft_attn_params* p, cudaStream_t strea
     a.partial = reinterpret_cast<float*>(reinterpret_cast<char*>(ctx->ws) + GRAFT_WS_HEADER);
     a.target = target_ctas(ctx->num_sms);
     a.G = p->Hq / p->Hkv;
+    a.dbg = 0;
     const int grid = max_slots(ctx->num_sms, p->B, p->Hq, p->Hkv, p->T_max);
     const size_t smem = (size_t)BR * D * 2 + 4 * (size_t)BN * D * 2;
     attn_mma_kernel<D><<<grid, NTHREADS, smem, stream>>>(a);

@@ -11,9 +11,11 @@
 //   warps 4-7   softmax of row block 0: thread i <-> TMEM lane i <-> row i
 //   warps 8-11  softmax of row block 1
 // The two row blocks ping-pong: while one block's softmax runs on the SIMT pipes, the tensor pipe
-// works on the other block.  TMEM columns: S0 [0,128) S1 [128,256) O0 [256,384) O1 [384,512); P (bf16)
-// overwrites the first 64 columns of its S.  tcgen05.mma instructions of one thread execute in
-// issue order, so Q K^T of the next tile may be issued right behind P V of the current one.
+// works on the other block (its P V of this tile, then its Q K^T of the next).  TMEM columns:
+// S0 [0,128) S1 [128,256) O0 [256,384) O1 [384,512); P (bf16) overwrites the first 64 columns of
+// its S.  tcgen05.mma instructions of one thread execute in issue order, so the Q K^T that refills S
+// may be issued right behind the P V that reads P from it, and "S of tile j+1 is ready" implies
+// "P V of tile j is complete" (O is quiescent whenever a softmax thread rescales it).
 //
 // Softmax keeps a reference maximum per row and rescales O only when the maximum grows by more
 // than 2^8 (P then stays below 256, harmless in bf16/fp32); the row sum absorbs the same factor.
@@ -25,7 +27,9 @@
 // waiting anywhere in the CTA, drains its outstanding copies, frees TMEM and returns.
 #include <cuda.h>
 #include <cuda_bf16.h>
+#include <cuda_fp16.h>
 #include <math_constants.h>
+#include <stdlib.h>
 #include "attn_merge.cuh"
 #include "attn_schedule.cuh"
 #include "graft_internal.cuh"
@@ -46,7 +50,15 @@ constexpr long long kWaitCycles = 1ll << 31;  // about a second
 
 using TcArgs = graft_merge::AttnArgs;
 
-// barrier indices
+// Experiment switches (component ablations, phase timers) exist only in builds with
+// -DGRAFT_TC_EXPERIMENTS; in the library build every DBG(x) is a compile-time false.
+#ifdef GRAFT_TC_EXPERIMENTS
+#define DBG(x) (a.dbg & (x))
+#else
+#define DBG(x) false
+#endif
+
+// barrier indices: ring slots; S ready / P ready per row block; O final
 enum { BAR_FULL = 0, BAR_EMPTY = NSLOT, BAR_S = 2 * NSLOT, BAR_P = 2 * NSLOT + 2, BAR_O = 2 * NSLOT + 4, BAR_COUNT = 2 * NSLOT + 5 };
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
@@ -133,6 +145,35 @@ __device__ __forceinline__ void tmem_st16(uint32_t taddr, const uint32_t (&r)[16
 __device__ __forceinline__ void tmem_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
 __device__ __forceinline__ void tmem_wait_st() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
 
+__device__ __forceinline__ float fmax3(float a, float b, float c) {
+    float d;
+    asm("max.f32 %0, %1, %2, %3;" : "=f"(d) : "f"(a), "f"(b), "f"(c));
+    return d;
+}
+__device__ __forceinline__ float ex2(float x) {
+    float y;
+    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+    return y;
+}
+// two fp32 lanes in one 64-bit register, for the packed fma / add of sm_100
+__device__ __forceinline__ unsigned long long pack2f(float lo, float hi) {
+    unsigned long long r;
+    asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "f"(lo), "f"(hi));
+    return r;
+}
+__device__ __forceinline__ void unpack2f(unsigned long long v, float& lo, float& hi) {
+    asm("mov.b64 {%0, %1}, %2;" : "=f"(lo), "=f"(hi) : "l"(v));
+}
+__device__ __forceinline__ unsigned long long ffma2(unsigned long long a, unsigned long long b, unsigned long long c) {
+    unsigned long long d;
+    asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(d) : "l"(a), "l"(b), "l"(c));
+    return d;
+}
+__device__ __forceinline__ unsigned long long fadd2(unsigned long long a, unsigned long long b) {
+    unsigned long long d;
+    asm("add.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
+    return d;
+}
 __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
     __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
     return *reinterpret_cast<uint32_t*>(&v);
@@ -141,15 +182,20 @@ __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
 // Shared-memory matrix descriptor, 128-byte swizzle, 8-row groups 1024 bytes apart (SBO).
 // lbo_bytes: K-major operands ignore it (16 is the canonical value); MN-major operands use it as the
 // distance between 64-element column blocks.
-__device__ __forceinline__ uint64_t smem_desc(uint32_t addr, uint32_t lbo_bytes) {
-    return (uint64_t)((addr >> 4) & 0x3FFFu) | ((uint64_t)((lbo_bytes >> 4) & 0x3FFFu) << 16) |
-           ((uint64_t)((1024u >> 4) & 0x3FFFu) << 32) | (1ull << 46) | (2ull << 61);
+constexpr uint64_t desc_fixed(uint32_t lbo_bytes) {
+    return ((uint64_t)((lbo_bytes >> 4) & 0x3FFFu) << 16) | ((uint64_t)((1024u >> 4) & 0x3FFFu) << 32) | (1ull << 46) |
+           (2ull << 61);
 }
+constexpr uint64_t kDescKMajor = desc_fixed(16);            // Q and K tiles
+constexpr uint64_t kDescVMajor = desc_fixed(HALF_BYTES);    // V tile as an MN-major operand
+// the start-address field holds (shared address >> 4); shared addresses stay below 2^18, so adding a
+// 16-byte-unit offset to a descriptor's low word never carries out of the field
+__device__ __forceinline__ uint64_t smem_desc(uint64_t fixed, uint32_t addr16) { return fixed | (uint64_t)addr16; }
 
-// instruction descriptor of kind::f16: fp32 accumulate, bf16 A and B, M = 128, N = 128
+// instruction descriptors of kind::f16: fp32 accumulate, bf16 A and B, M = 128
 constexpr uint32_t kIdescBase = (1u << 4) | (1u << 7) | (1u << 10) | ((128u >> 3) << 17) | ((128u >> 4) << 24);
-constexpr uint32_t kIdescQK = kIdescBase;                // A, B both K-major
-constexpr uint32_t kIdescPV = kIdescBase | (1u << 16);   // B (= V) MN-major
+constexpr uint32_t kIdescQK = kIdescBase;                // N = 128 keys; A, B both K-major
+constexpr uint32_t kIdescPV = kIdescBase | (1u << 16);   // N = d = 128; B (= V) MN-major
 
 __global__ void __launch_bounds__(NTHREADS, 1)
 attn_tc_kernel(const __grid_constant__ CUtensorMap kmap, const __grid_constant__ CUtensorMap vmap, TcArgs a, unsigned* status) {
@@ -162,20 +208,43 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap kmap, const __grid_constant__
     const graft_attn_params& p = a.p;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
 
-    if (warp == 0) {
-        graft_sched::Work w0 = graft_sched::find_work<BR, BN, true>(p.seq_len, p.tree_size, p.B, p.Hkv, a.G, p.T_max, p.S_cap,
-                                                                   a.target, blockIdx.x, -1);
-        if (lane == 0) { s_work = w0; s_abort = 0; }
-    }
-    __syncthreads();
-    const graft_sched::Work w = s_work;
-    if (!w.valid) return;
-
     const uint32_t sQ = (smem_u32(smem_raw) + 1023u) & ~1023u;
     const uint32_t sRing = sQ + 2 * TILE_BYTES;
     const uint32_t bar0 = smem_u32(s_bar);
     auto bar = [&](int i) { return bar0 + 8u * (uint32_t)i; };
     volatile int* abort_flag = &s_abort;
+    // ring load n: K (n even) or V (n odd) of this CTA's tile n / 2
+    auto issue_load = [&](const graft_sched::Work& ww, int n) {
+        const int slot = n % NSLOT;
+        const uint32_t dst = sRing + slot * TILE_BYTES;
+        const int key0 = (ww.tile_lo + (n >> 1)) * BN;
+        const CUtensorMap* map = (n & 1) ? &vmap : &kmap;
+        mbar_expect_tx(bar(BAR_FULL + slot), TILE_BYTES);
+        tma_load_4d(dst, map, 0, key0, ww.h, ww.b, bar(BAR_FULL + slot));
+        tma_load_4d(dst + HALF_BYTES, map, 64, key0, ww.h, ww.b, bar(BAR_FULL + slot));
+    };
+
+    if (warp == 0) {
+        graft_sched::Work w0 = graft_sched::find_work<BR, BN, true>(p.seq_len, p.tree_size, p.B, p.Hkv, a.G, p.T_max, p.S_cap,
+                                                                   a.target, blockIdx.x, -1);
+        if (lane == 0) {
+            s_work = w0;
+            s_abort = 0;
+            if (w0.valid) {
+                // barriers, then the first ring loads at once: their latency overlaps the Q load below
+                for (int i = 0; i < NSLOT; ++i) { mbar_init(bar(BAR_FULL + i), 1); mbar_init(bar(BAR_EMPTY + i), 1); }
+                for (int i = 0; i < 2; ++i) { mbar_init(bar(BAR_S + i), 1); mbar_init(bar(BAR_P + i), 4); }
+                mbar_init(bar(BAR_O), 1);
+                asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+                const int n_first = DBG(128) ? 0 : min(NSLOT, 2 * (w0.tile_hi - w0.tile_lo));
+                for (int n = 0; n < n_first; ++n) issue_load(w0, n);
+            }
+        }
+    }
+    __syncthreads();
+    const graft_sched::Work w = s_work;
+    if (!w.valid) return;
+    if (DBG(128)) return;
 
     const int G = a.G;
     const int R = w.T * G;
@@ -184,12 +253,6 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap kmap, const __grid_constant__
     const int n_keys = w.L + w.T;
     const int nt = w.tile_hi - w.tile_lo;
 
-    if (threadIdx.x == 0) {
-        for (int i = 0; i < NSLOT; ++i) { mbar_init(bar(BAR_FULL + i), 1); mbar_init(bar(BAR_EMPTY + i), 1); }
-        for (int i = 0; i < 2; ++i) { mbar_init(bar(BAR_S + i), 1); mbar_init(bar(BAR_P + i), 128); }
-        mbar_init(bar(BAR_O), 1);
-        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
-    }
     if (warp == 1) {
         asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&s_tmem)), "r"(512u) : "memory");
         asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
@@ -199,17 +262,28 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap kmap, const __grid_constant__
     {
         const __nv_bfloat16* Qg = reinterpret_cast<const __nv_bfloat16*>(p.Q) + (size_t)w.b * p.q_stride_b +
                                   (size_t)w.h * G * p.q_stride_h;
-        for (int c = threadIdx.x; c < BR * 16; c += NTHREADS) {
+        constexpr int PER = (BR * 16 + NTHREADS - 1) / NTHREADS;
+        uint4 v[PER];
+#pragma unroll
+        for (int q = 0; q < PER; ++q) {
+            const int c = threadIdx.x + q * NTHREADS;
             const int rl = c >> 4, ch = c & 15;
             const int r = row0 + rl;
-            uint4 v = make_uint4(0u, 0u, 0u, 0u);
-            if (r < R) {
+            v[q] = make_uint4(0u, 0u, 0u, 0u);
+            if (c < BR * 16 && r < R) {
                 const int t = r / G, g = r % G;
-                v = *reinterpret_cast<const uint4*>(Qg + (size_t)t * p.q_stride_t + (size_t)g * p.q_stride_h + ch * 8);
+                v[q] = *reinterpret_cast<const uint4*>(Qg + (size_t)t * p.q_stride_t + (size_t)g * p.q_stride_h + ch * 8);
             }
-            const int blk = rl >> 7, rr = rl & 127;
-            const uint32_t dst = sQ + blk * TILE_BYTES + (ch >> 3) * HALF_BYTES + rr * 128 + (((ch & 7) ^ (rr & 7)) << 4);
-            asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(dst), "r"(v.x), "r"(v.y), "r"(v.z), "r"(v.w) : "memory");
+        }
+#pragma unroll
+        for (int q = 0; q < PER; ++q) {
+            const int c = threadIdx.x + q * NTHREADS;
+            if (c < BR * 16) {
+                const int rl = c >> 4, ch = c & 15;
+                const int blk = rl >> 7, rr = rl & 127;
+                const uint32_t dst = sQ + blk * TILE_BYTES + (ch >> 3) * HALF_BYTES + rr * 128 + (((ch & 7) ^ (rr & 7)) << 4);
+                asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(dst), "r"(v[q].x), "r"(v[q].y), "r"(v[q].z), "r"(v[q].w) : "memory");
+            }
         }
         fence_async_smem();
     }
@@ -221,61 +295,74 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap kmap, const __grid_constant__
     if (warp == 0) {
         // =============================== TMA producer ===============================
         if (lane == 0) {
-            int n = 0;
-            for (int j = 0; j < nt; ++j) {
-                const int key0 = (w.tile_lo + j) * BN;
-                for (int which = 0; which < 2; ++which, ++n) {
-                    const int slot = n % NSLOT, use = n / NSLOT;
-                    if (use > 0) mbar_wait(bar(BAR_EMPTY + slot), (use - 1) & 1, abort_flag, status);
-                    const uint32_t dst = sRing + slot * TILE_BYTES;
-                    mbar_expect_tx(bar(BAR_FULL + slot), TILE_BYTES);
-                    const CUtensorMap* map = which ? &vmap : &kmap;
-                    tma_load_4d(dst, map, 0, key0, w.h, w.b, bar(BAR_FULL + slot));
-                    tma_load_4d(dst + HALF_BYTES, map, 64, key0, w.h, w.b, bar(BAR_FULL + slot));
+            const int n_total = 2 * nt;
+            int n = min(NSLOT, n_total);                      // the first loads were issued before the Q load
+            if (DBG(64)) {                                 // experiment: loads only, reuse a slot as soon as it landed
+                for (; n < n_total; ++n) {
+                    mbar_wait(bar(BAR_FULL + n % NSLOT), (n / NSLOT - 1) & 1, abort_flag, status);
+                    issue_load(w, n);
                 }
+            } else
+            for (; n < n_total; ++n) {
+                mbar_wait(bar(BAR_EMPTY + n % NSLOT), (n / NSLOT - 1) & 1, abort_flag, status);
+                issue_load(w, n);
             }
             // drain: every copy issued must have landed before the CTA may exit
             for (int m = max(0, n - NSLOT); m < n; ++m) mbar_wait(bar(BAR_FULL + m % NSLOT), (m / NSLOT) & 1, abort_flag, status);
         }
+    } else if (DBG(64)) {
     } else if (warp == 1) {
         // =============================== MMA issuer ===============================
         if (lane == 0) {
             auto wait_full = [&](int n) { mbar_wait(bar(BAR_FULL + n % NSLOT), (n / NSLOT) & 1, abort_flag, status); };
-            auto issue_qk = [&](int blk, int n) {
-                const uint32_t sK = sRing + (n % NSLOT) * TILE_BYTES;
-                const uint32_t sQb = sQ + blk * TILE_BYTES;
+            // S[blk] = Q[blk] K(j)^T
+            auto issue_qk = [&](int blk, int j) {
+                const uint32_t sK16 = (sRing + ((2 * j) % NSLOT) * TILE_BYTES) >> 4;
+                const uint32_t sQ16 = (sQ + blk * TILE_BYTES) >> 4;
+                if (!DBG(2))
 #pragma unroll
                 for (int k = 0; k < D / 16; ++k) {
-                    const uint32_t off = (k >> 2) * HALF_BYTES + (k & 3) * 32;
-                    mma_ss(tmem + blk * 128, smem_desc(sQb + off, 16), smem_desc(sK + off, 16), kIdescQK, k > 0);
+                    const uint32_t off16 = ((k >> 2) * HALF_BYTES + (k & 3) * 32) >> 4;
+                    mma_ss(tmem + blk * 128, smem_desc(kDescKMajor, sQ16 + off16), smem_desc(kDescKMajor, sK16 + off16), kIdescQK, k > 0);
                 }
+                tc_commit(bar(BAR_S + blk));
+                if (blk == nblk - 1) tc_commit(bar(BAR_EMPTY + (2 * j) % NSLOT));          // K tile fully read
             };
-            auto issue_pv = [&](int blk, int n, bool acc) {
-                const uint32_t sV = sRing + (n % NSLOT) * TILE_BYTES;
+            // O[blk] (+)= P[blk] V(j)
+            auto issue_pv = [&](int blk, int j) {
+                const uint32_t sV16 = (sRing + ((2 * j + 1) % NSLOT) * TILE_BYTES) >> 4;
+                if (!DBG(4))
 #pragma unroll
                 for (int k = 0; k < BN / 16; ++k)
-                    mma_ts(tmem + 256 + blk * 128, tmem + blk * 128 + k * 8, smem_desc(sV + k * 2048, HALF_BYTES), kIdescPV,
-                           (acc || k > 0) ? 1u : 0u);
+                    mma_ts(tmem + 256 + blk * 128, tmem + blk * 128 + k * 8, smem_desc(kDescVMajor, sV16 + k * (2048 >> 4)), kIdescPV,
+                           (j > 0 || k > 0) ? 1u : 0u);
+                if (blk == nblk - 1) tc_commit(bar(BAR_EMPTY + (2 * j + 1) % NSLOT));      // V tile fully read
             };
             wait_full(0);
             tc_fence_after();
-            for (int blk = 0; blk < nblk; ++blk) { issue_qk(blk, 0); tc_commit(bar(BAR_S + blk)); }
-            tc_commit(bar(BAR_EMPTY + 0));
+            for (int blk = 0; blk < nblk; ++blk) issue_qk(blk, 0);
+            long long m_waitp = 0, m_waitf = 0, m_issue = 0, mc0 = clock64(), mc1;
+            const bool mprof = DBG(4096) && blockIdx.x == 0;
             for (int j = 0; j < nt; ++j) {
-                const int nK1 = 2 * (j + 1), nV = 2 * j + 1;
                 for (int blk = 0; blk < nblk; ++blk) {
                     mbar_wait(bar(BAR_P + blk), j & 1, abort_flag, status);
-                    if (blk == 0) wait_full(nV);
+                    if (mprof) { mc1 = clock64(); m_waitp += mc1 - mc0; mc0 = mc1; }
+                    if (blk == 0) wait_full(2 * j + 1);
+                    if (mprof) { mc1 = clock64(); m_waitf += mc1 - mc0; mc0 = mc1; }
                     tc_fence_after();
-                    issue_pv(blk, nV, j > 0);
-                    if (blk == nblk - 1) tc_commit(bar(BAR_EMPTY + nV % NSLOT));
+                    issue_pv(blk, j);
+                    if (mprof) { mc1 = clock64(); m_issue += mc1 - mc0; mc0 = mc1; }
                     if (j + 1 < nt) {
-                        if (blk == 0) { wait_full(nK1); tc_fence_after(); }
-                        issue_qk(blk, nK1);
-                        tc_commit(bar(BAR_S + blk));
-                        if (blk == nblk - 1) tc_commit(bar(BAR_EMPTY + nK1 % NSLOT));
+                        if (blk == 0) { wait_full(2 * j + 2); tc_fence_after(); }
+                        if (mprof) { mc1 = clock64(); m_waitf += mc1 - mc0; mc0 = mc1; }
+                        issue_qk(blk, j + 1);
+                        if (mprof) { mc1 = clock64(); m_issue += mc1 - mc0; mc0 = mc1; }
                     }
                 }
+            }
+            if (mprof) {
+                unsigned* dbgw = status + 24;
+                dbgw[0] = (unsigned)(m_waitp / nt); dbgw[1] = (unsigned)(m_waitf / nt); dbgw[2] = (unsigned)(m_issue / nt);
             }
             tc_commit(bar(BAR_O));
         }
@@ -294,30 +381,50 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap kmap, const __grid_constant__
             const float sl2 = p.scale * kLog2e;
             float m_ref = -CUDART_INF_F, l = 0.f;
 
+            if (DBG(8192) && blk == 1) { const long long t0 = clock64(); while (clock64() - t0 < 1700) {} }
+            long long t_wait = 0, t_p1 = 0, t_p2 = 0, t_tail = 0, tc0 = clock64(), tc1;
+            const bool prof = DBG(4096) && blockIdx.x == 0 && rl == 0;
             for (int j = 0; j < nt; ++j) {
                 const int key0 = (w.tile_lo + j) * BN;
                 const bool boundary = key0 + BN > w.L;
                 mbar_wait(bar(BAR_S + blk), j & 1, abort_flag, status);
                 tc_fence_after();
-                // pass 1: row maximum of the (masked) scores
-                float mx = -CUDART_INF_F;
-#pragma unroll 1
-                for (int c = 0; c < 4; ++c) {
-                    uint32_t v[32];
-                    tmem_ld32(tS + c * 32, v);
-                    tmem_wait_ld();
-                    if (boundary) {
+                if (prof) { tc1 = clock64(); t_wait += tc1 - tc0; tc0 = tc1; }
+                // pass 1: row maximum of the (masked) scores, 64 columns in flight at a time
+                auto mask32 = [&](uint32_t (&x)[32], int col0) {
 #pragma unroll
-                        for (int i = 0; i < 32; ++i) {
-                            const int u = key0 + c * 32 + i - w.L;
-                            const bool vis = u < 0 || (u < w.T && ((anc >> (u & 63)) & 1ull));
-                            if (vis) mx = fmaxf(mx, __uint_as_float(v[i]));
-                        }
-                    } else {
-#pragma unroll
-                        for (int i = 0; i < 32; ++i) mx = fmaxf(mx, __uint_as_float(v[i]));
+                    for (int q = 0; q < 32; ++q) {
+                        const int u = key0 + col0 + q - w.L;
+                        if (!(u < 0 || (u < w.T && ((anc >> (u & 63)) & 1ull)))) x[q] = 0xff800000u;   // -inf
                     }
+                };
+                auto max32 = [&](const uint32_t (&x)[32], float& m0, float& m1) {
+#pragma unroll
+                    for (int q = 0; q < 32; q += 4) {
+                        m0 = fmax3(m0, __uint_as_float(x[q]), __uint_as_float(x[q + 1]));
+                        m1 = fmax3(m1, __uint_as_float(x[q + 2]), __uint_as_float(x[q + 3]));
+                    }
+                };
+                float mx0 = -CUDART_INF_F, mx1 = -CUDART_INF_F;
+                if (!DBG(8)) {
+                    uint32_t x0[32], x1[32];
+                    tmem_ld32(tS, x0);
+                    tmem_ld32(tS + 32, x1);
+                    tmem_wait_ld();
+                    if (boundary) { mask32(x0, 0); mask32(x1, 32); }
+                    max32(x0, mx0, mx1);
+                    max32(x1, mx0, mx1);
+                    tmem_ld32(tS + 64, x0);
+                    tmem_ld32(tS + 96, x1);
+                    tmem_wait_ld();
+                    if (boundary) { mask32(x0, 64); mask32(x1, 96); }
+                    max32(x0, mx0, mx1);
+                    max32(x1, mx0, mx1);
+                } else {
+                    mx0 = 0.f;
                 }
+                const float mx = fmaxf(mx0, mx1);
+                if (prof) { tc1 = clock64(); t_p1 += tc1 - tc0; tc0 = tc1; }
                 // reference maximum: move it only when the scores outgrow it by more than the threshold
                 if (mx != -CUDART_INF_F && (m_ref == -CUDART_INF_F || (mx - m_ref) * sl2 > kRescaleThreshold)) {
                     if (m_ref != -CUDART_INF_F) {
@@ -325,41 +432,56 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap kmap, const __grid_constant__
                         l *= alpha;
 #pragma unroll 1
                         for (int c = 0; c < 4; ++c) {       // O of the previous tiles is complete here
-                            uint32_t v[32];
-                            tmem_ld32(tO + c * 32, v);
+                            uint32_t o[32];
+                            tmem_ld32(tO + c * 32, o);
                             tmem_wait_ld();
 #pragma unroll
-                            for (int i = 0; i < 32; ++i) v[i] = __float_as_uint(__uint_as_float(v[i]) * alpha);
-                            tmem_st32(tO + c * 32, v);
+                            for (int q = 0; q < 32; ++q) o[q] = __float_as_uint(__uint_as_float(o[q]) * alpha);
+                            tmem_st32(tO + c * 32, o);
                         }
                         tmem_wait_st();
                     }
                     m_ref = mx;
                 }
                 const float off = m_ref == -CUDART_INF_F ? 0.f : m_ref * sl2;
-                // pass 2: P = 2^(s*scale*log2e - off) as bf16 into the first 64 columns of S
-                float sum = 0.f;
-#pragma unroll 1
-                for (int c = 0; c < 4; ++c) {
-                    uint32_t v[32];
-                    tmem_ld32(tS + c * 32, v);
-                    tmem_wait_ld();
+                // pass 2: P = 2^(s*scale*log2e - off) as bf16 into the first 64 columns of S.  P chunk c
+                // (columns 16c..16c+15) only overwrites score columns that are already in registers.
+                float sum0 = 0.f, sum1 = 0.f;
+                auto exp32 = [&](const uint32_t (&x)[32], uint32_t col) {
                     uint32_t pk[16];
 #pragma unroll
-                    for (int i = 0; i < 32; i += 2) {
-                        float p0 = exp2f(__uint_as_float(v[i]) * sl2 - off);
-                        float p1 = exp2f(__uint_as_float(v[i + 1]) * sl2 - off);
-                        if (boundary) {
-                            const int u0 = key0 + c * 32 + i - w.L, u1 = u0 + 1;
-                            if (!(u0 < 0 || (u0 < w.T && ((anc >> (u0 & 63)) & 1ull)))) p0 = 0.f;
-                            if (!(u1 < 0 || (u1 < w.T && ((anc >> (u1 & 63)) & 1ull)))) p1 = 0.f;
-                        }
-                        sum += p0 + p1;
-                        pk[i >> 1] = pack_bf16(p0, p1);
+                    for (int q = 0; q < 32; q += 2) {
+                        const float p0 = ex2(fmaf(__uint_as_float(x[q]), sl2, -off));
+                        const float p1 = ex2(fmaf(__uint_as_float(x[q + 1]), sl2, -off));
+                        sum0 += p0;
+                        sum1 += p1;
+                        pk[q >> 1] = pack_bf16(p0, p1);
                     }
-                    tmem_st16(tS + c * 16, pk);
+                    tmem_st16(tS + col, pk);
+                };
+                if (DBG(1)) {
+                    uint32_t pk[16];
+#pragma unroll
+                    for (int q = 0; q < 16; ++q) pk[q] = 0x3f803f80u;
+                    if (!DBG(16)) { tmem_st16(tS, pk); tmem_st16(tS + 16, pk); tmem_st16(tS + 32, pk); tmem_st16(tS + 48, pk); }
+                    sum0 = 128.f;
+                } else {
+                    uint32_t x0[32], x1[32];
+                    tmem_ld32(tS, x0);
+                    tmem_ld32(tS + 32, x1);
+                    tmem_wait_ld();
+                    if (boundary) { mask32(x0, 0); mask32(x1, 32); }
+                    exp32(x0, 0);
+                    tmem_ld32(tS + 64, x0);
+                    exp32(x1, 16);
+                    tmem_ld32(tS + 96, x1);
+                    tmem_wait_ld();
+                    if (boundary) { mask32(x0, 64); mask32(x1, 96); }
+                    exp32(x0, 32);
+                    exp32(x1, 48);
                 }
-                l += sum;
+                l += sum0 + sum1;
+                if (prof) { tc1 = clock64(); t_p2 += tc1 - tc0; tc0 = tc1; }
                 tmem_wait_st();
                 // last tile of the sequence: zero the V rows of slots that hold no key of this tree
                 if (blk == 0 && key0 + BN > n_keys) {
@@ -376,7 +498,14 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap kmap, const __grid_constant__
                     fence_async_smem();
                 }
                 tc_fence_before();
-                mbar_arrive(bar(BAR_P + blk));
+                __syncwarp();
+                if (lane == 0) mbar_arrive(bar(BAR_P + blk));      // one arrival per warp
+                if (prof) { tc1 = clock64(); t_tail += tc1 - tc0; tc0 = tc1; }
+            }
+            if (prof) {
+                unsigned* dbgw = status + 8 + blk * 8;
+                dbgw[0] = (unsigned)nt; dbgw[1] = (unsigned)(t_wait / nt); dbgw[2] = (unsigned)(t_p1 / nt);
+                dbgw[3] = (unsigned)(t_p2 / nt); dbgw[4] = (unsigned)(t_tail / nt);
             }
 
             // ---- epilogue: O row from TMEM, final result or partial
@@ -495,7 +624,13 @@ int graft_attn_tc_launch(graft_ctx* ctx, const graft_attn_params* p, cudaStream_
     a.partial = reinterpret_cast<float*>(reinterpret_cast<char*>(ctx->ws) + GRAFT_WS_HEADER);
     a.target = target_ctas(ctx->num_sms);
     a.G = p->Hq / p->Hkv;
+#ifdef GRAFT_TC_EXPERIMENTS
+    a.dbg = getenv("GRAFT_TC_DEBUG") ? atoi(getenv("GRAFT_TC_DEBUG")) : 0;
+#else
+    a.dbg = 0;
+#endif
     attn_tc_kernel<<<max_ctas(ctx->num_sms, p->B, p->Hq, p->Hkv, p->T_max), NTHREADS, SMEM_DYN, stream>>>(kmap, vmap, a, ctx->status);
     GRAFT_CHECK_CUDA(cudaGetLastError());
+    if (DBG(256)) return GRAFT_OK;
     return graft_merge::launch<D, BR, BN, true>(a, ctx->status, stream);
 }

@@ -81,32 +81,48 @@ class VerifyStep:
         self.Vc = Vc.to(self.dev).contiguous()
 
     # ---- the four calls -------------------------------------------------------------------------
+    # Each call marshals its params struct once per distinct set of buffers and re-issues the
+    # cached struct afterwards, so a benchmark loop is not bound by Python-side marshalling.
+    def _cached(self, key, make):
+        cache = self.__dict__.setdefault("_params", {})
+        if key not in cache:
+            cache[key] = make()
+        return cache[key]
+
     def build(self) -> None:
+        G.launch("graft_build_tree", self.ctx, self._cached("build", self._build_params))
+
+    def _build_params(self):
         w = self.w
-        G.graft_build_tree(self.ctx, mode=w.mode, K_max=w.K_max, V=w.V, k=w.k, S_cap=w.S_cap,
+        return G.build_tree_params(mode=w.mode, K_max=w.K_max, V=w.V, k=w.k, S_cap=w.S_cap,
                            draft_token=self.draft_token, draft_parent=self.draft_parent, draft_score=self.draft_score,
                            n_draft=self.n_draft, seq_len=self.seq_len, M=self.M, keep_count=self.keep_count,
                            k_max=self.k_max, gate_depth=w.gate_depth, node_threshold=w.node_threshold,
                            ckpt_depth=self.ckpt_depth, ckpt_keep=self.ckpt_keep, ckpt_log_tau=self.ckpt_log_tau,
                            tmpl_offset=self.tmpl_offset, tmpl_parent=self.tmpl_parent, tmpl_rank=self.tmpl_rank,
                            tree_token=self.tree_token, tree_parent=self.tree_parent, tree_pos=self.tree_pos,
-                           tree_src=self.tree_src, tree_anc=self.tree_anc, tree_size=self.tree_size)
+                                   tree_src=self.tree_src, tree_anc=self.tree_anc, tree_size=self.tree_size)
 
     def attn(self, variant: int = G.ATTN_AUTO, lse: bool = True) -> None:
-        K0 = self.Kc if self.Kc.dim() == 4 else self.Kc[0]
-        V0 = self.Vc if self.Vc.dim() == 4 else self.Vc[0]
-        G.graft_tree_verify_attn(self.ctx, Q=self.Q, Kc=K0, Vc=V0, O=self.O, seq_len=self.seq_len,
-                                 tree_size=self.tree_size, tree_anc=self.tree_anc, scale=self.w.scale,
-                                 LSE=self.LSE if lse else None, variant=variant)
+        def make():
+            K0 = self.Kc if self.Kc.dim() == 4 else self.Kc[0]
+            V0 = self.Vc if self.Vc.dim() == 4 else self.Vc[0]
+            return G.tree_verify_attn_params(Q=self.Q, Kc=K0, Vc=V0, O=self.O, seq_len=self.seq_len,
+                                             tree_size=self.tree_size, tree_anc=self.tree_anc, scale=self.w.scale,
+                                             LSE=self.LSE if lse else None, variant=variant)
+        key = ("attn", self.Q.data_ptr(), self.Kc.data_ptr(), self.Vc.data_ptr(), variant, lse)
+        G.launch("graft_tree_verify_attn", self.ctx, self._cached(key, make))
 
     def accept(self) -> None:
-        G.graft_accept(self.ctx, tree_token=self.tree_token, tree_parent=self.tree_parent, tree_anc=self.tree_anc,
-                       tree_size=self.tree_size, target_next=self.target_next, n_acc=self.n_acc, path=self.path,
-                       best_node=self.best_node, bonus=self.bonus)
+        G.launch("graft_accept", self.ctx, self._cached("accept", lambda: G.accept_params(
+            tree_token=self.tree_token, tree_parent=self.tree_parent, tree_anc=self.tree_anc, tree_size=self.tree_size,
+            target_next=self.target_next, n_acc=self.n_acc, path=self.path, best_node=self.best_node, bonus=self.bonus)))
 
     def compact(self) -> None:
-        G.graft_compact_kv(self.ctx, Kc=self.Kc, Vc=self.Vc, seq_len=self.seq_len, n_acc=self.n_acc, path=self.path,
-                           new_seq_len=self.new_seq_len)
+        key = ("compact", self.Kc.data_ptr(), self.Vc.data_ptr())
+        G.launch("graft_compact_kv", self.ctx, self._cached(key, lambda: G.compact_kv_params(
+            Kc=self.Kc, Vc=self.Vc, seq_len=self.seq_len, n_acc=self.n_acc, path=self.path,
+            new_seq_len=self.new_seq_len)))
 
     def run(self, variant: int = G.ATTN_AUTO) -> None:
         self.build()
