@@ -48,7 +48,8 @@ enum {
     GRAFT_ERR_INVALID_ARG = -1,        /* null pointer, non-positive size, misaligned base or stride   */
     GRAFT_ERR_UNSUPPORTED = -2,        /* T_max > 64, d not in {64,128}, H_q % H_kv != 0, k > 16 ...    */
     GRAFT_ERR_WORKSPACE_TOO_SMALL = -3,
-    GRAFT_ERR_CUDA = -4                /* a CUDA runtime call or launch failed                          */
+    GRAFT_ERR_CUDA = -4,               /* a CUDA runtime call or launch failed                          */
+    GRAFT_ERR_SCRATCH_LIMIT = -5       /* graft_tree_verify_attn_noalloc: shape exceeds the built-in scratch */
 };
 
 /* bits of the device status word */
@@ -175,6 +176,30 @@ typedef struct {
 } graft_attn_params;
 
 int graft_tree_verify_attn(graft_ctx* ctx, const graft_attn_params* p, void* stream);
+
+/*
+ * The same attention for callers that cannot allocate device memory (the paper has no counterpart:
+ * this is a packaging variant, not a step of the method).  A caller may be unable to allocate
+ * because its process gave all device memory to a fixed pool at start-up, because it runs inside a
+ * latency-critical section where cudaMalloc's device-wide synchronisation is not acceptable, or
+ * because it is a thin shim with no allocator in reach.  No graft_ctx and no workspace are needed:
+ * the split-KV partials and the status word live in one static device array of
+ * graft_noalloc_scratch_bytes() (32 MiB) that every GPU loading this library holds until the process
+ * exits.  The call allocates nothing (no cudaMalloc, cudaFree or allocating library routine).
+ *   - p: exactly as for graft_tree_verify_attn; inputs and outputs still belong to the caller.
+ *   - device_flags_out: optional DEVICE pointer; receives the GRAFT_FLAG_* word of this call (copied on
+ *     `stream`), or NULL.
+ *   - The first call on a device (made with that device current) resolves the array's device address
+ *     and configures the kernels; make it before any stream capture.
+ *   - Shapes whose partials do not fit the array are rejected with GRAFT_ERR_SCRATCH_LIMIT before any
+ *     launch (with GRAFT_ATTN_AUTO the call falls back from the tcgen05 kernel to the register-tile
+ *     kernel when only the latter's partials fit).
+ *   - All calls on a GPU share the one array, which keeps the previous call's contents; the call clears
+ *     the status word itself.  Two calls that overlap on the GPU (different streams) race: serialise
+ *     them.
+ */
+size_t graft_noalloc_scratch_bytes(void);
+int graft_tree_verify_attn_noalloc(const graft_attn_params* p, void* stream, unsigned* device_flags_out);
 
 /* ---- graft_accept ---------------------------------------------------------------------------- */
 /*

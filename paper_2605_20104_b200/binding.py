@@ -21,14 +21,15 @@ if not os.path.exists(LIB_PATH):
                       "(the CUDA library is the only implementation, there is no fallback)")
 _lib = C.CDLL(LIB_PATH)
 
-OK, ERR_INVALID_ARG, ERR_UNSUPPORTED, ERR_WORKSPACE_TOO_SMALL, ERR_CUDA = 0, -1, -2, -3, -4
+OK, ERR_INVALID_ARG, ERR_UNSUPPORTED, ERR_WORKSPACE_TOO_SMALL, ERR_CUDA, ERR_SCRATCH_LIMIT = 0, -1, -2, -3, -4, -5
 FLAG_BAD_SIZE, FLAG_BAD_PARENT, FLAG_BAD_TOKEN, FLAG_ORPHAN = 1, 2, 4, 8
 FLAG_BUDGET, FLAG_BAD_TEMPLATE, FLAG_NAN_SCORE, FLAG_BAD_PATH, FLAG_WAIT_TIMEOUT = 16, 32, 64, 128, 256
 PRUNE_NONE, PRUNE_TOPK, PRUNE_GATED, PRUNE_NODE = 0, 1, 2, 3
 ATTN_AUTO, ATTN_MMA_SYNC, ATTN_TCGEN05 = 0, 1, 2
 
 EXPORTS = ("graft_workspace_bytes", "graft_create", "graft_destroy", "graft_status_string", "graft_device_status",
-           "graft_build_tree", "graft_tree_verify_attn", "graft_accept", "graft_compact_kv")
+           "graft_build_tree", "graft_tree_verify_attn", "graft_accept", "graft_compact_kv",
+           "graft_noalloc_scratch_bytes", "graft_tree_verify_attn_noalloc")
 
 _vp = C.c_void_p
 
@@ -78,6 +79,12 @@ for _name, _typ in (("graft_build_tree", BuildParams), ("graft_tree_verify_attn"
                     ("graft_accept", AcceptParams), ("graft_compact_kv", CompactParams)):
     getattr(_lib, _name).restype = C.c_int
     getattr(_lib, _name).argtypes = [_vp, C.POINTER(_typ), _vp]
+
+
+_lib.graft_noalloc_scratch_bytes.restype = C.c_size_t
+_lib.graft_noalloc_scratch_bytes.argtypes = []
+_lib.graft_tree_verify_attn_noalloc.restype = C.c_int
+_lib.graft_tree_verify_attn_noalloc.argtypes = [C.POINTER(AttnParams), _vp, _vp]
 
 
 class GraftError(RuntimeError):
@@ -195,6 +202,19 @@ def tree_verify_attn_params(*, Q, Kc, Vc, O, seq_len, tree_size, tree_anc, scale
 
 def graft_tree_verify_attn(ctx: Context, **kw) -> None:
     launch("graft_tree_verify_attn", ctx, tree_verify_attn_params(**kw))
+
+
+def graft_noalloc_scratch_bytes() -> int:
+    return int(_lib.graft_noalloc_scratch_bytes())
+
+
+def graft_tree_verify_attn_noalloc(*, device_flags_out=None, **kw) -> None:
+    """The attention call for callers that cannot allocate: no Context, no workspace; scratch is the
+    library's static 32 MiB device array.  Same tensor arguments as graft_tree_verify_attn.
+    device_flags_out: optional int32 CUDA tensor (1 element) that receives the call's status flags."""
+    p = tree_verify_attn_params(**kw)
+    _check(_lib.graft_tree_verify_attn_noalloc(C.byref(p), _stream(), _ptr(device_flags_out, torch.int32)),
+           "graft_tree_verify_attn_noalloc")
 
 
 def accept_params(*, tree_token, tree_parent, tree_anc, tree_size, target_next, n_acc, path, best_node,

@@ -51,6 +51,7 @@ extern "C" const char* graft_status_string(int status) {
         case GRAFT_ERR_UNSUPPORTED: return "unsupported shape or device";
         case GRAFT_ERR_WORKSPACE_TOO_SMALL: return "workspace too small";
         case GRAFT_ERR_CUDA: return "CUDA error";
+        case GRAFT_ERR_SCRATCH_LIMIT: return "shape needs more scratch than the built-in array of graft_tree_verify_attn_noalloc";
         default: return "unknown status";
     }
 }
