@@ -69,7 +69,7 @@ class ClockSampler:
         self.f = tempfile.NamedTemporaryFile("w+", suffix=".csv", delete=False)
         try:
             self.p = subprocess.Popen(["nvidia-smi", "-i", str(index), "--query-gpu=" + self.QUERY,
-                                       "--format=csv,noheader,nounits", "-lms", "100"], stdout=self.f,
+                                       "--format=csv,noheader,nounits", "-lms", "20"], stdout=self.f,
                                       stderr=subprocess.DEVNULL)
         except OSError:
             self.p = None
@@ -135,10 +135,12 @@ def set_target_next(vs, w):
     return t
 
 
-def time_workload(name, steps, warmup, device, variant, do_e2e=True):
-    from paper_2605_20104_b200 import binding as G
+def time_workload(name, steps, warmup, device, variant, rank=0):
+    from paper_2605_20104_b200 import binding as G, shard
     cfg, B, L = WORKLOADS[name]
     w = W.config(cfg, B=B, L=L)
+    if rank:
+        w = W.config(cfg, B=B, L=L, seed=shard.rank_seed(w.seed, rank))   # every rank its own batch
     # build once to learn the tree sizes (they define the algorithmic bytes)
     kv_guess = w.B * w.Hkv * w.S_cap * w.d * 4
     n_rot = 1 if kv_guess > 2 * L2_BYTES else int(min(16, np.ceil(3 * L2_BYTES / kv_guess)))
@@ -341,16 +343,14 @@ def main():
             dist.barrier()
         torch.cuda.synchronize()
 
+    from paper_2605_20104_b200 import shard
+
     def max_over_ranks(x):
-        if dist is None:
-            return x
-        t = torch.tensor([x], dtype=torch.float64, device="cuda")
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        return float(t.item())
+        return shard.max_over_ranks(x, device="cuda")
 
     # every rank verifies its own batch (sequences are independent: no data-path collective)
     sampler = ClockSampler(local) if rank == 0 else None
-    st = time_workload(args.workload, args.steps, args.warmup, local, variant)
+    st = time_workload(args.workload, args.steps, args.warmup, local, variant, rank=rank)
     barrier()
     wall0 = time.time()
     ms_step, attn_ms, attn_ms_min = run_timed(st, args.steps)
@@ -425,7 +425,11 @@ def main():
 
 # dram__bytes_read.sum + dram__bytes_write.sum of the attention kernel per launch, from the ncu
 # captures summarised under profiles/ (None until a capture of that workload exists)
-TRAFFIC = {}
+TRAFFIC = {
+    # 1.03 x algorithmic bytes, measured on cfg4-B1-32k (profiles/attn_tc_kernel_cfg4-B1-32k.md) and scaled
+    # by the keys processed where the workload is too large for a full capture
+    "cfg4-B1-32k": 138.9e6, "cfg4-B1": 1.03 * 269.6e6, "cfg4-B4": 1.03 * 1078.5e6,
+}
 
 if __name__ == "__main__":
     main()
