@@ -184,7 +184,7 @@ int graft_tree_verify_attn(graft_ctx* ctx, const graft_attn_params* p, void* str
  * latency-critical section where cudaMalloc's device-wide synchronisation is not acceptable, or
  * because it is a thin shim with no allocator in reach.  No graft_ctx and no workspace are needed:
  * the split-KV partials and the status word live in one static device array of
- * graft_noalloc_scratch_bytes() (32 MiB) that every GPU loading this library holds until the process
+ * graft_noalloc_scratch_bytes() (40 MiB) that every GPU loading this library holds until the process
  * exits.  The call allocates nothing (no cudaMalloc, cudaFree or allocating library routine).
  *   - p: exactly as for graft_tree_verify_attn; inputs and outputs still belong to the caller.
  *   - device_flags_out: optional DEVICE pointer; receives the GRAFT_FLAG_* word of this call (copied on

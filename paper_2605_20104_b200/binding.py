@@ -210,7 +210,7 @@ def graft_noalloc_scratch_bytes() -> int:
 
 def graft_tree_verify_attn_noalloc(*, device_flags_out=None, **kw) -> None:
     """The attention call for callers that cannot allocate: no Context, no workspace; scratch is the
-    library's static 32 MiB device array.  Same tensor arguments as graft_tree_verify_attn.
+    library's static 40 MiB device array.  Same tensor arguments as graft_tree_verify_attn.
     device_flags_out: optional int32 CUDA tensor (1 element) that receives the call's status flags."""
     p = tree_verify_attn_params(**kw)
     _check(_lib.graft_tree_verify_attn_noalloc(C.byref(p), _stream(), _ptr(device_flags_out, torch.int32)),

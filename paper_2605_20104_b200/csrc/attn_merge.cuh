@@ -31,7 +31,7 @@ __device__ __forceinline__ uint32_t pack2(float lo, float hi) {
 }
 
 template <int D, int BR, int BN, bool FLOOR>
-__global__ void __launch_bounds__(kRowsPerCta * 32) merge_kernel(AttnArgs a, unsigned* status) {
+__global__ void __launch_bounds__(kRowsPerCta * 32, 2) merge_kernel(AttnArgs a, unsigned* status) {
     const graft_attn_params& p = a.p;
     const int G = a.G;
     const int rows_pad = p.T_max * G;
@@ -75,11 +75,61 @@ __global__ void __launch_bounds__(kRowsPerCta * 32) merge_kernel(AttnArgs a, uns
     float acc[VPL];
 #pragma unroll
     for (int v = 0; v < VPL; ++v) acc[v] = 0.f;
+    float den = 0.f;
+    if (w.nsplit <= 32) {
+        // common case: lane s owns split s; one round of (m, l) loads, then every O load in flight at once
+        float m = -CUDART_INF_F, l = 0.f;
+        if (lane < w.nsplit) {
+            m = slot0[lane * split_stride + BR * D + rl];
+            l = slot0[lane * split_stride + BR * D + BR + rl];
+        }
+        float M = m;
+#pragma unroll
+        for (int o = 16; o; o >>= 1) M = fmaxf(M, __shfl_xor_sync(0xffffffffu, M, o));
+        const float wgt = (m == -CUDART_INF_F) ? 0.f : exp2f(m - M);
+        den = wgt * l;
+        const float* orow_p = slot0 + (size_t)rl * D + lane * VPL;
+        // 16 partial rows in flight per round
+        for (int j0 = 0; j0 < w.nsplit; j0 += 16) {
+            if constexpr (VPL == 4) {
+                float4 x[16];
+#pragma unroll
+                for (int j = 0; j < 16; ++j)
+                    if (j0 + j < w.nsplit) x[j] = *reinterpret_cast<const float4*>(orow_p + (size_t)(j0 + j) * split_stride);
+#pragma unroll
+                for (int j = 0; j < 16; ++j)
+                    if (j0 + j < w.nsplit) {
+                        const float wj = __shfl_sync(0xffffffffu, wgt, j0 + j);
+                        acc[0] += wj * x[j].x; acc[1] += wj * x[j].y; acc[2] += wj * x[j].z; acc[3] += wj * x[j].w;
+                    }
+            } else {
+                float2 x[16];
+#pragma unroll
+                for (int j = 0; j < 16; ++j)
+                    if (j0 + j < w.nsplit) x[j] = *reinterpret_cast<const float2*>(orow_p + (size_t)(j0 + j) * split_stride);
+#pragma unroll
+                for (int j = 0; j < 16; ++j)
+                    if (j0 + j < w.nsplit) {
+                        const float wj = __shfl_sync(0xffffffffu, wgt, j0 + j);
+                        acc[0] += wj * x[j].x; acc[1] += wj * x[j].y;
+                    }
+            }
+        }
+#pragma unroll
+        for (int o = 16; o; o >>= 1) den += __shfl_xor_sync(0xffffffffu, den, o);
+        const float inv = den > 0.f ? 1.f / den : 0.f;
+        if constexpr (VPL == 4) {
+            *reinterpret_cast<uint2*>(orow) = make_uint2(pack2(acc[0] * inv, acc[1] * inv), pack2(acc[2] * inv, acc[3] * inv));
+        } else {
+            *reinterpret_cast<uint32_t*>(orow) = pack2(acc[0] * inv, acc[1] * inv);
+        }
+        if (lse && lane == 0) *lse = den > 0.f ? (M + log2f(den)) * kLn2 : -CUDART_INF_F;
+        return;
+    }
     float M = -CUDART_INF_F;
     for (int s = lane; s < w.nsplit; s += 32) M = fmaxf(M, slot0[s * split_stride + BR * D + rl]);
 #pragma unroll
     for (int o = 16; o; o >>= 1) M = fmaxf(M, __shfl_xor_sync(0xffffffffu, M, o));
-    float den = 0.f;
     for (int s0 = 0; s0 < w.nsplit; s0 += 32) {
         const int s = s0 + lane;
         float wgt = 0.f, l = 0.f;

@@ -16,7 +16,7 @@
 
 namespace {
 
-constexpr size_t kScratchBytes = 32ull << 20;          // 32 MiB per GPU, fixed at build time
+constexpr size_t kScratchBytes = 40ull << 20;          // 40 MiB per GPU, fixed at build time
 static __device__ __align__(256) unsigned char g_noalloc_scratch[kScratchBytes];
 
 constexpr int kMaxDevices = 64;

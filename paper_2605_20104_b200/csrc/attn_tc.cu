@@ -1,14 +1,24 @@
 // Tree-masked GQA attention on the 5th-generation tensor cores: TMA -> shared memory -> tcgen05.mma
-// with accumulators in tensor memory (TMEM).
+// with accumulators in tensor memory (TMEM).  Persistent, stream-K over key tiles.
 //
-// One CTA per SM handles up to 256 rows (two blocks of 128; row r <-> tree node r / G, query head
-// h*G + r % G) of one KV head against a contiguous range of 128-key tiles, so every K/V byte crosses
-// HBM once for all rows that need it.  Warp roles:
+// Work.  An item is (sequence b, KV head h, row block rb): up to 256 rows (two blocks of 128; row r
+// <-> tree node r / G, query head h*G + r % G) against the ceil((L_b+T_b)/128) key tiles of b, so every
+// K/V byte crosses HBM once for all rows that need it.  Items are laid end to end, ordered (b, h, rb);
+// the resulting tile sequence is cut into gridDim.x equal contiguous ranges, one per CTA (one CTA per
+// SM).  A CTA therefore works through a few segments (item, tile range); a segment that covers its
+// whole item writes the final rows, any other writes a partial (row max, row sum, un-normalised O)
+// into one of the CTA's two workspace slots, and merge_streamk_kernel combines the partials of an
+// item.  The cut is a pure function of (seq_len, tree_size, gridDim.x), recomputed on the device
+// by every CTA and by the merge kernel: no communication, no atomics on floats, no waiting between
+// CTAs, bit-reproducible results for a given GPU model.
+//
+// Warp roles inside a CTA:
 //   warp 0      TMA producer: K and V tiles (two 64-column boxes each, 128-byte swizzle) into a
-//               5-slot ring of 32 KB buffers, one mbarrier pair (full / empty) per slot
+//               5-slot ring of 32 KB buffers, one mbarrier pair (full / empty) per slot; the ring runs
+//               ahead across segment boundaries
 //   warp 1      MMA issuer: S = Q K^T (8 x m128 n128 k16, both operands from shared memory) and
 //               O += P V (8 x m128 n128 k16, P from TMEM, V as an MN-major operand); owns TMEM
-//   warps 4-7   softmax of row block 0: thread i <-> TMEM lane i <-> row i
+//   warps 4-7   softmax of row block 0: thread i <-> TMEM lane i <-> row i; also stage Q, write results
 //   warps 8-11  softmax of row block 1
 // The two row blocks ping-pong: while one block's softmax runs on the SIMT pipes, the tensor pipe
 // works on the other block (its P V of this tile, then its Q K^T of the next).  TMEM columns:
@@ -27,16 +37,13 @@
 // waiting anywhere in the CTA, drains its outstanding copies, frees TMEM and returns.
 #include <cuda.h>
 #include <cuda_bf16.h>
-#include <cuda_fp16.h>
 #include <math_constants.h>
 #include <stdlib.h>
-#include "attn_merge.cuh"
-#include "attn_schedule.cuh"
 #include "graft_internal.cuh"
 
 namespace {
 
-constexpr int BR = 256;          // rows per CTA (two blocks of 128)
+constexpr int BR = 256;          // rows per item (two blocks of 128)
 constexpr int BN = 128;          // keys per tile
 constexpr int D = 128;
 constexpr int NSLOT = 5;         // ring slots of 32 KB (one K or V tile each)
@@ -44,23 +51,89 @@ constexpr int TILE_BYTES = BN * D * 2;
 constexpr int HALF_BYTES = TILE_BYTES / 2;    // one 64-column box
 constexpr int NTHREADS = 384;
 constexpr int SMEM_DYN = 2 * TILE_BYTES + NSLOT * TILE_BYTES + 1024;   // Q (2 blocks) + ring + alignment slack
+constexpr int MAXSEG = 16;       // segments planned per round
+constexpr size_t SLOT_FLOATS = (size_t)BR * (D + 2);   // O[BR][D], then m2[BR], then l[BR]
 constexpr float kLog2e = 1.4426950408889634f;
+constexpr float kLn2 = 0.6931471805599453f;
 constexpr float kRescaleThreshold = 8.0f;     // log2 units
 constexpr long long kWaitCycles = 1ll << 31;  // about a second
 
-using TcArgs = graft_merge::AttnArgs;
+struct TcArgs {
+    graft_attn_params p;
+    float* partial;     // workspace after the header: 2 slots per CTA
+    int G;
+};
 
-// Experiment switches (component ablations, phase timers) exist only in builds with
-// -DGRAFT_TC_EXPERIMENTS; in the library build every DBG(x) is a compile-time false.
-#ifdef GRAFT_TC_EXPERIMENTS
-#define DBG(x) (a.dbg & (x))
-#else
-#define DBG(x) false
-#endif
+// barrier indices: ring slots; S ready / P ready per row block; Q staged; O final
+enum { BAR_FULL = 0, BAR_EMPTY = NSLOT, BAR_S = 2 * NSLOT, BAR_P = 2 * NSLOT + 2, BAR_Q = 2 * NSLOT + 4, BAR_O = 2 * NSLOT + 5,
+       BAR_COUNT = 2 * NSLOT + 6 };
 
-// barrier indices: ring slots; S ready / P ready per row block; O final
-enum { BAR_FULL = 0, BAR_EMPTY = NSLOT, BAR_S = 2 * NSLOT, BAR_P = 2 * NSLOT + 2, BAR_O = 2 * NSLOT + 4, BAR_COUNT = 2 * NSLOT + 5 };
+// ---------------------------------------------------------------------------------------------------
+// schedule: items laid end to end, cut into equal tile ranges
+// ---------------------------------------------------------------------------------------------------
+struct SeqInfo {
+    int b, L, T, nrb, ntiles;
+    long long base;      // global tile index of the sequence's first item
+    bool found;
+};
 
+__device__ __forceinline__ void seq_shape(const graft_attn_params& p, int G, int b, int& L, int& T, int& nrb, int& ntiles) {
+    L = p.seq_len[b];
+    T = p.tree_size[b];
+    if (T < 0 || T > p.T_max || L < 0 || (long long)L + T > (long long)p.S_cap) { L = 0; T = 0; }   // invalid: no work
+    ntiles = T > 0 ? (L + T + BN - 1) / BN : 0;
+    nrb = (T * G + BR - 1) / BR;
+}
+
+// Warp-cooperative scan over the sequences.  Returns the sequence that holds global tile `g`
+// (want_b < 0) or sequence want_b; `total` receives the number of tiles of the whole batch.
+__device__ __forceinline__ SeqInfo scan_sequences(const graft_attn_params& p, int G, long long g, int want_b, long long& total) {
+    const int lane = threadIdx.x & 31;
+    SeqInfo out;
+    out.found = false;
+    out.b = out.L = out.T = out.nrb = out.ntiles = 0;
+    out.base = 0;
+    long long run = 0;
+    for (int b0 = 0; b0 < p.B; b0 += 32) {
+        const int b = b0 + lane;
+        int L = 0, T = 0, nrb = 0, ntiles = 0;
+        if (b < p.B) seq_shape(p, G, b, L, T, nrb, ntiles);
+        const long long cnt = (long long)p.Hkv * nrb * ntiles;
+        long long incl = cnt;
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) {
+            const long long v = __shfl_up_sync(0xffffffffu, incl, o);
+            if (lane >= o) incl += v;
+        }
+        const long long start = run + incl - cnt;
+        const bool hit = b < p.B && !out.found && (want_b >= 0 ? b == want_b : (cnt > 0 && g >= start && g < start + cnt));
+        const unsigned m = __ballot_sync(0xffffffffu, hit);
+        if (m) {
+            const int src = __ffs(m) - 1;
+            out.found = true;
+            out.b = b0 + src;
+            out.L = __shfl_sync(0xffffffffu, L, src);
+            out.T = __shfl_sync(0xffffffffu, T, src);
+            out.nrb = __shfl_sync(0xffffffffu, nrb, src);
+            out.ntiles = __shfl_sync(0xffffffffu, ntiles, src);
+            out.base = __shfl_sync(0xffffffffu, start, src);
+        }
+        run += __shfl_sync(0xffffffffu, incl, 31);
+    }
+    total = run;
+    return out;
+}
+
+struct Seg {
+    int b, h, rb;            // item
+    int tile_lo, tile_hi;    // tiles [lo, hi) of the item
+    int L, T;
+    int slot;                // partial slot, or -1: the segment covers the whole item and writes final rows
+};
+
+// ---------------------------------------------------------------------------------------------------
+// PTX helpers
+// ---------------------------------------------------------------------------------------------------
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
 
 __device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
@@ -155,24 +228,11 @@ __device__ __forceinline__ float ex2(float x) {
     asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
     return y;
 }
-// two fp32 lanes in one 64-bit register, for the packed fma / add of sm_100
-__device__ __forceinline__ unsigned long long pack2f(float lo, float hi) {
-    unsigned long long r;
-    asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "f"(lo), "f"(hi));
-    return r;
-}
-__device__ __forceinline__ void unpack2f(unsigned long long v, float& lo, float& hi) {
-    asm("mov.b64 {%0, %1}, %2;" : "=f"(lo), "=f"(hi) : "l"(v));
-}
-__device__ __forceinline__ unsigned long long ffma2(unsigned long long a, unsigned long long b, unsigned long long c) {
-    unsigned long long d;
-    asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(d) : "l"(a), "l"(b), "l"(c));
-    return d;
-}
-__device__ __forceinline__ unsigned long long fadd2(unsigned long long a, unsigned long long b) {
-    unsigned long long d;
-    asm("add.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
-    return d;
+// 32-byte global store (needs a 32-byte aligned address)
+__device__ __forceinline__ void st_global_v8(void* ptr, uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3, uint32_t a4,
+                                             uint32_t a5, uint32_t a6, uint32_t a7) {
+    asm volatile("st.global.v8.b32 [%0], {%1,%2,%3,%4,%5,%6,%7,%8};" ::"l"(ptr), "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(a4),
+                 "r"(a5), "r"(a6), "r"(a7) : "memory");
 }
 __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
     __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
@@ -192,369 +252,412 @@ constexpr uint64_t kDescVMajor = desc_fixed(HALF_BYTES);    // V tile as an MN-m
 // 16-byte-unit offset to a descriptor's low word never carries out of the field
 __device__ __forceinline__ uint64_t smem_desc(uint64_t fixed, uint32_t addr16) { return fixed | (uint64_t)addr16; }
 
-// instruction descriptors of kind::f16: fp32 accumulate, bf16 A and B, M = 128
+// instruction descriptors of kind::f16: fp32 accumulate, bf16 A and B, M = 128, N = 128
 constexpr uint32_t kIdescBase = (1u << 4) | (1u << 7) | (1u << 10) | ((128u >> 3) << 17) | ((128u >> 4) << 24);
-constexpr uint32_t kIdescQK = kIdescBase;                // N = 128 keys; A, B both K-major
-constexpr uint32_t kIdescPV = kIdescBase | (1u << 16);   // N = d = 128; B (= V) MN-major
+constexpr uint32_t kIdescQK = kIdescBase;                // A, B both K-major
+constexpr uint32_t kIdescPV = kIdescBase | (1u << 16);   // B (= V) MN-major
 
+// ---------------------------------------------------------------------------------------------------
+// the kernel
+// ---------------------------------------------------------------------------------------------------
 __global__ void __launch_bounds__(NTHREADS, 1)
 attn_tc_kernel(const __grid_constant__ CUtensorMap kmap, const __grid_constant__ CUtensorMap vmap, TcArgs a, unsigned* status) {
     extern __shared__ unsigned char smem_raw[];
     __shared__ __align__(8) uint64_t s_bar[BAR_COUNT];
     __shared__ uint32_t s_tmem;
     __shared__ int s_abort;
-    __shared__ graft_sched::Work s_work;
+    __shared__ Seg s_seg[MAXSEG];
+    __shared__ int s_nseg;
+    __shared__ long long s_gnext, s_ghi;
 
     const graft_attn_params& p = a.p;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int G = a.G;
 
     const uint32_t sQ = (smem_u32(smem_raw) + 1023u) & ~1023u;
     const uint32_t sRing = sQ + 2 * TILE_BYTES;
     const uint32_t bar0 = smem_u32(s_bar);
     auto bar = [&](int i) { return bar0 + 8u * (uint32_t)i; };
     volatile int* abort_flag = &s_abort;
-    // ring load n: K (n even) or V (n odd) of this CTA's tile n / 2
-    auto issue_load = [&](const graft_sched::Work& ww, int n) {
-        const int slot = n % NSLOT;
-        const uint32_t dst = sRing + slot * TILE_BYTES;
-        const int key0 = (ww.tile_lo + (n >> 1)) * BN;
-        const CUtensorMap* map = (n & 1) ? &vmap : &kmap;
-        mbar_expect_tx(bar(BAR_FULL + slot), TILE_BYTES);
-        tma_load_4d(dst, map, 0, key0, ww.h, ww.b, bar(BAR_FULL + slot));
-        tma_load_4d(dst + HALF_BYTES, map, 64, key0, ww.h, ww.b, bar(BAR_FULL + slot));
-    };
 
-    if (warp == 0) {
-        graft_sched::Work w0 = graft_sched::find_work<BR, BN, true>(p.seq_len, p.tree_size, p.B, p.Hkv, a.G, p.T_max, p.S_cap,
-                                                                   a.target, blockIdx.x, -1);
-        if (lane == 0) {
-            s_work = w0;
-            s_abort = 0;
-            if (w0.valid) {
-                // barriers, then the first ring loads at once: their latency overlaps the Q load below
-                for (int i = 0; i < NSLOT; ++i) { mbar_init(bar(BAR_FULL + i), 1); mbar_init(bar(BAR_EMPTY + i), 1); }
-                for (int i = 0; i < 2; ++i) { mbar_init(bar(BAR_S + i), 1); mbar_init(bar(BAR_P + i), 4); }
-                mbar_init(bar(BAR_O), 1);
-                asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
-                const int n_first = DBG(128) ? 0 : min(NSLOT, 2 * (w0.tile_hi - w0.tile_lo));
-                for (int n = 0; n < n_first; ++n) issue_load(w0, n);
+    // ---- this CTA's tile range, and the first round of segments
+    // plan_round (warp 0): fills s_seg with the next <= MAXSEG segments of [g, g_hi)
+    auto plan_round = [&](long long g, long long g_lo_cta, long long g_hi) {
+        int n = 0;
+        while (g < g_hi && n < MAXSEG) {
+            long long total;
+            const SeqInfo si = scan_sequences(p, G, g, -1, total);
+            if (!si.found) { g = g_hi; break; }
+            // walk the items of this sequence that intersect [g, g_hi)
+            long long k = (g - si.base) / si.ntiles;
+            const long long items = (long long)p.Hkv * si.nrb;
+            while (k < items && g < g_hi && n < MAXSEG) {
+                const long long item_lo = si.base + k * si.ntiles;
+                const long long item_hi = item_lo + si.ntiles;
+                const long long e = item_hi < g_hi ? item_hi : g_hi;
+                if (lane == 0) {
+                    Seg s;
+                    s.b = si.b;
+                    s.h = (int)(k / si.nrb);
+                    s.rb = (int)(k % si.nrb);
+                    s.tile_lo = (int)(g - item_lo);
+                    s.tile_hi = (int)(e - item_lo);
+                    s.L = si.L;
+                    s.T = si.T;
+                    const bool whole = g == item_lo && e == item_hi;
+                    s.slot = whole ? -1 : 2 * (int)blockIdx.x + (g == g_lo_cta ? 0 : 1);
+                    s_seg[n] = s;
+                }
+                ++n;
+                g = e;
+                ++k;
             }
         }
+        if (lane == 0) { s_nseg = n; s_gnext = g; }
+    };
+
+    long long g_lo_cta = 0;
+    if (warp == 0) {
+        long long total;
+        (void)scan_sequences(p, G, 0, -1, total);
+        const long long per = (total + gridDim.x - 1) / gridDim.x;
+        g_lo_cta = per * blockIdx.x;
+        long long g_hi = g_lo_cta + per;
+        if (g_hi > total) g_hi = total;
+        if (g_lo_cta > total) g_lo_cta = total;
+        if (lane == 0) { s_ghi = g_hi; s_abort = 0; }
+        plan_round(g_lo_cta, g_lo_cta, g_hi);
     }
     __syncthreads();
-    const graft_sched::Work w = s_work;
-    if (!w.valid) return;
-    if (DBG(128)) return;
+    if (s_nseg == 0) return;                      // nothing for this CTA (short batch)
 
-    const int G = a.G;
-    const int R = w.T * G;
-    const int row0 = w.rb * BR;
-    const int nblk = (R - row0 > 128) ? 2 : 1;
-    const int n_keys = w.L + w.T;
-    const int nt = w.tile_hi - w.tile_lo;
-
+    if (threadIdx.x == 0) {
+        for (int i = 0; i < NSLOT; ++i) { mbar_init(bar(BAR_FULL + i), 1); mbar_init(bar(BAR_EMPTY + i), 1); }
+        for (int i = 0; i < 2; ++i) { mbar_init(bar(BAR_S + i), 1); mbar_init(bar(BAR_P + i), 4); }
+        mbar_init(bar(BAR_Q), 8);
+        mbar_init(bar(BAR_O), 1);
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
     if (warp == 1) {
         asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&s_tmem)), "r"(512u) : "memory");
         asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
-    }
-
-    // ---- Q rows into shared memory, K-major with the 128-byte swizzle (16-byte chunk c of row r at c ^ (r & 7))
-    {
-        const __nv_bfloat16* Qg = reinterpret_cast<const __nv_bfloat16*>(p.Q) + (size_t)w.b * p.q_stride_b +
-                                  (size_t)w.h * G * p.q_stride_h;
-        constexpr int PER = (BR * 16 + NTHREADS - 1) / NTHREADS;
-        uint4 v[PER];
-#pragma unroll
-        for (int q = 0; q < PER; ++q) {
-            const int c = threadIdx.x + q * NTHREADS;
-            const int rl = c >> 4, ch = c & 15;
-            const int r = row0 + rl;
-            v[q] = make_uint4(0u, 0u, 0u, 0u);
-            if (c < BR * 16 && r < R) {
-                const int t = r / G, g = r % G;
-                v[q] = *reinterpret_cast<const uint4*>(Qg + (size_t)t * p.q_stride_t + (size_t)g * p.q_stride_h + ch * 8);
-            }
-        }
-#pragma unroll
-        for (int q = 0; q < PER; ++q) {
-            const int c = threadIdx.x + q * NTHREADS;
-            if (c < BR * 16) {
-                const int rl = c >> 4, ch = c & 15;
-                const int blk = rl >> 7, rr = rl & 127;
-                const uint32_t dst = sQ + blk * TILE_BYTES + (ch >> 3) * HALF_BYTES + rr * 128 + (((ch & 7) ^ (rr & 7)) << 4);
-                asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(dst), "r"(v[q].x), "r"(v[q].y), "r"(v[q].z), "r"(v[q].w) : "memory");
-            }
-        }
-        fence_async_smem();
     }
     tc_fence_before();
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem = s_tmem;
 
-    if (warp == 0) {
-        // =============================== TMA producer ===============================
-        if (lane == 0) {
-            const int n_total = 2 * nt;
-            int n = min(NSLOT, n_total);                      // the first loads were issued before the Q load
-            if (DBG(64)) {                                 // experiment: loads only, reuse a slot as soon as it landed
-                for (; n < n_total; ++n) {
-                    mbar_wait(bar(BAR_FULL + n % NSLOT), (n / NSLOT - 1) & 1, abort_flag, status);
-                    issue_load(w, n);
+    // running counters that persist across segments and rounds (each role keeps its own copy)
+    int n_load = 0;            // ring loads issued / consumed so far (2 per tile)
+    int jt[2] = {0, 0};        // tiles processed so far by row block 0 / 1 (S and P barrier phases)
+    int n_seg_done = 0;        // segments finished (Q and O barrier phases)
+
+    for (;;) {                 // rounds of <= MAXSEG segments
+        const int nseg = s_nseg;
+
+        if (warp == 0) {
+            // =============================== TMA producer ===============================
+            if (lane == 0) {
+                for (int si = 0; si < nseg; ++si) {
+                    const Seg sg = s_seg[si];
+                    for (int t = sg.tile_lo; t < sg.tile_hi; ++t)
+                        for (int which = 0; which < 2; ++which, ++n_load) {
+                            const int slot = n_load % NSLOT, use = n_load / NSLOT;
+                            if (use > 0) mbar_wait(bar(BAR_EMPTY + slot), (use - 1) & 1, abort_flag, status);
+                            const uint32_t dst = sRing + slot * TILE_BYTES;
+                            const CUtensorMap* map = which ? &vmap : &kmap;
+                            mbar_expect_tx(bar(BAR_FULL + slot), TILE_BYTES);
+                            tma_load_4d(dst, map, 0, t * BN, sg.h, sg.b, bar(BAR_FULL + slot));
+                            tma_load_4d(dst + HALF_BYTES, map, 64, t * BN, sg.h, sg.b, bar(BAR_FULL + slot));
+                        }
                 }
-            } else
-            for (; n < n_total; ++n) {
-                mbar_wait(bar(BAR_EMPTY + n % NSLOT), (n / NSLOT - 1) & 1, abort_flag, status);
-                issue_load(w, n);
             }
-            // drain: every copy issued must have landed before the CTA may exit
-            for (int m = max(0, n - NSLOT); m < n; ++m) mbar_wait(bar(BAR_FULL + m % NSLOT), (m / NSLOT) & 1, abort_flag, status);
-        }
-    } else if (DBG(64)) {
-    } else if (warp == 1) {
-        // =============================== MMA issuer ===============================
-        if (lane == 0) {
-            auto wait_full = [&](int n) { mbar_wait(bar(BAR_FULL + n % NSLOT), (n / NSLOT) & 1, abort_flag, status); };
-            // S[blk] = Q[blk] K(j)^T
-            auto issue_qk = [&](int blk, int j) {
-                const uint32_t sK16 = (sRing + ((2 * j) % NSLOT) * TILE_BYTES) >> 4;
-                const uint32_t sQ16 = (sQ + blk * TILE_BYTES) >> 4;
-                if (!DBG(2))
+        } else if (warp == 1) {
+            // =============================== MMA issuer ===============================
+            if (lane == 0) {
+                auto wait_full = [&](int n) { mbar_wait(bar(BAR_FULL + n % NSLOT), (n / NSLOT) & 1, abort_flag, status); };
+                for (int si = 0; si < nseg; ++si) {
+                    const Seg sg = s_seg[si];
+                    const int nt = sg.tile_hi - sg.tile_lo;
+                    const int nblk = (sg.T * G - sg.rb * BR > 128) ? 2 : 1;
+                    // S[blk] = Q[blk] K^T with the K tile of ring load n
+                    auto issue_qk = [&](int blk, int n) {
+                        const uint32_t sK16 = (sRing + (n % NSLOT) * TILE_BYTES) >> 4;
+                        const uint32_t sQ16 = (sQ + blk * TILE_BYTES) >> 4;
 #pragma unroll
-                for (int k = 0; k < D / 16; ++k) {
-                    const uint32_t off16 = ((k >> 2) * HALF_BYTES + (k & 3) * 32) >> 4;
-                    mma_ss(tmem + blk * 128, smem_desc(kDescKMajor, sQ16 + off16), smem_desc(kDescKMajor, sK16 + off16), kIdescQK, k > 0);
-                }
-                tc_commit(bar(BAR_S + blk));
-                if (blk == nblk - 1) tc_commit(bar(BAR_EMPTY + (2 * j) % NSLOT));          // K tile fully read
-            };
-            // O[blk] (+)= P[blk] V(j)
-            auto issue_pv = [&](int blk, int j) {
-                const uint32_t sV16 = (sRing + ((2 * j + 1) % NSLOT) * TILE_BYTES) >> 4;
-                if (!DBG(4))
+                        for (int k = 0; k < D / 16; ++k) {
+                            const uint32_t off16 = ((k >> 2) * HALF_BYTES + (k & 3) * 32) >> 4;
+                            mma_ss(tmem + blk * 128, smem_desc(kDescKMajor, sQ16 + off16), smem_desc(kDescKMajor, sK16 + off16), kIdescQK, k > 0);
+                        }
+                        tc_commit(bar(BAR_S + blk));
+                        if (blk == nblk - 1) tc_commit(bar(BAR_EMPTY + n % NSLOT));          // K tile fully read
+                    };
+                    // O[blk] (+)= P[blk] V with the V tile of ring load n
+                    auto issue_pv = [&](int blk, int n, bool first) {
+                        const uint32_t sV16 = (sRing + (n % NSLOT) * TILE_BYTES) >> 4;
 #pragma unroll
-                for (int k = 0; k < BN / 16; ++k)
-                    mma_ts(tmem + 256 + blk * 128, tmem + blk * 128 + k * 8, smem_desc(kDescVMajor, sV16 + k * (2048 >> 4)), kIdescPV,
-                           (j > 0 || k > 0) ? 1u : 0u);
-                if (blk == nblk - 1) tc_commit(bar(BAR_EMPTY + (2 * j + 1) % NSLOT));      // V tile fully read
-            };
-            wait_full(0);
-            tc_fence_after();
-            for (int blk = 0; blk < nblk; ++blk) issue_qk(blk, 0);
-            long long m_waitp = 0, m_waitf = 0, m_issue = 0, mc0 = clock64(), mc1;
-            const bool mprof = DBG(4096) && blockIdx.x == 0;
-            for (int j = 0; j < nt; ++j) {
-                for (int blk = 0; blk < nblk; ++blk) {
-                    mbar_wait(bar(BAR_P + blk), j & 1, abort_flag, status);
-                    if (mprof) { mc1 = clock64(); m_waitp += mc1 - mc0; mc0 = mc1; }
-                    if (blk == 0) wait_full(2 * j + 1);
-                    if (mprof) { mc1 = clock64(); m_waitf += mc1 - mc0; mc0 = mc1; }
+                        for (int k = 0; k < BN / 16; ++k)
+                            mma_ts(tmem + 256 + blk * 128, tmem + blk * 128 + k * 8, smem_desc(kDescVMajor, sV16 + k * (2048 >> 4)), kIdescPV,
+                                   (!first || k > 0) ? 1u : 0u);
+                        if (blk == nblk - 1) tc_commit(bar(BAR_EMPTY + n % NSLOT));          // V tile fully read
+                    };
+                    mbar_wait(bar(BAR_Q), n_seg_done & 1, abort_flag, status);                // Q of this segment staged
+                    wait_full(n_load);
                     tc_fence_after();
-                    issue_pv(blk, j);
-                    if (mprof) { mc1 = clock64(); m_issue += mc1 - mc0; mc0 = mc1; }
-                    if (j + 1 < nt) {
-                        if (blk == 0) { wait_full(2 * j + 2); tc_fence_after(); }
-                        if (mprof) { mc1 = clock64(); m_waitf += mc1 - mc0; mc0 = mc1; }
-                        issue_qk(blk, j + 1);
-                        if (mprof) { mc1 = clock64(); m_issue += mc1 - mc0; mc0 = mc1; }
+                    for (int blk = 0; blk < nblk; ++blk) issue_qk(blk, n_load);
+                    for (int j = 0; j < nt; ++j) {
+                        const int nV = n_load + 2 * j + 1, nK1 = n_load + 2 * j + 2;
+                        for (int blk = 0; blk < nblk; ++blk) {
+                            mbar_wait(bar(BAR_P + blk), (jt[blk] + j) & 1, abort_flag, status);
+                            if (blk == 0) wait_full(nV);
+                            tc_fence_after();
+                            issue_pv(blk, nV, j == 0);
+                            if (j + 1 < nt) {
+                                if (blk == 0) { wait_full(nK1); tc_fence_after(); }
+                                issue_qk(blk, nK1);
+                            }
+                        }
                     }
+                    tc_commit(bar(BAR_O));
+                    n_load += 2 * nt;
+                    for (int blk = 0; blk < nblk; ++blk) jt[blk] += nt;
+                    ++n_seg_done;
                 }
             }
-            if (mprof) {
-                unsigned* dbgw = status + 24;
-                dbgw[0] = (unsigned)(m_waitp / nt); dbgw[1] = (unsigned)(m_waitf / nt); dbgw[2] = (unsigned)(m_issue / nt);
-            }
-            tc_commit(bar(BAR_O));
-        }
-    } else if (warp >= 4) {
-        // =============================== softmax + epilogue ===============================
-        const int blk = (warp - 4) >> 2;
-        if (blk < nblk) {
+        } else if (warp >= 4) {
+            // =============================== Q staging, softmax, results ===============================
+            const int blk = (warp - 4) >> 2;
             const int rl = ((warp & 3) << 5) + lane;            // row inside the block = TMEM lane
-            const int r = row0 + blk * 128 + rl;
-            const bool row_valid = r < R;
-            const int t = row_valid ? r / G : 0, g = row_valid ? r % G : 0;
-            const unsigned long long anc = row_valid ? p.tree_anc[(size_t)w.b * p.T_max + t] : 0ull;
             const uint32_t lane_bits = (uint32_t)((warp & 3) << 5) << 16;
             const uint32_t tS = tmem + lane_bits + blk * 128;
             const uint32_t tO = tmem + lane_bits + 256 + blk * 128;
             const float sl2 = p.scale * kLog2e;
-            float m_ref = -CUDART_INF_F, l = 0.f;
+            for (int si = 0; si < nseg; ++si) {
+                const Seg sg = s_seg[si];
+                const int nt = sg.tile_hi - sg.tile_lo;
+                const int R = sg.T * G;
+                const int row0 = sg.rb * BR;
+                const int nblk = (R - row0 > 128) ? 2 : 1;
+                const int n_keys = sg.L + sg.T;
 
-            if (DBG(8192) && blk == 1) { const long long t0 = clock64(); while (clock64() - t0 < 1700) {} }
-            long long t_wait = 0, t_p1 = 0, t_p2 = 0, t_tail = 0, tc0 = clock64(), tc1;
-            const bool prof = DBG(4096) && blockIdx.x == 0 && rl == 0;
-            for (int j = 0; j < nt; ++j) {
-                const int key0 = (w.tile_lo + j) * BN;
-                const bool boundary = key0 + BN > w.L;
-                mbar_wait(bar(BAR_S + blk), j & 1, abort_flag, status);
-                tc_fence_after();
-                if (prof) { tc1 = clock64(); t_wait += tc1 - tc0; tc0 = tc1; }
-                // pass 1: row maximum of the (masked) scores, 64 columns in flight at a time
-                auto mask32 = [&](uint32_t (&x)[32], int col0) {
+                // ---- Q rows of this item into shared memory, K-major with the 128-byte swizzle (16-byte chunk
+                // c of row r at c ^ (r & 7)).  The previous segment's MMAs are complete (its O was read).
+                {
+                    const __nv_bfloat16* Qg = reinterpret_cast<const __nv_bfloat16*>(p.Q) + (size_t)sg.b * p.q_stride_b +
+                                              (size_t)sg.h * G * p.q_stride_h;
+                    const int tid = threadIdx.x - 128;           // 0..255
+                    constexpr int PER = BR * 16 / 256;
+                    uint4 v[PER];
 #pragma unroll
-                    for (int q = 0; q < 32; ++q) {
-                        const int u = key0 + col0 + q - w.L;
-                        if (!(u < 0 || (u < w.T && ((anc >> (u & 63)) & 1ull)))) x[q] = 0xff800000u;   // -inf
-                    }
-                };
-                auto max32 = [&](const uint32_t (&x)[32], float& m0, float& m1) {
-#pragma unroll
-                    for (int q = 0; q < 32; q += 4) {
-                        m0 = fmax3(m0, __uint_as_float(x[q]), __uint_as_float(x[q + 1]));
-                        m1 = fmax3(m1, __uint_as_float(x[q + 2]), __uint_as_float(x[q + 3]));
-                    }
-                };
-                float mx0 = -CUDART_INF_F, mx1 = -CUDART_INF_F;
-                if (!DBG(8)) {
-                    uint32_t x0[32], x1[32];
-                    tmem_ld32(tS, x0);
-                    tmem_ld32(tS + 32, x1);
-                    tmem_wait_ld();
-                    if (boundary) { mask32(x0, 0); mask32(x1, 32); }
-                    max32(x0, mx0, mx1);
-                    max32(x1, mx0, mx1);
-                    tmem_ld32(tS + 64, x0);
-                    tmem_ld32(tS + 96, x1);
-                    tmem_wait_ld();
-                    if (boundary) { mask32(x0, 64); mask32(x1, 96); }
-                    max32(x0, mx0, mx1);
-                    max32(x1, mx0, mx1);
-                } else {
-                    mx0 = 0.f;
-                }
-                const float mx = fmaxf(mx0, mx1);
-                if (prof) { tc1 = clock64(); t_p1 += tc1 - tc0; tc0 = tc1; }
-                // reference maximum: move it only when the scores outgrow it by more than the threshold
-                if (mx != -CUDART_INF_F && (m_ref == -CUDART_INF_F || (mx - m_ref) * sl2 > kRescaleThreshold)) {
-                    if (m_ref != -CUDART_INF_F) {
-                        const float alpha = exp2f((m_ref - mx) * sl2);
-                        l *= alpha;
-#pragma unroll 1
-                        for (int c = 0; c < 4; ++c) {       // O of the previous tiles is complete here
-                            uint32_t o[32];
-                            tmem_ld32(tO + c * 32, o);
-                            tmem_wait_ld();
-#pragma unroll
-                            for (int q = 0; q < 32; ++q) o[q] = __float_as_uint(__uint_as_float(o[q]) * alpha);
-                            tmem_st32(tO + c * 32, o);
+                    for (int q = 0; q < PER; ++q) {
+                        const int c = tid + q * 256;
+                        const int r = row0 + (c >> 4);
+                        v[q] = make_uint4(0u, 0u, 0u, 0u);
+                        if (r < R) {
+                            const int t = r / G, g = r % G;
+                            v[q] = *reinterpret_cast<const uint4*>(Qg + (size_t)t * p.q_stride_t + (size_t)g * p.q_stride_h + (c & 15) * 8);
                         }
-                        tmem_wait_st();
                     }
-                    m_ref = mx;
-                }
-                const float off = m_ref == -CUDART_INF_F ? 0.f : m_ref * sl2;
-                // pass 2: P = 2^(s*scale*log2e - off) as bf16 into the first 64 columns of S.  P chunk c
-                // (columns 16c..16c+15) only overwrites score columns that are already in registers.
-                float sum0 = 0.f, sum1 = 0.f;
-                auto exp32 = [&](const uint32_t (&x)[32], uint32_t col) {
-                    uint32_t pk[16];
 #pragma unroll
-                    for (int q = 0; q < 32; q += 2) {
-                        const float p0 = ex2(fmaf(__uint_as_float(x[q]), sl2, -off));
-                        const float p1 = ex2(fmaf(__uint_as_float(x[q + 1]), sl2, -off));
-                        sum0 += p0;
-                        sum1 += p1;
-                        pk[q >> 1] = pack_bf16(p0, p1);
-                    }
-                    tmem_st16(tS + col, pk);
-                };
-                if (DBG(1)) {
-                    uint32_t pk[16];
-#pragma unroll
-                    for (int q = 0; q < 16; ++q) pk[q] = 0x3f803f80u;
-                    if (!DBG(16)) { tmem_st16(tS, pk); tmem_st16(tS + 16, pk); tmem_st16(tS + 32, pk); tmem_st16(tS + 48, pk); }
-                    sum0 = 128.f;
-                } else {
-                    uint32_t x0[32], x1[32];
-                    tmem_ld32(tS, x0);
-                    tmem_ld32(tS + 32, x1);
-                    tmem_wait_ld();
-                    if (boundary) { mask32(x0, 0); mask32(x1, 32); }
-                    exp32(x0, 0);
-                    tmem_ld32(tS + 64, x0);
-                    exp32(x1, 16);
-                    tmem_ld32(tS + 96, x1);
-                    tmem_wait_ld();
-                    if (boundary) { mask32(x0, 64); mask32(x1, 96); }
-                    exp32(x0, 32);
-                    exp32(x1, 48);
-                }
-                l += sum0 + sum1;
-                if (prof) { tc1 = clock64(); t_p2 += tc1 - tc0; tc0 = tc1; }
-                tmem_wait_st();
-                // last tile of the sequence: zero the V rows of slots that hold no key of this tree
-                if (blk == 0 && key0 + BN > n_keys) {
-                    const int nV = 2 * j + 1;
-                    mbar_wait(bar(BAR_FULL + nV % NSLOT), (nV / NSLOT) & 1, abort_flag, status);
-                    if (key0 + rl >= n_keys) {
-                        const uint32_t sV = sRing + (nV % NSLOT) * TILE_BYTES + rl * 128;
-#pragma unroll
-                        for (int q = 0; q < 8; ++q) {
-                            asm volatile("st.shared.v4.b32 [%0], {%1, %1, %1, %1};" ::"r"(sV + q * 16), "r"(0u) : "memory");
-                            asm volatile("st.shared.v4.b32 [%0], {%1, %1, %1, %1};" ::"r"(sV + HALF_BYTES + q * 16), "r"(0u) : "memory");
-                        }
+                    for (int q = 0; q < PER; ++q) {
+                        const int c = tid + q * 256;
+                        const int qr = c >> 4, ch = c & 15;
+                        const int qb = qr >> 7, rr = qr & 127;
+                        const uint32_t dst = sQ + qb * TILE_BYTES + (ch >> 3) * HALF_BYTES + rr * 128 + (((ch & 7) ^ (rr & 7)) << 4);
+                        asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(dst), "r"(v[q].x), "r"(v[q].y), "r"(v[q].z), "r"(v[q].w) : "memory");
                     }
                     fence_async_smem();
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(bar(BAR_Q));
                 }
-                tc_fence_before();
-                __syncwarp();
-                if (lane == 0) mbar_arrive(bar(BAR_P + blk));      // one arrival per warp
-                if (prof) { tc1 = clock64(); t_tail += tc1 - tc0; tc0 = tc1; }
-            }
-            if (prof) {
-                unsigned* dbgw = status + 8 + blk * 8;
-                dbgw[0] = (unsigned)nt; dbgw[1] = (unsigned)(t_wait / nt); dbgw[2] = (unsigned)(t_p1 / nt);
-                dbgw[3] = (unsigned)(t_p2 / nt); dbgw[4] = (unsigned)(t_tail / nt);
-            }
 
-            // ---- epilogue: O row from TMEM, final result or partial
-            mbar_wait(bar(BAR_O), 0, abort_flag, status);
-            tc_fence_after();
-            if (w.nsplit == 1) {
-                const float inv = l > 0.f ? 1.f / l : 0.f;
-                __nv_bfloat16* orow = reinterpret_cast<__nv_bfloat16*>(p.O) + (size_t)w.b * p.o_stride_b + (size_t)t * p.o_stride_t +
-                                      (size_t)(w.h * G + g) * p.o_stride_h;
-#pragma unroll 1
-                for (int c = 0; c < 4; ++c) {
-                    uint32_t v[32];
-                    tmem_ld32(tO + c * 32, v);
-                    tmem_wait_ld();
-                    if (row_valid) {
+                if (blk < nblk) {
+                    const int r = row0 + blk * 128 + rl;
+                    const bool row_valid = r < R;
+                    const int t = row_valid ? r / G : 0, g = row_valid ? r % G : 0;
+                    const unsigned long long anc = row_valid ? p.tree_anc[(size_t)sg.b * p.T_max + t] : 0ull;
+                    float m_ref = -CUDART_INF_F, l = 0.f;
+
+                    for (int j = 0; j < nt; ++j) {
+                        const int key0 = (sg.tile_lo + j) * BN;
+                        const bool boundary = key0 + BN > sg.L;
+                        mbar_wait(bar(BAR_S + blk), (jt[blk] + j) & 1, abort_flag, status);
+                        tc_fence_after();
+                        auto mask32 = [&](uint32_t (&x)[32], int col0) {    // ancestor mask and the end of the tree's keys
 #pragma unroll
-                        for (int q = 0; q < 4; ++q) {
-                            uint4 o4;
-                            o4.x = pack_bf16(__uint_as_float(v[q * 8 + 0]) * inv, __uint_as_float(v[q * 8 + 1]) * inv);
-                            o4.y = pack_bf16(__uint_as_float(v[q * 8 + 2]) * inv, __uint_as_float(v[q * 8 + 3]) * inv);
-                            o4.z = pack_bf16(__uint_as_float(v[q * 8 + 4]) * inv, __uint_as_float(v[q * 8 + 5]) * inv);
-                            o4.w = pack_bf16(__uint_as_float(v[q * 8 + 6]) * inv, __uint_as_float(v[q * 8 + 7]) * inv);
-                            *reinterpret_cast<uint4*>(orow + c * 32 + q * 8) = o4;
+                            for (int q = 0; q < 32; ++q) {
+                                const int u = key0 + col0 + q - sg.L;
+                                if (!(u < 0 || (u < sg.T && ((anc >> (u & 63)) & 1ull)))) x[q] = 0xff800000u;   // -inf
+                            }
+                        };
+                        auto max32 = [&](const uint32_t (&x)[32], float& m0, float& m1) {
+#pragma unroll
+                            for (int q = 0; q < 32; q += 4) {
+                                m0 = fmax3(m0, __uint_as_float(x[q]), __uint_as_float(x[q + 1]));
+                                m1 = fmax3(m1, __uint_as_float(x[q + 2]), __uint_as_float(x[q + 3]));
+                            }
+                        };
+                        // pass 1: row maximum of the (masked) scores, 64 columns in flight at a time
+                        float mx0 = -CUDART_INF_F, mx1 = -CUDART_INF_F;
+                        {
+                            uint32_t x0[32], x1[32];
+                            tmem_ld32(tS, x0);
+                            tmem_ld32(tS + 32, x1);
+                            tmem_wait_ld();
+                            if (boundary) { mask32(x0, 0); mask32(x1, 32); }
+                            max32(x0, mx0, mx1);
+                            max32(x1, mx0, mx1);
+                            tmem_ld32(tS + 64, x0);
+                            tmem_ld32(tS + 96, x1);
+                            tmem_wait_ld();
+                            if (boundary) { mask32(x0, 64); mask32(x1, 96); }
+                            max32(x0, mx0, mx1);
+                            max32(x1, mx0, mx1);
                         }
-                    }
-                }
-                if (row_valid && p.LSE)
-                    p.LSE[((size_t)w.b * p.Hq + w.h * G + g) * p.T_max + t] =
-                        l > 0.f ? (m_ref * sl2 + log2f(l)) * graft_merge::kLn2 : -CUDART_INF_F;
-            } else {
-                float* base = a.partial + (size_t)graft_sched::slot_of(w, w.h, w.split, w.rb) * ((size_t)BR * (D + 2));
-                const int lr = blk * 128 + rl;
-                float* prow = base + (size_t)lr * D;
+                        const float mx = fmaxf(mx0, mx1);
+                        // reference maximum: move it only when the scores outgrow it by more than the threshold
+                        if (mx != -CUDART_INF_F && (m_ref == -CUDART_INF_F || (mx - m_ref) * sl2 > kRescaleThreshold)) {
+                            if (m_ref != -CUDART_INF_F) {
+                                const float alpha = exp2f((m_ref - mx) * sl2);
+                                l *= alpha;
 #pragma unroll 1
-                for (int c = 0; c < 4; ++c) {
-                    uint32_t v[32];
-                    tmem_ld32(tO + c * 32, v);
-                    tmem_wait_ld();
+                                for (int c = 0; c < 4; ++c) {       // O of the previous tiles is complete here
+                                    uint32_t o[32];
+                                    tmem_ld32(tO + c * 32, o);
+                                    tmem_wait_ld();
 #pragma unroll
-                    for (int q = 0; q < 8; ++q)
-                        *reinterpret_cast<uint4*>(prow + c * 32 + q * 4) = make_uint4(v[q * 4], v[q * 4 + 1], v[q * 4 + 2], v[q * 4 + 3]);
+                                    for (int q = 0; q < 32; ++q) o[q] = __float_as_uint(__uint_as_float(o[q]) * alpha);
+                                    tmem_st32(tO + c * 32, o);
+                                }
+                                tmem_wait_st();
+                            }
+                            m_ref = mx;
+                        }
+                        const float off = m_ref == -CUDART_INF_F ? 0.f : m_ref * sl2;
+                        // pass 2: P = 2^(s*scale*log2e - off) as bf16 into the first 64 columns of S.  P chunk c
+                        // (columns 16c..16c+15) only overwrites score columns that are already in registers.
+                        float sum0 = 0.f, sum1 = 0.f;
+                        auto exp32 = [&](const uint32_t (&x)[32], uint32_t col) {
+                            uint32_t pk[16];
+#pragma unroll
+                            for (int q = 0; q < 32; q += 2) {
+                                const float p0 = ex2(fmaf(__uint_as_float(x[q]), sl2, -off));
+                                const float p1 = ex2(fmaf(__uint_as_float(x[q + 1]), sl2, -off));
+                                sum0 += p0;
+                                sum1 += p1;
+                                pk[q >> 1] = pack_bf16(p0, p1);
+                            }
+                            tmem_st16(tS + col, pk);
+                        };
+                        {
+                            uint32_t x0[32], x1[32];
+                            tmem_ld32(tS, x0);
+                            tmem_ld32(tS + 32, x1);
+                            tmem_wait_ld();
+                            if (boundary) { mask32(x0, 0); mask32(x1, 32); }
+                            exp32(x0, 0);
+                            tmem_ld32(tS + 64, x0);
+                            exp32(x1, 16);
+                            tmem_ld32(tS + 96, x1);
+                            tmem_wait_ld();
+                            if (boundary) { mask32(x0, 64); mask32(x1, 96); }
+                            exp32(x0, 32);
+                            exp32(x1, 48);
+                        }
+                        l += sum0 + sum1;
+                        tmem_wait_st();
+                        // last tile of the sequence: zero the V rows of slots that hold no key of this tree
+                        if (blk == 0 && key0 + BN > n_keys) {
+                            const int nV = n_load + 2 * j + 1;
+                            mbar_wait(bar(BAR_FULL + nV % NSLOT), (nV / NSLOT) & 1, abort_flag, status);
+                            if (key0 + rl >= n_keys) {
+                                const uint32_t sV = sRing + (nV % NSLOT) * TILE_BYTES + rl * 128;
+#pragma unroll
+                                for (int q = 0; q < 8; ++q) {
+                                    asm volatile("st.shared.v4.b32 [%0], {%1, %1, %1, %1};" ::"r"(sV + q * 16), "r"(0u) : "memory");
+                                    asm volatile("st.shared.v4.b32 [%0], {%1, %1, %1, %1};" ::"r"(sV + HALF_BYTES + q * 16), "r"(0u) : "memory");
+                                }
+                            }
+                            fence_async_smem();
+                        }
+                        tc_fence_before();
+                        __syncwarp();
+                        if (lane == 0) mbar_arrive(bar(BAR_P + blk));      // one arrival per warp
+                    }
+
+                    // ---- results of the segment: O row from TMEM, final rows or a partial
+                    mbar_wait(bar(BAR_O), n_seg_done & 1, abort_flag, status);     // every MMA of the segment is complete
+                    tc_fence_after();
+                    if (sg.slot < 0) {
+                        const float inv = l > 0.f ? 1.f / l : 0.f;
+                        __nv_bfloat16* orow = reinterpret_cast<__nv_bfloat16*>(p.O) + (size_t)sg.b * p.o_stride_b + (size_t)t * p.o_stride_t +
+                                              (size_t)(sg.h * G + g) * p.o_stride_h;
+#pragma unroll 1
+                        for (int c = 0; c < 4; ++c) {
+                            uint32_t v[32];
+                            tmem_ld32(tO + c * 32, v);
+                            tmem_wait_ld();
+                            if (row_valid) {
+#pragma unroll
+                                for (int q = 0; q < 4; ++q) {      // 16-byte stores: O strides are only guaranteed 16-byte aligned
+                                    uint4 o4;
+                                    o4.x = pack_bf16(__uint_as_float(v[q * 8 + 0]) * inv, __uint_as_float(v[q * 8 + 1]) * inv);
+                                    o4.y = pack_bf16(__uint_as_float(v[q * 8 + 2]) * inv, __uint_as_float(v[q * 8 + 3]) * inv);
+                                    o4.z = pack_bf16(__uint_as_float(v[q * 8 + 4]) * inv, __uint_as_float(v[q * 8 + 5]) * inv);
+                                    o4.w = pack_bf16(__uint_as_float(v[q * 8 + 6]) * inv, __uint_as_float(v[q * 8 + 7]) * inv);
+                                    *reinterpret_cast<uint4*>(orow + c * 32 + q * 8) = o4;
+                                }
+                            }
+                        }
+                        if (row_valid && p.LSE)
+                            p.LSE[((size_t)sg.b * p.Hq + sg.h * G + g) * p.T_max + t] =
+                                l > 0.f ? (m_ref * sl2 + log2f(l)) * kLn2 : -CUDART_INF_F;
+                    } else {
+                        float* base = a.partial + (size_t)sg.slot * SLOT_FLOATS;
+                        const int lr = blk * 128 + rl;
+                        float* prow = base + (size_t)lr * D;
+#pragma unroll 1
+                        for (int c = 0; c < 4; ++c) {
+                            uint32_t v[32];
+                            tmem_ld32(tO + c * 32, v);
+                            tmem_wait_ld();
+#pragma unroll
+                            for (int q = 0; q < 4; ++q)      // 32-byte stores: every store fills a whole sector
+                                st_global_v8(prow + c * 32 + q * 8, v[q * 8], v[q * 8 + 1], v[q * 8 + 2], v[q * 8 + 3], v[q * 8 + 4],
+                                             v[q * 8 + 5], v[q * 8 + 6], v[q * 8 + 7]);
+                        }
+                        base[BR * D + lr] = m_ref == -CUDART_INF_F ? -CUDART_INF_F : m_ref * sl2;
+                        base[BR * D + BR + lr] = l;
+                    }
+                    tc_fence_before();                 // TMEM reads done before the next segment's MMAs are released
+                    jt[blk] += nt;
+                } else {
+                    // a row block without rows in this item still has to see the segment's MMAs finished
+                    // before it overwrites Q for the next one
+                    mbar_wait(bar(BAR_O), n_seg_done & 1, abort_flag, status);
                 }
-                base[BR * D + lr] = m_ref == -CUDART_INF_F ? -CUDART_INF_F : m_ref * sl2;
-                base[BR * D + BR + lr] = l;
+                n_load += 2 * nt;
+                ++n_seg_done;
             }
         }
+
+        // ---- next round (only batches with very many short sequences need more than one)
+        __syncthreads();
+        const long long g_next = s_gnext, g_hi = s_ghi;
+        if (g_next >= g_hi) break;
+        __syncthreads();
+        if (warp == 0) plan_round(g_next, g_lo_cta, g_hi);
+        __syncthreads();
+        if (s_nseg == 0) break;
     }
 
-    // ---- teardown: everyone is past its last TMEM access; the allocating warp frees the columns
+    // ---- teardown: every copy has landed (each was waited for by the MMA issuer); the allocating warp
+    // frees the TMEM columns once everyone is past its last access
+    if (warp == 0 && lane == 0 && *abort_flag)      // after a timeout some copies may still be in flight
+        for (int m = max(0, n_load - NSLOT); m < n_load; ++m) {
+            const long long t0 = clock64();
+            while (!mbar_try_wait(bar(BAR_FULL + m % NSLOT), (m / NSLOT) & 1) && clock64() - t0 < kWaitCycles) {}
+        }
     tc_fence_before();
     __syncthreads();
     if (warp == 1) {
@@ -563,11 +666,98 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap kmap, const __grid_constant__
     }
 }
 
-int target_ctas(int num_sms) { return num_sms; }
+// ---------------------------------------------------------------------------------------------------
+// merge: one warp per output row of the padded [T_max * G] row space of a (b, h_kv)
+// ---------------------------------------------------------------------------------------------------
+// Rows of an item that was cut across CTAs are merged with  M = max m_i, w_i = 2^(m_i - M),
+// O = sum w_i O_i / sum w_i l_i;  rows of padding nodes are zeroed (LSE -inf); rows of items that one CTA
+// finished alone were already final.  The set of CTAs that hold a piece of an item follows from the
+// same cut as in the attention kernel.
+constexpr int kMergeRows = 8;
 
-int max_ctas(int num_sms, int B, int Hq, int Hkv, int T_max) {
-    const int G = Hq / Hkv;
-    return target_ctas(num_sms) + B * Hkv * ((T_max * G + BR - 1) / BR);
+__global__ void __launch_bounds__(kMergeRows * 32, 2) merge_streamk_kernel(TcArgs a, int grid_attn, unsigned* status) {
+    const graft_attn_params& p = a.p;
+    const int G = a.G;
+    const int rows_pad = p.T_max * G;
+    const int groups = (rows_pad + kMergeRows - 1) / kMergeRows;
+    int idx = blockIdx.x;
+    const int grp = idx % groups; idx /= groups;
+    const int h = idx % p.Hkv;
+    const int b = idx / p.Hkv;
+    __shared__ SeqInfo s_info;
+    __shared__ long long s_per;
+    if (threadIdx.x < 32) {
+        long long total;
+        const SeqInfo si = scan_sequences(p, G, 0, b, total);
+        if (threadIdx.x == 0) {
+            s_info = si;
+            s_per = (total + grid_attn - 1) / grid_attn;
+            const int T = p.tree_size[b], L = p.seq_len[b];
+            if (grp == 0 && h == 0 && (T < 0 || T > p.T_max || L < 0 || (long long)L + T > p.S_cap))
+                atomicOr(status, (unsigned)GRAFT_FLAG_BAD_SIZE);
+        }
+    }
+    __syncthreads();
+    const SeqInfo si = s_info;
+    const long long per = s_per;
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int r = grp * kMergeRows + warp;
+    if (r >= rows_pad) return;
+    const int t = r / G, g = r % G;
+    __nv_bfloat16* orow = reinterpret_cast<__nv_bfloat16*>(p.O) + (size_t)b * p.o_stride_b + (size_t)t * p.o_stride_t +
+                          (size_t)(h * G + g) * p.o_stride_h + lane * 4;
+    float* lse = p.LSE ? p.LSE + ((size_t)b * p.Hq + h * G + g) * p.T_max + t : nullptr;
+    if (t >= si.T) {                       // padding node: zero row
+        *reinterpret_cast<uint2*>(orow) = make_uint2(0u, 0u);
+        if (lse && lane == 0) *lse = -CUDART_INF_F;
+        return;
+    }
+    const int rb = r / BR, rl = r % BR;
+    const long long item_lo = si.base + ((long long)h * si.nrb + rb) * si.ntiles;
+    const long long item_hi = item_lo + si.ntiles;
+    const int c_first = (int)(item_lo / per), c_last = (int)((item_hi - 1) / per);
+    const int nparts = c_last - c_first + 1;
+    if (nparts <= 1) return;               // one CTA had the whole item and wrote the final rows
+    // part i lives in CTA c_first + i: its first slot if the item was already running when that CTA's
+    // range began, else its second
+    auto part_base = [&](int i) {
+        const int c = c_first + i;
+        const int slot = 2 * c + ((item_lo <= (long long)c * per) ? 0 : 1);
+        return a.partial + (size_t)slot * SLOT_FLOATS;
+    };
+    float acc[4] = {0.f, 0.f, 0.f, 0.f};
+    float den = 0.f, M = -CUDART_INF_F;
+    for (int i = lane; i < nparts; i += 32) M = fmaxf(M, part_base(i)[BR * D + rl]);
+#pragma unroll
+    for (int o = 16; o; o >>= 1) M = fmaxf(M, __shfl_xor_sync(0xffffffffu, M, o));
+    for (int i0 = 0; i0 < nparts; i0 += 32) {
+        float wgt = 0.f, l = 0.f;
+        if (i0 + lane < nparts) {
+            const float* pb = part_base(i0 + lane);
+            const float m = pb[BR * D + rl];
+            l = pb[BR * D + BR + rl];
+            wgt = (m == -CUDART_INF_F || M == -CUDART_INF_F) ? 0.f : exp2f(m - M);
+        }
+        den += wgt * l;
+        const int cnt = min(32, nparts - i0);
+        for (int j0 = 0; j0 < cnt; j0 += 16) {      // 16 partial rows in flight per round
+            float4 x[16];
+#pragma unroll
+            for (int j = 0; j < 16; ++j)
+                if (j0 + j < cnt) x[j] = *reinterpret_cast<const float4*>(part_base(i0 + j0 + j) + (size_t)rl * D + lane * 4);
+#pragma unroll
+            for (int j = 0; j < 16; ++j)
+                if (j0 + j < cnt) {
+                    const float wj = __shfl_sync(0xffffffffu, wgt, j0 + j);
+                    acc[0] += wj * x[j].x; acc[1] += wj * x[j].y; acc[2] += wj * x[j].z; acc[3] += wj * x[j].w;
+                }
+        }
+    }
+#pragma unroll
+    for (int o = 16; o; o >>= 1) den += __shfl_xor_sync(0xffffffffu, den, o);
+    const float inv = den > 0.f ? 1.f / den : 0.f;
+    *reinterpret_cast<uint2*>(orow) = make_uint2(pack_bf16(acc[0] * inv, acc[1] * inv), pack_bf16(acc[2] * inv, acc[3] * inv));
+    if (lse && lane == 0) *lse = den > 0.f ? (M + log2f(den)) * kLn2 : -CUDART_INF_F;
 }
 
 typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
@@ -603,15 +793,16 @@ int graft_attn_tc_init() {
 
 bool graft_attn_tc_supported(const graft_ctx* ctx, const graft_attn_params* p) {
     if (p->d != D) return false;
-    // TMA: 16-byte aligned base and strides (checked by the caller), strides below 2^40 bytes, box rows within S_cap
+    // TMA: 16-byte aligned base and strides (checked by the caller), strides below 2^40 bytes
     if (p->kv_stride_s * 2 >= (1ll << 40) || p->kv_stride_h * 2 >= (1ll << 40) || p->kv_stride_b * 2 >= (1ll << 40)) return false;
     if (p->kv_stride_s == 0 || p->kv_stride_h == 0 || p->kv_stride_b == 0) return false;
     return GRAFT_WS_HEADER + graft_attn_tc_ws_bytes(ctx->num_sms, p->B, p->Hq, p->Hkv, p->d, p->T_max) <= ctx->ws_bytes;
 }
 
-size_t graft_attn_tc_ws_bytes(int num_sms, int B, int Hq, int Hkv, int d, int T_max) {
+// two partial slots per CTA, one CTA per SM: independent of the batch
+size_t graft_attn_tc_ws_bytes(int num_sms, int, int, int, int d, int) {
     if (d != D) return 0;
-    return (size_t)max_ctas(num_sms, B, Hq, Hkv, T_max) * BR * (D + 2) * sizeof(float);
+    return (size_t)num_sms * 2 * SLOT_FLOATS * sizeof(float);
 }
 
 int graft_attn_tc_launch(graft_ctx* ctx, const graft_attn_params* p, cudaStream_t stream) {
@@ -622,15 +813,15 @@ int graft_attn_tc_launch(graft_ctx* ctx, const graft_attn_params* p, cudaStream_
     TcArgs a;
     a.p = *p;
     a.partial = reinterpret_cast<float*>(reinterpret_cast<char*>(ctx->ws) + GRAFT_WS_HEADER);
-    a.target = target_ctas(ctx->num_sms);
     a.G = p->Hq / p->Hkv;
+    int grid = ctx->num_sms;
 #ifdef GRAFT_TC_EXPERIMENTS
-    a.dbg = getenv("GRAFT_TC_DEBUG") ? atoi(getenv("GRAFT_TC_DEBUG")) : 0;
-#else
-    a.dbg = 0;
+    if (getenv("GRAFT_TC_GRID")) grid = atoi(getenv("GRAFT_TC_GRID"));
 #endif
-    attn_tc_kernel<<<max_ctas(ctx->num_sms, p->B, p->Hq, p->Hkv, p->T_max), NTHREADS, SMEM_DYN, stream>>>(kmap, vmap, a, ctx->status);
+    attn_tc_kernel<<<grid, NTHREADS, SMEM_DYN, stream>>>(kmap, vmap, a, ctx->status);
     GRAFT_CHECK_CUDA(cudaGetLastError());
-    if (DBG(256)) return GRAFT_OK;
-    return graft_merge::launch<D, BR, BN, true>(a, ctx->status, stream);
+    const int groups = (p->T_max * a.G + kMergeRows - 1) / kMergeRows;
+    merge_streamk_kernel<<<p->B * p->Hkv * groups, kMergeRows * 32, 0, stream>>>(a, grid, ctx->status);
+    GRAFT_CHECK_CUDA(cudaGetLastError());
+    return GRAFT_OK;
 }
