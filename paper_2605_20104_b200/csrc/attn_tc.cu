@@ -8,9 +8,13 @@
 // SM).  A CTA therefore works through a few segments (item, tile range); a segment that covers its
 // whole item writes the final rows, any other writes a partial (row max, row sum, un-normalised O)
 // into one of the CTA's two workspace slots, and merge_streamk_kernel combines the partials of an
-// item.  The cut is a pure function of (seq_len, tree_size, gridDim.x), recomputed on the device
-// by every CTA and by the merge kernel: no communication, no atomics on floats, no waiting between
-// CTAs, bit-reproducible results for a given GPU model.
+// item.  When that range would be short (fewer than kStreamMinTiles tiles per CTA) a segment switch
+// (results out, next Q in, pipeline refill) is not amortised; the cut then falls back to whole
+// pieces: every item is divided into equal pieces of about that length and each CTA takes exactly one
+// piece, provided there are no more pieces than CTAs.  Either cut is a pure function of (seq_len,
+// tree_size, gridDim.x), recomputed on the device by every CTA and by the merge kernel: no
+// communication, no atomics on floats, no waiting between CTAs, bit-reproducible results for a given
+// GPU model.
 //
 // Warp roles inside a CTA:
 //   warp 0      TMA producer: K and V tiles (two 64-column boxes each, 128-byte swizzle) into a
@@ -18,7 +22,10 @@
 //               ahead across segment boundaries
 //   warp 1      MMA issuer: S = Q K^T (8 x m128 n128 k16, both operands from shared memory) and
 //               O += P V (8 x m128 n128 k16, P from TMEM, V as an MN-major operand); owns TMEM
-//   warps 4-7   softmax of row block 0: thread i <-> TMEM lane i <-> row i; also stage Q, write results
+//   warps 2-3   Q stagers: copy the item's Q rows into shared memory (swizzled, K-major); for the next
+//               segment they do so as soon as the current segment's last Q K^T has completed (the MMA issuer
+//               commits a barrier right behind it), i.e. while the last softmax, P V and result write-out run
+//   warps 4-7   softmax of row block 0: thread i <-> TMEM lane i <-> row i; write results
 //   warps 8-11  softmax of row block 1
 // The two row blocks ping-pong: while one block's softmax runs on the SIMT pipes, the tensor pipe
 // works on the other block (its P V of this tile, then its Q K^T of the next).  TMEM columns:
@@ -52,6 +59,7 @@ constexpr int HALF_BYTES = TILE_BYTES / 2;    // one 64-column box
 constexpr int NTHREADS = 384;
 constexpr int SMEM_DYN = 2 * TILE_BYTES + NSLOT * TILE_BYTES + 1024;   // Q (2 blocks) + ring + alignment slack
 constexpr int MAXSEG = 16;       // segments planned per round
+constexpr int kStreamMinTiles = 64;   // shorter per-CTA ranges use one piece per CTA instead of stream-K
 constexpr size_t SLOT_FLOATS = (size_t)BR * (D + 2);   // O[BR][D], then m2[BR], then l[BR]
 constexpr float kLog2e = 1.4426950408889634f;
 constexpr float kLn2 = 0.6931471805599453f;
@@ -64,9 +72,9 @@ struct TcArgs {
     int G;
 };
 
-// barrier indices: ring slots; S ready / P ready per row block; Q staged; O final
+// barrier indices: ring slots; S ready / P ready per row block; Q staged; O final; Q no longer needed
 enum { BAR_FULL = 0, BAR_EMPTY = NSLOT, BAR_S = 2 * NSLOT, BAR_P = 2 * NSLOT + 2, BAR_Q = 2 * NSLOT + 4, BAR_O = 2 * NSLOT + 5,
-       BAR_COUNT = 2 * NSLOT + 6 };
+       BAR_QFREE = 2 * NSLOT + 6, BAR_COUNT = 2 * NSLOT + 7 };
 
 // ---------------------------------------------------------------------------------------------------
 // schedule: items laid end to end, cut into equal tile ranges
@@ -85,9 +93,21 @@ __device__ __forceinline__ void seq_shape(const graft_attn_params& p, int G, int
     nrb = (T * G + BR - 1) / BR;
 }
 
-// Warp-cooperative scan over the sequences.  Returns the sequence that holds global tile `g`
-// (want_b < 0) or sequence want_b; `total` receives the number of tiles of the whole batch.
-__device__ __forceinline__ SeqInfo scan_sequences(const graft_attn_params& p, int G, long long g, int want_b, long long& total) {
+// An item of ntiles tiles in pieces of about `per` tiles: nsplit equal, non-empty pieces of plen tiles.
+__device__ __forceinline__ void piece_shape(int ntiles, long long per, int& nsplit, int& plen) {
+    nsplit = plen = 0;
+    if (ntiles <= 0) return;
+    long long want = ntiles / per;
+    if (want < 1) want = 1;
+    plen = (int)((ntiles + want - 1) / want);
+    nsplit = (ntiles + plen - 1) / plen;
+}
+
+// Warp-cooperative scan over the sequences.  Every sequence has a weight: its tiles over all its items
+// (per_piece == 0, stream-K cut) or its pieces (per_piece > 0, one-piece-per-CTA cut).  Returns the
+// sequence whose weight interval holds `g` (want_b < 0) or sequence want_b; `total` receives the sum.
+__device__ __forceinline__ SeqInfo scan_sequences(const graft_attn_params& p, int G, long long g, int want_b, long long& total,
+                                                  long long per_piece = 0) {
     const int lane = threadIdx.x & 31;
     SeqInfo out;
     out.found = false;
@@ -98,7 +118,12 @@ __device__ __forceinline__ SeqInfo scan_sequences(const graft_attn_params& p, in
         const int b = b0 + lane;
         int L = 0, T = 0, nrb = 0, ntiles = 0;
         if (b < p.B) seq_shape(p, G, b, L, T, nrb, ntiles);
-        const long long cnt = (long long)p.Hkv * nrb * ntiles;
+        long long cnt = (long long)p.Hkv * nrb * ntiles;
+        if (per_piece > 0) {
+            int nsplit, plen;
+            piece_shape(ntiles, per_piece, nsplit, plen);
+            cnt = (long long)p.Hkv * nrb * nsplit;
+        }
         long long incl = cnt;
 #pragma unroll
         for (int o = 1; o < 32; o <<= 1) {
@@ -122,6 +147,20 @@ __device__ __forceinline__ SeqInfo scan_sequences(const graft_attn_params& p, in
     }
     total = run;
     return out;
+}
+
+// The cut of a batch over `grid` CTAs (warp-cooperative): per = tiles per CTA; pieces = true selects the
+// one-piece-per-CTA cut.
+__device__ __forceinline__ void choose_cut(const graft_attn_params& p, int G, int grid, long long& total, long long& per, bool& pieces) {
+    (void)scan_sequences(p, G, 0, -1, total);
+    per = (total + grid - 1) / grid;
+    if (per < 1) per = 1;
+    pieces = false;
+    if (per < kStreamMinTiles) {
+        long long units;
+        (void)scan_sequences(p, G, 0, -1, units, per);
+        pieces = units <= grid;
+    }
 }
 
 struct Seg {
@@ -273,6 +312,13 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap kmap, const __grid_constant__
     const graft_attn_params& p = a.p;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int G = a.G;
+#ifdef GRAFT_TC_EXPERIMENTS
+    const long long t_entry = clock64();
+    const bool prof = blockIdx.x == 0 && threadIdx.x == 128;
+#define STAMP(i) do { if (prof) status[16 + (i)] = (unsigned)(clock64() - t_entry); } while (0)
+#else
+#define STAMP(i) do { } while (0)
+#endif
 
     const uint32_t sQ = (smem_u32(smem_raw) + 1023u) & ~1023u;
     const uint32_t sRing = sQ + 2 * TILE_BYTES;
@@ -316,36 +362,117 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap kmap, const __grid_constant__
         if (lane == 0) { s_nseg = n; s_gnext = g; }
     };
 
+    // Q rows of an item into shared memory, K-major with the 128-byte swizzle (16-byte chunk c of row r at
+    // c ^ (r & 7)), by `nthr` threads numbered tid = 0 .. nthr-1; 16 independent global loads per thread and round
+    auto stage_q = [&](const Seg& sg, int tid, int nthr) {
+        const int R = sg.T * G;
+        const int row0 = sg.rb * BR;
+        const __nv_bfloat16* Qg = reinterpret_cast<const __nv_bfloat16*>(p.Q) + (size_t)sg.b * p.q_stride_b +
+                                  (size_t)sg.h * G * p.q_stride_h;
+        for (int c0 = 0; c0 < BR * 16; c0 += nthr * 16) {
+            uint4 v[16];
+#pragma unroll
+            for (int q = 0; q < 16; ++q) {
+                const int c = c0 + tid + q * nthr;
+                const int r = row0 + (c >> 4);
+                v[q] = make_uint4(0u, 0u, 0u, 0u);
+                if (c < BR * 16 && r < R) {
+                    const int t = r / G, g = r % G;
+                    v[q] = *reinterpret_cast<const uint4*>(Qg + (size_t)t * p.q_stride_t + (size_t)g * p.q_stride_h + (c & 15) * 8);
+                }
+            }
+#pragma unroll
+            for (int q = 0; q < 16; ++q) {
+                const int c = c0 + tid + q * nthr;
+                if (c < BR * 16) {
+                    const int qr = c >> 4, ch = c & 15;
+                    const int qb = qr >> 7, rr = qr & 127;
+                    const uint32_t dst = sQ + qb * TILE_BYTES + (ch >> 3) * HALF_BYTES + rr * 128 + (((ch & 7) ^ (rr & 7)) << 4);
+                    asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(dst), "r"(v[q].x), "r"(v[q].y), "r"(v[q].z), "r"(v[q].w) : "memory");
+                }
+            }
+        }
+        fence_async_smem();
+    };
+
     long long g_lo_cta = 0;
     if (warp == 0) {
-        long long total;
-        (void)scan_sequences(p, G, 0, -1, total);
-        const long long per = (total + gridDim.x - 1) / gridDim.x;
-        g_lo_cta = per * blockIdx.x;
-        long long g_hi = g_lo_cta + per;
-        if (g_hi > total) g_hi = total;
-        if (g_lo_cta > total) g_lo_cta = total;
-        if (lane == 0) { s_ghi = g_hi; s_abort = 0; }
-        plan_round(g_lo_cta, g_lo_cta, g_hi);
+        long long total, per;
+        bool pieces;
+        choose_cut(p, G, (int)gridDim.x, total, per, pieces);
+        if (lane == 0) s_abort = 0;
+        if (pieces) {
+            // exactly one piece of one item for this CTA
+            long long units;
+            const SeqInfo si = scan_sequences(p, G, blockIdx.x, -1, units, per);
+            if (lane == 0) {
+                s_nseg = 0;
+                s_gnext = s_ghi = 0;
+                if (si.found) {
+                    int nsplit, plen;
+                    piece_shape(si.ntiles, per, nsplit, plen);
+                    const int local = (int)(blockIdx.x - si.base);
+                    const int k = local / nsplit, sp = local % nsplit;
+                    Seg sg;
+                    sg.b = si.b;
+                    sg.h = k / si.nrb;
+                    sg.rb = k % si.nrb;
+                    sg.tile_lo = sp * plen;
+                    sg.tile_hi = min(si.ntiles, sg.tile_lo + plen);
+                    sg.L = si.L;
+                    sg.T = si.T;
+                    sg.slot = nsplit == 1 ? -1 : 2 * (int)blockIdx.x;
+                    s_seg[0] = sg;
+                    s_nseg = 1;
+                }
+            }
+        } else {
+            g_lo_cta = per * blockIdx.x;
+            long long g_hi = g_lo_cta + per;
+            if (g_hi > total) g_hi = total;
+            if (g_lo_cta > total) g_lo_cta = total;
+            if (lane == 0) s_ghi = g_hi;
+            plan_round(g_lo_cta, g_lo_cta, g_hi);
+        }
     }
     __syncthreads();
     if (s_nseg == 0) return;                      // nothing for this CTA (short batch)
 
+    // ring load n of a segment's tile t: K (which = 0) or V (which = 1)
+    auto issue_load = [&](const Seg& sg, int t, int which, int n) {
+        const int slot = n % NSLOT;
+        const uint32_t dst = sRing + slot * TILE_BYTES;
+        const CUtensorMap* map = which ? &vmap : &kmap;
+        mbar_expect_tx(bar(BAR_FULL + slot), TILE_BYTES);
+        tma_load_4d(dst, map, 0, t * BN, sg.h, sg.b, bar(BAR_FULL + slot));
+        tma_load_4d(dst + HALF_BYTES, map, 64, t * BN, sg.h, sg.b, bar(BAR_FULL + slot));
+    };
+    int n_prefetched = 0;      // producer thread: ring loads already issued here, before Q is staged
     if (threadIdx.x == 0) {
         for (int i = 0; i < NSLOT; ++i) { mbar_init(bar(BAR_FULL + i), 1); mbar_init(bar(BAR_EMPTY + i), 1); }
         for (int i = 0; i < 2; ++i) { mbar_init(bar(BAR_S + i), 1); mbar_init(bar(BAR_P + i), 4); }
-        mbar_init(bar(BAR_Q), 8);
+        mbar_init(bar(BAR_Q), 2);                  // the two stager warps
         mbar_init(bar(BAR_O), 1);
+        mbar_init(bar(BAR_QFREE), 1);
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        // fill the ring at once: these copies overlap the staging of Q below
+        for (int si = 0; si < s_nseg && n_prefetched < NSLOT; ++si) {
+            const Seg sg = s_seg[si];
+            for (int t = sg.tile_lo; t < sg.tile_hi && n_prefetched < NSLOT; ++t)
+                for (int which = 0; which < 2 && n_prefetched < NSLOT; ++which, ++n_prefetched) issue_load(sg, t, which, n_prefetched);
+        }
     }
     if (warp == 1) {
         asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&s_tmem)), "r"(512u) : "memory");
         asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
     }
+    stage_q(s_seg[0], threadIdx.x, NTHREADS);      // the first segment's Q, by everyone
+    STAMP(0);
     tc_fence_before();
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem = s_tmem;
+    STAMP(1);
 
     // running counters that persist across segments and rounds (each role keeps its own copy)
     int n_load = 0;            // ring loads issued / consumed so far (2 per tile)
@@ -362,13 +489,10 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap kmap, const __grid_constant__
                     const Seg sg = s_seg[si];
                     for (int t = sg.tile_lo; t < sg.tile_hi; ++t)
                         for (int which = 0; which < 2; ++which, ++n_load) {
+                            if (n_load < n_prefetched) continue;          // issued before Q was staged
                             const int slot = n_load % NSLOT, use = n_load / NSLOT;
                             if (use > 0) mbar_wait(bar(BAR_EMPTY + slot), (use - 1) & 1, abort_flag, status);
-                            const uint32_t dst = sRing + slot * TILE_BYTES;
-                            const CUtensorMap* map = which ? &vmap : &kmap;
-                            mbar_expect_tx(bar(BAR_FULL + slot), TILE_BYTES);
-                            tma_load_4d(dst, map, 0, t * BN, sg.h, sg.b, bar(BAR_FULL + slot));
-                            tma_load_4d(dst + HALF_BYTES, map, 64, t * BN, sg.h, sg.b, bar(BAR_FULL + slot));
+                            issue_load(sg, t, which, n_load);
                         }
                 }
             }
@@ -405,16 +529,30 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap kmap, const __grid_constant__
                     wait_full(n_load);
                     tc_fence_after();
                     for (int blk = 0; blk < nblk; ++blk) issue_qk(blk, n_load);
+                    if (nt == 1) tc_commit(bar(BAR_QFREE));          // the segment's last Q K^T is in the pipe
                     for (int j = 0; j < nt; ++j) {
                         const int nV = n_load + 2 * j + 1, nK1 = n_load + 2 * j + 2;
                         for (int blk = 0; blk < nblk; ++blk) {
                             mbar_wait(bar(BAR_P + blk), (jt[blk] + j) & 1, abort_flag, status);
+#ifdef GRAFT_TC_EXPERIMENTS
+                            if (blockIdx.x == 0 && n_seg_done == 0 && j < 2) status[40 + j * 8 + blk * 4 + 0] = (unsigned)(clock64() - t_entry);
+#endif
                             if (blk == 0) wait_full(nV);
+#ifdef GRAFT_TC_EXPERIMENTS
+                            if (blockIdx.x == 0 && n_seg_done == 0 && j < 2) status[40 + j * 8 + blk * 4 + 1] = (unsigned)(clock64() - t_entry);
+#endif
                             tc_fence_after();
                             issue_pv(blk, nV, j == 0);
                             if (j + 1 < nt) {
                                 if (blk == 0) { wait_full(nK1); tc_fence_after(); }
+#ifdef GRAFT_TC_EXPERIMENTS
+                                if (blockIdx.x == 0 && n_seg_done == 0 && j < 2) status[40 + j * 8 + blk * 4 + 2] = (unsigned)(clock64() - t_entry);
+#endif
                                 issue_qk(blk, nK1);
+#ifdef GRAFT_TC_EXPERIMENTS
+                                if (blockIdx.x == 0 && n_seg_done == 0 && j < 2) status[40 + j * 8 + blk * 4 + 3] = (unsigned)(clock64() - t_entry);
+#endif
+                                if (blk == nblk - 1 && j + 2 == nt) tc_commit(bar(BAR_QFREE));
                             }
                         }
                     }
@@ -424,8 +562,19 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap kmap, const __grid_constant__
                     ++n_seg_done;
                 }
             }
+        } else if (warp == 2 || warp == 3) {
+            // =============================== Q stagers ===============================
+            for (int si = 0; si < nseg; ++si) {
+                const Seg sg = s_seg[si];
+                // Q may be overwritten once the previous segment's last Q K^T is complete (one phase per segment)
+                if (n_seg_done > 0) mbar_wait(bar(BAR_QFREE), (n_seg_done - 1) & 1, abort_flag, status);
+                if (n_seg_done > 0) stage_q(sg, threadIdx.x - 64, 64);      // the first segment's Q was staged by all warps
+                __syncwarp();
+                if (lane == 0) mbar_arrive(bar(BAR_Q));
+                ++n_seg_done;
+            }
         } else if (warp >= 4) {
-            // =============================== Q staging, softmax, results ===============================
+            // =============================== softmax, results ===============================
             const int blk = (warp - 4) >> 2;
             const int rl = ((warp & 3) << 5) + lane;            // row inside the block = TMEM lane
             const uint32_t lane_bits = (uint32_t)((warp & 3) << 5) << 16;
@@ -440,37 +589,6 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap kmap, const __grid_constant__
                 const int nblk = (R - row0 > 128) ? 2 : 1;
                 const int n_keys = sg.L + sg.T;
 
-                // ---- Q rows of this item into shared memory, K-major with the 128-byte swizzle (16-byte chunk
-                // c of row r at c ^ (r & 7)).  The previous segment's MMAs are complete (its O was read).
-                {
-                    const __nv_bfloat16* Qg = reinterpret_cast<const __nv_bfloat16*>(p.Q) + (size_t)sg.b * p.q_stride_b +
-                                              (size_t)sg.h * G * p.q_stride_h;
-                    const int tid = threadIdx.x - 128;           // 0..255
-                    constexpr int PER = BR * 16 / 256;
-                    uint4 v[PER];
-#pragma unroll
-                    for (int q = 0; q < PER; ++q) {
-                        const int c = tid + q * 256;
-                        const int r = row0 + (c >> 4);
-                        v[q] = make_uint4(0u, 0u, 0u, 0u);
-                        if (r < R) {
-                            const int t = r / G, g = r % G;
-                            v[q] = *reinterpret_cast<const uint4*>(Qg + (size_t)t * p.q_stride_t + (size_t)g * p.q_stride_h + (c & 15) * 8);
-                        }
-                    }
-#pragma unroll
-                    for (int q = 0; q < PER; ++q) {
-                        const int c = tid + q * 256;
-                        const int qr = c >> 4, ch = c & 15;
-                        const int qb = qr >> 7, rr = qr & 127;
-                        const uint32_t dst = sQ + qb * TILE_BYTES + (ch >> 3) * HALF_BYTES + rr * 128 + (((ch & 7) ^ (rr & 7)) << 4);
-                        asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(dst), "r"(v[q].x), "r"(v[q].y), "r"(v[q].z), "r"(v[q].w) : "memory");
-                    }
-                    fence_async_smem();
-                    __syncwarp();
-                    if (lane == 0) mbar_arrive(bar(BAR_Q));
-                }
-
                 if (blk < nblk) {
                     const int r = row0 + blk * 128 + rl;
                     const bool row_valid = r < R;
@@ -483,6 +601,8 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap kmap, const __grid_constant__
                         const bool boundary = key0 + BN > sg.L;
                         mbar_wait(bar(BAR_S + blk), (jt[blk] + j) & 1, abort_flag, status);
                         tc_fence_after();
+                        if (j == 0) STAMP(3 + 8 * min(si, 1));
+                        if (j == 1) STAMP(4 + 8 * min(si, 1));
                         auto mask32 = [&](uint32_t (&x)[32], int col0) {    // ancestor mask and the end of the tree's keys
 #pragma unroll
                             for (int q = 0; q < 32; ++q) {
@@ -585,9 +705,11 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap kmap, const __grid_constant__
                         if (lane == 0) mbar_arrive(bar(BAR_P + blk));      // one arrival per warp
                     }
 
+                    STAMP(5 + 8 * min(si, 1));
                     // ---- results of the segment: O row from TMEM, final rows or a partial
                     mbar_wait(bar(BAR_O), n_seg_done & 1, abort_flag, status);     // every MMA of the segment is complete
                     tc_fence_after();
+                    STAMP(6 + 8 * min(si, 1));
                     if (sg.slot < 0) {
                         const float inv = l > 0.f ? 1.f / l : 0.f;
                         __nv_bfloat16* orow = reinterpret_cast<__nv_bfloat16*>(p.O) + (size_t)sg.b * p.o_stride_b + (size_t)t * p.o_stride_t +
@@ -630,11 +752,11 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap kmap, const __grid_constant__
                         base[BR * D + BR + lr] = l;
                     }
                     tc_fence_before();                 // TMEM reads done before the next segment's MMAs are released
+                    STAMP(7 + 8 * min(si, 1));
+#ifdef GRAFT_TC_EXPERIMENTS
+                    if (prof) status[15] = (unsigned)nt;
+#endif
                     jt[blk] += nt;
-                } else {
-                    // a row block without rows in this item still has to see the segment's MMAs finished
-                    // before it overwrites Q for the next one
-                    mbar_wait(bar(BAR_O), n_seg_done & 1, abort_flag, status);
                 }
                 n_load += 2 * nt;
                 ++n_seg_done;
@@ -686,12 +808,17 @@ __global__ void __launch_bounds__(kMergeRows * 32, 2) merge_streamk_kernel(TcArg
     const int b = idx / p.Hkv;
     __shared__ SeqInfo s_info;
     __shared__ long long s_per;
+    __shared__ int s_pieces;
     if (threadIdx.x < 32) {
-        long long total;
-        const SeqInfo si = scan_sequences(p, G, 0, b, total);
+        long long total, per;
+        bool pieces;
+        choose_cut(p, G, grid_attn, total, per, pieces);
+        long long dummy;
+        const SeqInfo si = scan_sequences(p, G, 0, b, dummy, pieces ? per : 0);
         if (threadIdx.x == 0) {
             s_info = si;
-            s_per = (total + grid_attn - 1) / grid_attn;
+            s_per = per;
+            s_pieces = pieces;
             const int T = p.tree_size[b], L = p.seq_len[b];
             if (grp == 0 && h == 0 && (T < 0 || T > p.T_max || L < 0 || (long long)L + T > p.S_cap))
                 atomicOr(status, (unsigned)GRAFT_FLAG_BAD_SIZE);
@@ -700,6 +827,7 @@ __global__ void __launch_bounds__(kMergeRows * 32, 2) merge_streamk_kernel(TcArg
     __syncthreads();
     const SeqInfo si = s_info;
     const long long per = s_per;
+    const bool pieces = s_pieces != 0;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int r = grp * kMergeRows + warp;
     if (r >= rows_pad) return;
@@ -713,16 +841,31 @@ __global__ void __launch_bounds__(kMergeRows * 32, 2) merge_streamk_kernel(TcArg
         return;
     }
     const int rb = r / BR, rl = r % BR;
-    const long long item_lo = si.base + ((long long)h * si.nrb + rb) * si.ntiles;
-    const long long item_hi = item_lo + si.ntiles;
-    const int c_first = (int)(item_lo / per), c_last = (int)((item_hi - 1) / per);
-    const int nparts = c_last - c_first + 1;
+    // the partial slots that hold pieces of this item, from the same cut as in the attention kernel
+    int nparts, c_first = 0, piece_cta0 = 0;
+    long long item_lo = 0;
+    if (pieces) {
+        int nsplit, plen;
+        piece_shape(si.ntiles, per, nsplit, plen);
+        nparts = nsplit;
+        piece_cta0 = (int)si.base + (h * si.nrb + rb) * nsplit;      // CTA of the item's first piece
+    } else {
+        item_lo = si.base + ((long long)h * si.nrb + rb) * si.ntiles;
+        const long long item_hi = item_lo + si.ntiles;
+        c_first = (int)(item_lo / per);
+        nparts = (int)((item_hi - 1) / per) - c_first + 1;
+    }
     if (nparts <= 1) return;               // one CTA had the whole item and wrote the final rows
-    // part i lives in CTA c_first + i: its first slot if the item was already running when that CTA's
-    // range began, else its second
+    // stream-K: part i lives in CTA c_first + i, in its first slot if the item was already running when
+    // that CTA's range began, else in its second
     auto part_base = [&](int i) {
-        const int c = c_first + i;
-        const int slot = 2 * c + ((item_lo <= (long long)c * per) ? 0 : 1);
+        int slot;
+        if (pieces) {
+            slot = 2 * (piece_cta0 + i);
+        } else {
+            const int c = c_first + i;
+            slot = 2 * c + ((item_lo <= (long long)c * per) ? 0 : 1);
+        }
         return a.partial + (size_t)slot * SLOT_FLOATS;
     };
     float acc[4] = {0.f, 0.f, 0.f, 0.f};
