@@ -3,18 +3,19 @@
 //
 // Work.  An item is (sequence b, KV head h, row block rb): up to 256 rows (two blocks of 128; row r
 // <-> tree node r / G, query head h*G + r % G) against the ceil((L_b+T_b)/128) key tiles of b, so every
-// K/V byte crosses HBM once for all rows that need it.  Items are laid end to end, ordered (b, h, rb);
-// the resulting tile sequence is cut into gridDim.x equal contiguous ranges, one per CTA (one CTA per
-// SM).  A CTA therefore works through a few segments (item, tile range); a segment that covers its
-// whole item writes the final rows, any other writes a partial (row max, row sum, un-normalised O)
-// into one of the CTA's two workspace slots, and merge_streamk_kernel combines the partials of an
-// item.  When that range would be short (fewer than kStreamMinTiles tiles per CTA) a segment switch
-// (results out, next Q in, pipeline refill) is not amortised; the cut then falls back to whole
-// pieces: every item is divided into equal pieces of about that length and each CTA takes exactly one
-// piece, provided there are no more pieces than CTAs.  Either cut is a pure function of (seq_len,
-// tree_size, gridDim.x), recomputed on the device by every CTA and by the merge kernel: no
-// communication, no atomics on floats, no waiting between CTAs, bit-reproducible results for a given
-// GPU model.
+// K/V byte crosses HBM once for all rows that need it.  A tile of an item costs kW2 units if it carries
+// two 128-row blocks and kW1 if one.  Items are laid end to end, ordered (b, h, rb); the resulting unit axis is
+// cut into gridDim.x equal ranges, one per CTA (one CTA per SM), and a tile belongs to the CTA whose
+// range holds its first unit.  A CTA therefore works through a few segments (item, tile range); a
+// segment that covers its whole item writes the final rows, any other writes a partial (row max, row
+// sum, un-normalised O) into one of the CTA's two workspace slots and records the item in the slot's
+// descriptor, and merge_streamk_kernel combines the partials of an item.  When a CTA's range would be
+// short (fewer than kStreamMinTiles tiles) a segment switch (results out, pipeline refill) is not
+// amortised; the cut then falls back to whole pieces: every item is divided into equal pieces of
+// about that length and each CTA takes exactly one piece, provided there are no more pieces than
+// CTAs.  Either cut is a pure function of (seq_len, tree_size, gridDim.x), recomputed on the device
+// by every CTA and by the merge kernel: no communication, no atomics on floats, no waiting between
+// CTAs, bit-reproducible results for a given GPU model.
 //
 // Warp roles inside a CTA:
 //   warp 0      TMA producer: K and V tiles (two 64-column boxes each, 128-byte swizzle) into a
@@ -59,6 +60,7 @@ constexpr int HALF_BYTES = TILE_BYTES / 2;    // one 64-column box
 constexpr int NTHREADS = 384;
 constexpr int SMEM_DYN = 2 * TILE_BYTES + NSLOT * TILE_BYTES + 1024;   // Q (2 blocks) + ring + alignment slack
 constexpr int MAXSEG = 16;       // segments planned per round
+constexpr int kW2 = 5, kW1 = 4;        // cost units of a tile that carries two / one 128-row blocks (measured ratio ~1.25)
 constexpr int kStreamMinTiles = 64;   // shorter per-CTA ranges use one piece per CTA instead of stream-K
 constexpr size_t SLOT_FLOATS = (size_t)BR * (D + 2);   // O[BR][D], then m2[BR], then l[BR]
 constexpr float kLog2e = 1.4426950408889634f;
@@ -66,10 +68,20 @@ constexpr float kLn2 = 0.6931471805599453f;
 constexpr float kRescaleThreshold = 8.0f;     // log2 units
 constexpr long long kWaitCycles = 1ll << 31;  // about a second
 
+// Workspace after the header: slot descriptors (2 ints per CTA), then the cut of this call (written by
+// CTA 0 for the merge kernel: one CutHeader, one SeqEntry per sequence), then the partial slots.
+constexpr size_t kDescBytes = 2048;
+struct CutHeader { long long per; int pieces; int pad; };
+struct SeqEntry { long long base; int L, T, nrb, ntiles, wlast, pad; };
+__host__ __device__ constexpr size_t cut_bytes(int B) { return (sizeof(CutHeader) + (size_t)B * sizeof(SeqEntry) + 255) / 256 * 256; }
+
 struct TcArgs {
     graft_attn_params p;
-    float* partial;     // workspace after the header: 2 slots per CTA
+    int* desc;          // [2 * grid] item id held by each partial slot of this call, -1 if none
+    CutHeader* cut;     // this call's cut, followed by B SeqEntry records
+    float* partial;     // 2 slots per CTA
     int G;
+    int prof_cta;       // experiments: CTA whose timeline is recorded
 };
 
 // barrier indices: ring slots; S ready / P ready per row block; Q staged; O final; Q no longer needed
@@ -81,16 +93,22 @@ enum { BAR_FULL = 0, BAR_EMPTY = NSLOT, BAR_S = 2 * NSLOT, BAR_P = 2 * NSLOT + 2
 // ---------------------------------------------------------------------------------------------------
 struct SeqInfo {
     int b, L, T, nrb, ntiles;
-    long long base;      // global tile index of the sequence's first item
+    int wlast;           // cost units per tile of the last row block (kW1 or kW2); the others cost kW2
+    long long base;      // position of the sequence's first item on the cut axis
     bool found;
 };
 
-__device__ __forceinline__ void seq_shape(const graft_attn_params& p, int G, int b, int& L, int& T, int& nrb, int& ntiles) {
+__device__ __forceinline__ void seq_shape(const graft_attn_params& p, int G, int b, int& L, int& T, int& nrb, int& ntiles, int& wlast) {
     L = p.seq_len[b];
     T = p.tree_size[b];
     if (T < 0 || T > p.T_max || L < 0 || (long long)L + T > (long long)p.S_cap) { L = 0; T = 0; }   // invalid: no work
     ntiles = T > 0 ? (L + T + BN - 1) / BN : 0;
     nrb = (T * G + BR - 1) / BR;
+    wlast = (T * G - (nrb - 1) * BR > 128) ? kW2 : kW1;
+}
+// units of one KV head of a sequence
+__device__ __forceinline__ long long head_units(int ntiles, int nrb, int wlast) {
+    return nrb > 0 ? (long long)ntiles * (kW2 * (nrb - 1) + wlast) : 0;
 }
 
 // An item of ntiles tiles in pieces of about `per` tiles: nsplit equal, non-empty pieces of plen tiles.
@@ -103,27 +121,29 @@ __device__ __forceinline__ void piece_shape(int ntiles, long long per, int& nspl
     nsplit = (ntiles + plen - 1) / plen;
 }
 
-// Warp-cooperative scan over the sequences.  Every sequence has a weight: its tiles over all its items
-// (per_piece == 0, stream-K cut) or its pieces (per_piece > 0, one-piece-per-CTA cut).  Returns the
-// sequence whose weight interval holds `g` (want_b < 0) or sequence want_b; `total` receives the sum.
+// Warp-cooperative scan over the sequences.  The cut axis counts units (per_piece == 0, stream-K cut) or
+// pieces (per_piece > 0, one-piece-per-CTA cut with pieces of about per_piece tiles).  Returns the
+// sequence whose interval holds `g` (want_b < 0) or sequence want_b; `total` receives the axis length,
+// `total_tiles` the number of tiles of the batch.
 __device__ __forceinline__ SeqInfo scan_sequences(const graft_attn_params& p, int G, long long g, int want_b, long long& total,
-                                                  long long per_piece = 0) {
+                                                  long long& total_tiles, long long per_piece, SeqEntry* table = nullptr) {
     const int lane = threadIdx.x & 31;
     SeqInfo out;
     out.found = false;
-    out.b = out.L = out.T = out.nrb = out.ntiles = 0;
+    out.b = out.L = out.T = out.nrb = out.ntiles = out.wlast = 0;
     out.base = 0;
-    long long run = 0;
+    long long run = 0, tiles = 0;
     for (int b0 = 0; b0 < p.B; b0 += 32) {
         const int b = b0 + lane;
-        int L = 0, T = 0, nrb = 0, ntiles = 0;
-        if (b < p.B) seq_shape(p, G, b, L, T, nrb, ntiles);
-        long long cnt = (long long)p.Hkv * nrb * ntiles;
+        int L = 0, T = 0, nrb = 0, ntiles = 0, wlast = 1;
+        if (b < p.B) seq_shape(p, G, b, L, T, nrb, ntiles, wlast);
+        long long cnt = (long long)p.Hkv * head_units(ntiles, nrb, wlast);
         if (per_piece > 0) {
             int nsplit, plen;
             piece_shape(ntiles, per_piece, nsplit, plen);
             cnt = (long long)p.Hkv * nrb * nsplit;
         }
+        tiles += (long long)p.Hkv * nrb * ntiles;
         long long incl = cnt;
 #pragma unroll
         for (int o = 1; o < 32; o <<= 1) {
@@ -131,6 +151,11 @@ __device__ __forceinline__ SeqInfo scan_sequences(const graft_attn_params& p, in
             if (lane >= o) incl += v;
         }
         const long long start = run + incl - cnt;
+        if (table && b < p.B) {
+            SeqEntry e;
+            e.base = start; e.L = L; e.T = T; e.nrb = nrb; e.ntiles = ntiles; e.wlast = wlast; e.pad = 0;
+            table[b] = e;
+        }
         const bool hit = b < p.B && !out.found && (want_b >= 0 ? b == want_b : (cnt > 0 && g >= start && g < start + cnt));
         const unsigned m = __ballot_sync(0xffffffffu, hit);
         if (m) {
@@ -141,27 +166,47 @@ __device__ __forceinline__ SeqInfo scan_sequences(const graft_attn_params& p, in
             out.T = __shfl_sync(0xffffffffu, T, src);
             out.nrb = __shfl_sync(0xffffffffu, nrb, src);
             out.ntiles = __shfl_sync(0xffffffffu, ntiles, src);
+            out.wlast = __shfl_sync(0xffffffffu, wlast, src);
             out.base = __shfl_sync(0xffffffffu, start, src);
         }
         run += __shfl_sync(0xffffffffu, incl, 31);
     }
+#pragma unroll
+    for (int o = 16; o; o >>= 1) tiles += __shfl_xor_sync(0xffffffffu, tiles, o);
     total = run;
+    total_tiles = tiles;
     return out;
 }
 
-// The cut of a batch over `grid` CTAs (warp-cooperative): per = tiles per CTA; pieces = true selects the
-// one-piece-per-CTA cut.
-__device__ __forceinline__ void choose_cut(const graft_attn_params& p, int G, int grid, long long& total, long long& per, bool& pieces) {
-    (void)scan_sequences(p, G, 0, -1, total);
-    per = (total + grid - 1) / grid;
-    if (per < 1) per = 1;
+// The cut of a batch over `grid` CTAs (warp-cooperative).  pieces = false: stream-K, `per` units per CTA
+// out of `total`; pieces = true: one piece of about `per` tiles per CTA.
+__device__ __forceinline__ void choose_cut(const graft_attn_params& p, int G, int grid, long long& total, long long& per, bool& pieces,
+                                           CutHeader* record = nullptr) {
+    SeqEntry* table = record ? reinterpret_cast<SeqEntry*>(record + 1) : nullptr;
+    long long tiles;
+    (void)scan_sequences(p, G, 0, -1, total, tiles, 0, table);
+    const long long per_tiles = (tiles + grid - 1) / grid > 0 ? (tiles + grid - 1) / grid : 1;
     pieces = false;
-    if (per < kStreamMinTiles) {
-        long long units;
-        (void)scan_sequences(p, G, 0, -1, units, per);
-        pieces = units <= grid;
+    per = (total + grid - 1) / grid;
+    if (per < kW2) per = kW2;   // a range never shorter than the heaviest tile, so every CTA inside an item's span owns a tile
+    if (per_tiles < kStreamMinTiles) {
+        long long units, dummy;
+        (void)scan_sequences(p, G, 0, -1, units, dummy, per_tiles, nullptr);
+        if (units <= grid) {
+            pieces = true;
+            per = per_tiles;
+            if (table) (void)scan_sequences(p, G, 0, -1, units, dummy, per_tiles, table);   // bases on the piece axis
+        }
     }
+    if (record && (threadIdx.x & 31) == 0) { record->per = per; record->pieces = pieces ? 1 : 0; record->pad = 0; }
 }
+
+// position and weight of item (h, rb) of a sequence on the unit axis
+__device__ __forceinline__ void item_span(const SeqInfo& si, int h, int rb, long long& U, int& w) {
+    U = si.base + (long long)h * head_units(si.ntiles, si.nrb, si.wlast) + (long long)rb * si.ntiles * kW2;
+    w = rb < si.nrb - 1 ? kW2 : si.wlast;
+}
+__device__ __forceinline__ int item_id(const graft_attn_params& p, int b, int h, int rb) { return ((b * p.Hkv + h) << 3) | rb; }
 
 struct Seg {
     int b, h, rb;            // item
@@ -308,13 +353,14 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap kmap, const __grid_constant__
     __shared__ Seg s_seg[MAXSEG];
     __shared__ int s_nseg;
     __shared__ long long s_gnext, s_ghi;
+    __shared__ int s_npartial;
 
     const graft_attn_params& p = a.p;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int G = a.G;
 #ifdef GRAFT_TC_EXPERIMENTS
     const long long t_entry = clock64();
-    const bool prof = blockIdx.x == 0 && threadIdx.x == 128;
+    const bool prof = blockIdx.x == a.prof_cta && threadIdx.x == 128;
 #define STAMP(i) do { if (prof) status[16 + (i)] = (unsigned)(clock64() - t_entry); } while (0)
 #else
 #define STAMP(i) do { } while (0)
@@ -326,40 +372,55 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap kmap, const __grid_constant__
     auto bar = [&](int i) { return bar0 + 8u * (uint32_t)i; };
     volatile int* abort_flag = &s_abort;
 
-    // ---- this CTA's tile range, and the first round of segments
-    // plan_round (warp 0): fills s_seg with the next <= MAXSEG segments of [g, g_hi)
-    auto plan_round = [&](long long g, long long g_lo_cta, long long g_hi) {
+    // ---- this CTA's range, and the first round of segments
+    // plan_round (warp 0): fills s_seg with the next <= MAXSEG segments of the unit range [g, g_hi); g_lo is the
+    // start of the CTA's range (a tile belongs to the range that holds its first unit)
+    auto plan_round = [&](long long g, long long g_lo, long long g_hi) {
         int n = 0;
+        int n_partial = s_npartial;
         while (g < g_hi && n < MAXSEG) {
-            long long total;
-            const SeqInfo si = scan_sequences(p, G, g, -1, total);
+            long long total, tiles;
+            const SeqInfo si = scan_sequences(p, G, g, -1, total, tiles, 0);
             if (!si.found) { g = g_hi; break; }
-            // walk the items of this sequence that intersect [g, g_hi)
-            long long k = (g - si.base) / si.ntiles;
-            const long long items = (long long)p.Hkv * si.nrb;
-            while (k < items && g < g_hi && n < MAXSEG) {
-                const long long item_lo = si.base + k * si.ntiles;
-                const long long item_hi = item_lo + si.ntiles;
-                const long long e = item_hi < g_hi ? item_hi : g_hi;
-                if (lane == 0) {
-                    Seg s;
-                    s.b = si.b;
-                    s.h = (int)(k / si.nrb);
-                    s.rb = (int)(k % si.nrb);
-                    s.tile_lo = (int)(g - item_lo);
-                    s.tile_hi = (int)(e - item_lo);
-                    s.L = si.L;
-                    s.T = si.T;
-                    const bool whole = g == item_lo && e == item_hi;
-                    s.slot = whole ? -1 : 2 * (int)blockIdx.x + (g == g_lo_cta ? 0 : 1);
-                    s_seg[n] = s;
+            const long long hu = head_units(si.ntiles, si.nrb, si.wlast);
+            const long long seq_end = si.base + (long long)p.Hkv * hu;
+            // walk the items of this sequence from the one that holds unit g
+            int h = (int)((g - si.base) / hu);
+            const long long rem = (g - si.base) % hu;
+            int rb = (int)(rem / ((long long)si.ntiles * kW2));
+            if (rb > si.nrb - 1) rb = si.nrb - 1;
+            while (g < g_hi && g < seq_end && n < MAXSEG) {
+                long long U;
+                int w;
+                item_span(si, h, rb, U, w);
+                const long long item_end = U + (long long)si.ntiles * w;
+                long long t_lo = (g - U + w - 1) / w, t_hi = (g_hi - U + w - 1) / w;
+                if (t_lo < 0) t_lo = 0;
+                if (t_hi > si.ntiles) t_hi = si.ntiles;
+                if (t_lo < t_hi) {
+                    const bool whole = t_lo == 0 && t_hi == si.ntiles;
+                    if (lane == 0) {
+                        Seg sg;
+                        sg.b = si.b;
+                        sg.h = h;
+                        sg.rb = rb;
+                        sg.tile_lo = (int)t_lo;
+                        sg.tile_hi = (int)t_hi;
+                        sg.L = si.L;
+                        sg.T = si.T;
+                        sg.slot = whole ? -1 : 2 * (int)blockIdx.x + (n_partial < 1 ? n_partial : 1);
+                        s_seg[n] = sg;
+                        if (!whole) a.desc[sg.slot] = item_id(p, si.b, h, rb);
+                    }
+                    if (!whole) ++n_partial;
+                    ++n;
                 }
-                ++n;
-                g = e;
-                ++k;
+                g = item_end < g_hi ? item_end : g_hi;
+                if (++rb == si.nrb) { rb = 0; ++h; }
             }
         }
-        if (lane == 0) { s_nseg = n; s_gnext = g; }
+        (void)g_lo;
+        if (lane == 0) { s_nseg = n; s_gnext = g; s_npartial = n_partial; }
     };
 
     // Q rows of an item into shared memory, K-major with the 128-byte swizzle (16-byte chunk c of row r at
@@ -399,12 +460,18 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap kmap, const __grid_constant__
     if (warp == 0) {
         long long total, per;
         bool pieces;
-        choose_cut(p, G, (int)gridDim.x, total, per, pieces);
-        if (lane == 0) s_abort = 0;
+        choose_cut(p, G, (int)gridDim.x, total, per, pieces, blockIdx.x == 0 ? a.cut : nullptr);
+        if (lane == 0) {
+            s_abort = 0;
+            s_npartial = 0;
+            a.desc[2 * blockIdx.x] = -1;           // this call's slot descriptors
+            a.desc[2 * blockIdx.x + 1] = -1;
+        }
+        __syncwarp();
         if (pieces) {
             // exactly one piece of one item for this CTA
-            long long units;
-            const SeqInfo si = scan_sequences(p, G, blockIdx.x, -1, units, per);
+            long long units, tiles;
+            const SeqInfo si = scan_sequences(p, G, blockIdx.x, -1, units, tiles, per);
             if (lane == 0) {
                 s_nseg = 0;
                 s_gnext = s_ghi = 0;
@@ -535,22 +602,22 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap kmap, const __grid_constant__
                         for (int blk = 0; blk < nblk; ++blk) {
                             mbar_wait(bar(BAR_P + blk), (jt[blk] + j) & 1, abort_flag, status);
 #ifdef GRAFT_TC_EXPERIMENTS
-                            if (blockIdx.x == 0 && n_seg_done == 0 && j < 2) status[40 + j * 8 + blk * 4 + 0] = (unsigned)(clock64() - t_entry);
+                            if (blockIdx.x == a.prof_cta && n_seg_done == 0 && j < 2) status[40 + j * 8 + blk * 4 + 0] = (unsigned)(clock64() - t_entry);
 #endif
                             if (blk == 0) wait_full(nV);
 #ifdef GRAFT_TC_EXPERIMENTS
-                            if (blockIdx.x == 0 && n_seg_done == 0 && j < 2) status[40 + j * 8 + blk * 4 + 1] = (unsigned)(clock64() - t_entry);
+                            if (blockIdx.x == a.prof_cta && n_seg_done == 0 && j < 2) status[40 + j * 8 + blk * 4 + 1] = (unsigned)(clock64() - t_entry);
 #endif
                             tc_fence_after();
                             issue_pv(blk, nV, j == 0);
                             if (j + 1 < nt) {
                                 if (blk == 0) { wait_full(nK1); tc_fence_after(); }
 #ifdef GRAFT_TC_EXPERIMENTS
-                                if (blockIdx.x == 0 && n_seg_done == 0 && j < 2) status[40 + j * 8 + blk * 4 + 2] = (unsigned)(clock64() - t_entry);
+                                if (blockIdx.x == a.prof_cta && n_seg_done == 0 && j < 2) status[40 + j * 8 + blk * 4 + 2] = (unsigned)(clock64() - t_entry);
 #endif
                                 issue_qk(blk, nK1);
 #ifdef GRAFT_TC_EXPERIMENTS
-                                if (blockIdx.x == 0 && n_seg_done == 0 && j < 2) status[40 + j * 8 + blk * 4 + 3] = (unsigned)(clock64() - t_entry);
+                                if (blockIdx.x == a.prof_cta && n_seg_done == 0 && j < 2) status[40 + j * 8 + blk * 4 + 3] = (unsigned)(clock64() - t_entry);
 #endif
                                 if (blk == nblk - 1 && j + 2 == nt) tc_commit(bar(BAR_QFREE));
                             }
@@ -780,6 +847,15 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap kmap, const __grid_constant__
             const long long t0 = clock64();
             while (!mbar_try_wait(bar(BAR_FULL + m % NSLOT), (m / NSLOT) & 1) && clock64() - t0 < kWaitCycles) {}
         }
+#ifdef GRAFT_TC_EXPERIMENTS
+    if (threadIdx.x == 128) {      // per-CTA totals for load-balance studies
+        if (2 * gridDim.x + 3 * (blockIdx.x + 1) <= kDescBytes / 4) {
+            a.desc[2 * gridDim.x + 3 * blockIdx.x] = (int)(clock64() - t_entry);
+            a.desc[2 * gridDim.x + 3 * blockIdx.x + 1] = n_seg_done;
+            a.desc[2 * gridDim.x + 3 * blockIdx.x + 2] = n_load / 2;
+        }
+    }
+#endif
     tc_fence_before();
     __syncthreads();
     if (warp == 1) {
@@ -795,13 +871,13 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap kmap, const __grid_constant__
 // O = sum w_i O_i / sum w_i l_i;  rows of padding nodes are zeroed (LSE -inf); rows of items that one CTA
 // finished alone were already final.  The set of CTAs that hold a piece of an item follows from the
 // same cut as in the attention kernel.
-constexpr int kMergeRows = 8;
+constexpr int kMergeWarps = 8;       // warps per CTA; rows per CTA is a launch parameter (8: one per warp, or 32)
 
-__global__ void __launch_bounds__(kMergeRows * 32, 2) merge_streamk_kernel(TcArgs a, int grid_attn, unsigned* status) {
+__global__ void __launch_bounds__(kMergeWarps * 32, 2) merge_streamk_kernel(TcArgs a, int rows_per_cta, unsigned* status) {
     const graft_attn_params& p = a.p;
     const int G = a.G;
     const int rows_pad = p.T_max * G;
-    const int groups = (rows_pad + kMergeRows - 1) / kMergeRows;
+    const int groups = (rows_pad + rows_per_cta - 1) / rows_per_cta;
     int idx = blockIdx.x;
     const int grp = idx % groups; idx /= groups;
     const int h = idx % p.Hkv;
@@ -809,28 +885,24 @@ __global__ void __launch_bounds__(kMergeRows * 32, 2) merge_streamk_kernel(TcArg
     __shared__ SeqInfo s_info;
     __shared__ long long s_per;
     __shared__ int s_pieces;
-    if (threadIdx.x < 32) {
-        long long total, per;
-        bool pieces;
-        choose_cut(p, G, grid_attn, total, per, pieces);
-        long long dummy;
-        const SeqInfo si = scan_sequences(p, G, 0, b, dummy, pieces ? per : 0);
-        if (threadIdx.x == 0) {
-            s_info = si;
-            s_per = per;
-            s_pieces = pieces;
-            const int T = p.tree_size[b], L = p.seq_len[b];
-            if (grp == 0 && h == 0 && (T < 0 || T > p.T_max || L < 0 || (long long)L + T > p.S_cap))
-                atomicOr(status, (unsigned)GRAFT_FLAG_BAD_SIZE);
-        }
+    if (threadIdx.x == 0) {
+        // the cut was recorded by the attention kernel: no need to scan the batch again
+        const SeqEntry e = reinterpret_cast<const SeqEntry*>(a.cut + 1)[b];
+        SeqInfo si;
+        si.b = b; si.L = e.L; si.T = e.T; si.nrb = e.nrb; si.ntiles = e.ntiles; si.wlast = e.wlast; si.base = e.base; si.found = true;
+        s_info = si;
+        s_per = a.cut->per;
+        s_pieces = a.cut->pieces;
+        const int T = p.tree_size[b], L = p.seq_len[b];
+        if (grp == 0 && h == 0 && (T < 0 || T > p.T_max || L < 0 || (long long)L + T > p.S_cap))
+            atomicOr(status, (unsigned)GRAFT_FLAG_BAD_SIZE);
     }
     __syncthreads();
     const SeqInfo si = s_info;
     const long long per = s_per;
     const bool pieces = s_pieces != 0;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const int r = grp * kMergeRows + warp;
-    if (r >= rows_pad) return;
+    for (int r = grp * rows_per_cta + warp; r < min(rows_pad, (grp + 1) * rows_per_cta); r += kMergeWarps) {
     const int t = r / G, g = r % G;
     __nv_bfloat16* orow = reinterpret_cast<__nv_bfloat16*>(p.O) + (size_t)b * p.o_stride_b + (size_t)t * p.o_stride_t +
                           (size_t)(h * G + g) * p.o_stride_h + lane * 4;
@@ -838,47 +910,51 @@ __global__ void __launch_bounds__(kMergeRows * 32, 2) merge_streamk_kernel(TcArg
     if (t >= si.T) {                       // padding node: zero row
         *reinterpret_cast<uint2*>(orow) = make_uint2(0u, 0u);
         if (lse && lane == 0) *lse = -CUDART_INF_F;
-        return;
+        continue;
     }
     const int rb = r / BR, rl = r % BR;
     // the partial slots that hold pieces of this item, from the same cut as in the attention kernel
     int nparts, c_first = 0, piece_cta0 = 0;
-    long long item_lo = 0;
+    const int id = item_id(p, b, h, rb);
     if (pieces) {
         int nsplit, plen;
         piece_shape(si.ntiles, per, nsplit, plen);
         nparts = nsplit;
         piece_cta0 = (int)si.base + (h * si.nrb + rb) * nsplit;      // CTA of the item's first piece
     } else {
-        item_lo = si.base + ((long long)h * si.nrb + rb) * si.ntiles;
-        const long long item_hi = item_lo + si.ntiles;
-        c_first = (int)(item_lo / per);
-        nparts = (int)((item_hi - 1) / per) - c_first + 1;
+        long long U;
+        int w;
+        item_span(si, h, rb, U, w);
+        c_first = (int)(U / per);
+        nparts = (int)((U + (long long)(si.ntiles - 1) * w) / per) - c_first + 1;
     }
-    if (nparts <= 1) return;               // one CTA had the whole item and wrote the final rows
-    // stream-K: part i lives in CTA c_first + i, in its first slot if the item was already running when
-    // that CTA's range began, else in its second
-    auto part_base = [&](int i) {
+    if (nparts <= 1) continue;             // one CTA had the whole item and wrote the final rows
+    // stream-K: part i lives in CTA c_first + i, in the slot whose descriptor names this item (none if
+    // that CTA's range held no tile of the item)
+    auto part_base = [&](int i) -> const float* {
         int slot;
         if (pieces) {
             slot = 2 * (piece_cta0 + i);
         } else {
             const int c = c_first + i;
-            slot = 2 * c + ((item_lo <= (long long)c * per) ? 0 : 1);
+            slot = a.desc[2 * c] == id ? 2 * c : (a.desc[2 * c + 1] == id ? 2 * c + 1 : -1);
         }
-        return a.partial + (size_t)slot * SLOT_FLOATS;
+        return slot < 0 ? nullptr : a.partial + (size_t)slot * SLOT_FLOATS;
     };
     float acc[4] = {0.f, 0.f, 0.f, 0.f};
     float den = 0.f, M = -CUDART_INF_F;
-    for (int i = lane; i < nparts; i += 32) M = fmaxf(M, part_base(i)[BR * D + rl]);
+    for (int i = lane; i < nparts; i += 32) {
+        const float* pb = part_base(i);
+        if (pb) M = fmaxf(M, pb[BR * D + rl]);
+    }
 #pragma unroll
     for (int o = 16; o; o >>= 1) M = fmaxf(M, __shfl_xor_sync(0xffffffffu, M, o));
     for (int i0 = 0; i0 < nparts; i0 += 32) {
         float wgt = 0.f, l = 0.f;
-        if (i0 + lane < nparts) {
-            const float* pb = part_base(i0 + lane);
-            const float m = pb[BR * D + rl];
-            l = pb[BR * D + BR + rl];
+        const float* my_pb = i0 + lane < nparts ? part_base(i0 + lane) : nullptr;
+        if (my_pb) {
+            const float m = my_pb[BR * D + rl];
+            l = my_pb[BR * D + BR + rl];
             wgt = (m == -CUDART_INF_F || M == -CUDART_INF_F) ? 0.f : exp2f(m - M);
         }
         den += wgt * l;
@@ -887,7 +963,12 @@ __global__ void __launch_bounds__(kMergeRows * 32, 2) merge_streamk_kernel(TcArg
             float4 x[16];
 #pragma unroll
             for (int j = 0; j < 16; ++j)
-                if (j0 + j < cnt) x[j] = *reinterpret_cast<const float4*>(part_base(i0 + j0 + j) + (size_t)rl * D + lane * 4);
+                if (j0 + j < cnt) {
+                    // the owner lane of part j0 + j knows whether it exists; a missing part has weight 0
+                    const unsigned long long pbj = __shfl_sync(0xffffffffu, (unsigned long long)my_pb, j0 + j);
+                    x[j] = pbj ? *reinterpret_cast<const float4*>(reinterpret_cast<const float*>(pbj) + (size_t)rl * D + lane * 4)
+                               : make_float4(0.f, 0.f, 0.f, 0.f);
+                }
 #pragma unroll
             for (int j = 0; j < 16; ++j)
                 if (j0 + j < cnt) {
@@ -901,6 +982,7 @@ __global__ void __launch_bounds__(kMergeRows * 32, 2) merge_streamk_kernel(TcArg
     const float inv = den > 0.f ? 1.f / den : 0.f;
     *reinterpret_cast<uint2*>(orow) = make_uint2(pack_bf16(acc[0] * inv, acc[1] * inv), pack_bf16(acc[2] * inv, acc[3] * inv));
     if (lse && lane == 0) *lse = den > 0.f ? (M + log2f(den)) * kLn2 : -CUDART_INF_F;
+    }
 }
 
 typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
@@ -942,10 +1024,10 @@ bool graft_attn_tc_supported(const graft_ctx* ctx, const graft_attn_params* p) {
     return GRAFT_WS_HEADER + graft_attn_tc_ws_bytes(ctx->num_sms, p->B, p->Hq, p->Hkv, p->d, p->T_max) <= ctx->ws_bytes;
 }
 
-// two partial slots per CTA, one CTA per SM: independent of the batch
-size_t graft_attn_tc_ws_bytes(int num_sms, int, int, int, int d, int) {
+// two partial slots per CTA, one CTA per SM (independent of the batch), plus the recorded cut
+size_t graft_attn_tc_ws_bytes(int num_sms, int B, int, int, int d, int) {
     if (d != D) return 0;
-    return (size_t)num_sms * 2 * SLOT_FLOATS * sizeof(float);
+    return kDescBytes + cut_bytes(B) + (size_t)num_sms * 2 * SLOT_FLOATS * sizeof(float);
 }
 
 int graft_attn_tc_launch(graft_ctx* ctx, const graft_attn_params* p, cudaStream_t stream) {
@@ -955,16 +1037,25 @@ int graft_attn_tc_launch(graft_ctx* ctx, const graft_attn_params* p, cudaStream_
     if (rc != GRAFT_OK) return rc;
     TcArgs a;
     a.p = *p;
-    a.partial = reinterpret_cast<float*>(reinterpret_cast<char*>(ctx->ws) + GRAFT_WS_HEADER);
+    a.desc = reinterpret_cast<int*>(reinterpret_cast<char*>(ctx->ws) + GRAFT_WS_HEADER);
+    a.cut = reinterpret_cast<CutHeader*>(reinterpret_cast<char*>(ctx->ws) + GRAFT_WS_HEADER + kDescBytes);
+    a.partial = reinterpret_cast<float*>(reinterpret_cast<char*>(ctx->ws) + GRAFT_WS_HEADER + kDescBytes + cut_bytes(p->B));
     a.G = p->Hq / p->Hkv;
+    a.prof_cta = 0;
+#ifdef GRAFT_TC_EXPERIMENTS
+    if (getenv("GRAFT_TC_PROF_CTA")) a.prof_cta = atoi(getenv("GRAFT_TC_PROF_CTA"));
+#endif
     int grid = ctx->num_sms;
 #ifdef GRAFT_TC_EXPERIMENTS
     if (getenv("GRAFT_TC_GRID")) grid = atoi(getenv("GRAFT_TC_GRID"));
 #endif
     attn_tc_kernel<<<grid, NTHREADS, SMEM_DYN, stream>>>(kmap, vmap, a, ctx->status);
     GRAFT_CHECK_CUDA(cudaGetLastError());
-    const int groups = (p->T_max * a.G + kMergeRows - 1) / kMergeRows;
-    merge_streamk_kernel<<<p->B * p->Hkv * groups, kMergeRows * 32, 0, stream>>>(a, grid, ctx->status);
+    // few rows: one row per warp (the merge is latency-bound); many rows: four, to keep the CTA count down
+    const int rows_pad = p->T_max * a.G;
+    const int rows_per_cta = (long long)p->B * p->Hkv * rows_pad >= 16384 ? 32 : 8;
+    const int groups = (rows_pad + rows_per_cta - 1) / rows_per_cta;
+    merge_streamk_kernel<<<p->B * p->Hkv * groups, kMergeWarps * 32, 0, stream>>>(a, rows_per_cta, ctx->status);
     GRAFT_CHECK_CUDA(cudaGetLastError());
     return GRAFT_OK;
 }
