@@ -1053,7 +1053,7 @@ int graft_attn_tc_launch(graft_ctx* ctx, const graft_attn_params* p, cudaStream_
     GRAFT_CHECK_CUDA(cudaGetLastError());
     // few rows: one row per warp (the merge is latency-bound); many rows: four, to keep the CTA count down
     const int rows_pad = p->T_max * a.G;
-    const int rows_per_cta = (long long)p->B * p->Hkv * rows_pad >= 16384 ? 32 : 8;
+    const int rows_per_cta = (long long)p->B * p->Hkv * rows_pad >= 32768 ? 32 : 8;
     const int groups = (rows_pad + rows_per_cta - 1) / rows_per_cta;
     merge_streamk_kernel<<<p->B * p->Hkv * groups, kMergeWarps * 32, 0, stream>>>(a, rows_per_cta, ctx->status);
     GRAFT_CHECK_CUDA(cudaGetLastError());
