@@ -308,3 +308,53 @@ def test_full_size_configs(orc, G, Step, cfg, B, n_rows, variant):
     tree = orc.build_tree(w)
     rows = sample_rows(np.random.default_rng(int(cfg) + 100), tree["tree_size"], w.Hq, n_rows)
     full_case(orc, G, Step, w, variant, rows=rows)
+
+
+# ---------------------------------------------------------------------------------------------
+# schedule edge cases of the persistent attention kernel
+# ---------------------------------------------------------------------------------------------
+def test_many_short_sequences(orc, G, Step):
+    """Far more (sequence, KV head) items than SMs, one or two key tiles each: every CTA walks through
+    many whole items, in more than one planning round."""
+    rng = np.random.default_rng(21)
+    B = 300
+    parents = [W.random_tree_parents(rng, int(rng.integers(1, 9))) for _ in range(B)]
+    L = rng.integers(0, 200, size=B).tolist()
+    w = W.custom(parents, Hq=8, Hkv=8, d=128, L=L, T_max=8, seed=21)
+    full_case(orc, G, Step, w, "auto")
+
+
+def test_one_and_two_block_items_mixed(orc, G, Step):
+    """G = 16 with tree sizes whose last row block has at most / more than 128 rows, ragged lengths:
+    items of different cost per tile on the cut axis, several row blocks per KV head."""
+    rng = np.random.default_rng(22)
+    sizes = [5, 8, 9, 16, 17, 24, 25, 40, 41, 64, 33, 3]
+    parents = [W.random_tree_parents(rng, n) for n in sizes]
+    L = rng.integers(100, 3000, size=len(sizes)).tolist()
+    w = W.custom(parents, Hq=32, Hkv=2, d=128, L=L, T_max=64, seed=22)
+    full_case(orc, G, Step, w, "auto")
+
+
+def test_invalid_sequence_inside_a_batch(orc, G, Step):
+    """A sequence whose tree_size is out of range is skipped (zero rows, BAD_SIZE flag); the others are exact."""
+    rng = np.random.default_rng(23)
+    w = W.custom([W.random_tree_parents(rng, 20) for _ in range(3)], Hq=8, Hkv=2, d=128, L=[500, 300, 900], T_max=32,
+                 seed=23)
+    tree = orc.build_tree(w)
+    W.make_qkv(w, tree["tree_size"], poison=True)
+    vs = Step(w)
+    vs.build()
+    vs.tree_size[1] = 33                                   # larger than T_max: invalid
+    for variant in VARIANTS:
+        vs.O.fill_(float("nan"))
+        vs.attn(variant_id(G, variant))
+        torch.cuda.synchronize()
+        assert vs.ctx.device_status() == G.FLAG_BAD_SIZE
+        O = vs.O.cpu().to(torch.float64).numpy()
+        assert (O[1] == 0).all()
+        out = orc.tree_attn(W.bf16_bits(w.Q), W.bf16_bits(w.Kc), W.bf16_bits(w.Vc), w.seq_len, tree["tree_size"],
+                            tree["tree_anc"], w.scale)
+        for b in (0, 2):
+            err = np.abs(O[b, :20] - out["O"][b, :20])
+            assert err.max() <= MAX_ABS and err.mean() <= MEAN_ABS
+            assert (O[b, 20:] == 0).all()
