@@ -81,6 +81,7 @@ struct TcArgs {
     CutHeader* cut;     // this call's cut, followed by B SeqEntry records
     float* partial;     // 2 slots per CTA
     int G;
+    int q_tma;          // Q tiles are fetched by TMA (group size divides 128); otherwise threads copy them
     int prof_cta;       // experiments: CTA whose timeline is recorded
 };
 
@@ -255,6 +256,11 @@ __device__ __forceinline__ void tma_load_4d(uint32_t dst, const CUtensorMap* map
                  ::"r"(dst), "l"(map), "r"(x), "r"(y), "r"(z), "r"(w), "r"(bar) : "memory");
 }
 
+__device__ __forceinline__ void tma_load_5d(uint32_t dst, const CUtensorMap* map, int x, int y, int z, int w, int v, uint32_t bar) {
+    asm volatile("cp.async.bulk.tensor.5d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4, %5, %6}], [%7];"
+                 ::"r"(dst), "l"(map), "r"(x), "r"(y), "r"(z), "r"(w), "r"(v), "r"(bar) : "memory");
+}
+
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tc_commit(uint32_t bar) {
@@ -345,7 +351,8 @@ constexpr uint32_t kIdescPV = kIdescBase | (1u << 16);   // B (= V) MN-major
 // the kernel
 // ---------------------------------------------------------------------------------------------------
 __global__ void __launch_bounds__(NTHREADS, 1)
-attn_tc_kernel(const __grid_constant__ CUtensorMap kmap, const __grid_constant__ CUtensorMap vmap, TcArgs a, unsigned* status) {
+attn_tc_kernel(const __grid_constant__ CUtensorMap kmap, const __grid_constant__ CUtensorMap vmap, const __grid_constant__ CUtensorMap qmap,
+               TcArgs a, unsigned* status) {
     extern __shared__ unsigned char smem_raw[];
     __shared__ __align__(8) uint64_t s_bar[BAR_COUNT];
     __shared__ uint32_t s_tmem;
@@ -430,30 +437,41 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap kmap, const __grid_constant__
         const int row0 = sg.rb * BR;
         const __nv_bfloat16* Qg = reinterpret_cast<const __nv_bfloat16*>(p.Q) + (size_t)sg.b * p.q_stride_b +
                                   (size_t)sg.h * G * p.q_stride_h;
-        for (int c0 = 0; c0 < BR * 16; c0 += nthr * 16) {
-            uint4 v[16];
-#pragma unroll
-            for (int q = 0; q < 16; ++q) {
-                const int c = c0 + tid + q * nthr;
-                const int r = row0 + (c >> 4);
-                v[q] = make_uint4(0u, 0u, 0u, 0u);
-                if (c < BR * 16 && r < R) {
-                    const int t = r / G, g = r % G;
-                    v[q] = *reinterpret_cast<const uint4*>(Qg + (size_t)t * p.q_stride_t + (size_t)g * p.q_stride_h + (c & 15) * 8);
-                }
-            }
-#pragma unroll
-            for (int q = 0; q < 16; ++q) {
-                const int c = c0 + tid + q * nthr;
-                if (c < BR * 16) {
-                    const int qr = c >> 4, ch = c & 15;
-                    const int qb = qr >> 7, rr = qr & 127;
-                    const uint32_t dst = sQ + qb * TILE_BYTES + (ch >> 3) * HALF_BYTES + rr * 128 + (((ch & 7) ^ (rr & 7)) << 4);
-                    asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(dst), "r"(v[q].x), "r"(v[q].y), "r"(v[q].z), "r"(v[q].w) : "memory");
-                }
-            }
+        // asynchronous 16-byte copies, all in flight at once: the loads queue behind the K/V stream in a
+        // saturated memory system, so their latency must overlap rather than add up
+        const int step = nthr >> 4;              // rows per pass: 16 threads copy one 256-byte row
+        const int ch = tid & 15;
+        int r = row0 + (tid >> 4);
+        int g = r % G;
+        const int dt = step / G, dg = step - dt * G;
+        const __nv_bfloat16* src_t = Qg + (size_t)(r / G) * p.q_stride_t + ch * 8;       // row of tree node t, head g = 0
+        const size_t inc_t = (size_t)dt * p.q_stride_t;
+        for (int qr = tid >> 4; qr < BR; qr += step) {
+            const bool valid = r < R;
+            const __nv_bfloat16* src = valid ? src_t + (size_t)g * p.q_stride_h : Qg;
+            const int rr = qr & 127;
+            const uint32_t dst = sQ + (qr >> 7) * TILE_BYTES + (ch >> 3) * HALF_BYTES + rr * 128 + (((ch & 7) ^ (rr & 7)) << 4);
+            asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"(dst), "l"(src), "r"(valid ? 16 : 0) : "memory");   // rows past the tree read as zero
+            r += step;
+            g += dg;
+            src_t += inc_t;
+            if (g >= G) { g -= G; src_t += p.q_stride_t; }
         }
+        asm volatile("cp.async.wait_all;" ::: "memory");
         fence_async_smem();
+    };
+
+    // The same Q rows by TMA (one thread): the map's box is 64 columns x G heads x 128/G tree nodes, which lands
+    // as 128 rows r = t*G + g in the swizzled K-major layout.  Rows of tree nodes past the sequence's tree hold
+    // whatever the caller's buffer holds there (zero past T_max); their scores stay in their own accumulator
+    // rows and are never written out.  The expect_tx is one of the two arrivals of the barrier.
+    auto issue_q = [&](const Seg& sg) {
+        const int row0 = sg.rb * BR;
+        const int nblk = (sg.T * G - row0 > 128) ? 2 : 1;
+        mbar_expect_tx(bar(BAR_Q), nblk * TILE_BYTES);
+        for (int blk = 0; blk < nblk; ++blk)
+            for (int half = 0; half < 2; ++half)
+                tma_load_5d(sQ + blk * TILE_BYTES + half * HALF_BYTES, &qmap, half * 64, 0, (row0 + blk * 128) / G, sg.h, sg.b, bar(BAR_Q));
     };
 
     long long g_lo_cta = 0;
@@ -522,6 +540,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap kmap, const __grid_constant__
         mbar_init(bar(BAR_O), 1);
         mbar_init(bar(BAR_QFREE), 1);
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        if (a.q_tma) issue_q(s_seg[0]);
         // fill the ring at once: these copies overlap the staging of Q below
         for (int si = 0; si < s_nseg && n_prefetched < NSLOT; ++si) {
             const Seg sg = s_seg[si];
@@ -533,7 +552,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap kmap, const __grid_constant__
         asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&s_tmem)), "r"(512u) : "memory");
         asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
     }
-    stage_q(s_seg[0], threadIdx.x, NTHREADS);      // the first segment's Q, by everyone
+    if (!a.q_tma) stage_q(s_seg[0], threadIdx.x, NTHREADS);      // the first segment's Q, by everyone
     STAMP(0);
     tc_fence_before();
     __syncthreads();
@@ -635,9 +654,17 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap kmap, const __grid_constant__
                 const Seg sg = s_seg[si];
                 // Q may be overwritten once the previous segment's last Q K^T is complete (one phase per segment)
                 if (n_seg_done > 0) mbar_wait(bar(BAR_QFREE), (n_seg_done - 1) & 1, abort_flag, status);
-                if (n_seg_done > 0) stage_q(sg, threadIdx.x - 64, 64);      // the first segment's Q was staged by all warps
-                __syncwarp();
-                if (lane == 0) mbar_arrive(bar(BAR_Q));
+                if (a.q_tma) {
+                    // the very first segment's copy was issued (and one arrival made) by thread 0 at start-up
+                    if (lane == 0) {
+                        if (warp == 3) mbar_arrive(bar(BAR_Q));
+                        else if (n_seg_done > 0) issue_q(sg);
+                    }
+                } else {
+                    if (n_seg_done > 0) stage_q(sg, threadIdx.x - 64, 64);      // the first segment's Q was staged by all warps
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(bar(BAR_Q));
+                }
                 ++n_seg_done;
             }
         } else if (warp >= 4) {
@@ -661,6 +688,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap kmap, const __grid_constant__
                     const bool row_valid = r < R;
                     const int t = row_valid ? r / G : 0, g = row_valid ? r % G : 0;
                     const unsigned long long anc = row_valid ? p.tree_anc[(size_t)sg.b * p.T_max + t] : 0ull;
+                    const unsigned long long allowed = sg.T >= 64 ? anc : (anc & ((1ull << sg.T) - 1ull));
                     float m_ref = -CUDART_INF_F, l = 0.f;
 
                     for (int j = 0; j < nt; ++j) {
@@ -670,12 +698,17 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap kmap, const __grid_constant__
                         tc_fence_after();
                         if (j == 0) STAMP(3 + 8 * min(si, 1));
                         if (j == 1) STAMP(4 + 8 * min(si, 1));
-                        auto mask32 = [&](uint32_t (&x)[32], int col0) {    // ancestor mask and the end of the tree's keys
+                        // ancestor mask and the end of the tree's keys: one 32-bit word of allowed columns per chunk
+                        auto mask32 = [&](uint32_t (&x)[32], int col0) {
+                            const int u0 = key0 + col0 - sg.L;         // tree index of the chunk's first column
+                            uint32_t w;
+                            if (u0 >= 64) w = 0u;
+                            else if (u0 >= 0) w = (uint32_t)(allowed >> u0);
+                            else if (u0 <= -32) w = 0xffffffffu;
+                            else w = (uint32_t)((allowed << (-u0)) | ((1ull << (-u0)) - 1ull));
 #pragma unroll
-                            for (int q = 0; q < 32; ++q) {
-                                const int u = key0 + col0 + q - sg.L;
-                                if (!(u < 0 || (u < sg.T && ((anc >> (u & 63)) & 1ull)))) x[q] = 0xff800000u;   // -inf
-                            }
+                            for (int q = 0; q < 32; ++q)
+                                if (!((w >> q) & 1u)) x[q] = 0xff800000u;   // -inf
                         };
                         auto max32 = [&](const uint32_t (&x)[32], float& m0, float& m1) {
 #pragma unroll
@@ -847,15 +880,6 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap kmap, const __grid_constant__
             const long long t0 = clock64();
             while (!mbar_try_wait(bar(BAR_FULL + m % NSLOT), (m / NSLOT) & 1) && clock64() - t0 < kWaitCycles) {}
         }
-#ifdef GRAFT_TC_EXPERIMENTS
-    if (threadIdx.x == 128) {      // per-CTA totals for load-balance studies
-        if (2 * gridDim.x + 3 * (blockIdx.x + 1) <= kDescBytes / 4) {
-            a.desc[2 * gridDim.x + 3 * blockIdx.x] = (int)(clock64() - t_entry);
-            a.desc[2 * gridDim.x + 3 * blockIdx.x + 1] = n_seg_done;
-            a.desc[2 * gridDim.x + 3 * blockIdx.x + 2] = n_load / 2;
-        }
-    }
-#endif
     tc_fence_before();
     __syncthreads();
     if (warp == 1) {
@@ -1001,6 +1025,28 @@ int make_kv_map(CUtensorMap* map, const void* base, const graft_attn_params* p) 
     return rc == CUDA_SUCCESS ? GRAFT_OK : GRAFT_ERR_CUDA;
 }
 
+// Q [B, T_max, Hq, d] seen as (d, g, t, KV head, b): one box is 128 consecutive rows r = t*G + g of one KV head.
+int make_q_map(CUtensorMap* map, const graft_attn_params* p, int G) {
+    const cuuint64_t dims[5] = {(cuuint64_t)p->d, (cuuint64_t)G, (cuuint64_t)p->T_max, (cuuint64_t)p->Hkv, (cuuint64_t)p->B};
+    const cuuint64_t strides[4] = {(cuuint64_t)p->q_stride_h * 2, (cuuint64_t)p->q_stride_t * 2, (cuuint64_t)p->q_stride_h * 2 * G,
+                                   (cuuint64_t)p->q_stride_b * 2};
+    const cuuint32_t box[5] = {64, (cuuint32_t)G, (cuuint32_t)(128 / G), 1, 1};
+    const cuuint32_t estr[5] = {1, 1, 1, 1, 1};
+    const CUresult rc = g_encode(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 5, const_cast<void*>(p->Q), dims, strides, box, estr,
+                                 CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                                 CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    return rc == CUDA_SUCCESS ? GRAFT_OK : GRAFT_ERR_CUDA;
+}
+
+// TMA wants 16-byte aligned base and strides, strides below 2^40 bytes; the box wants G to divide 128
+bool q_map_possible(const graft_attn_params* p, int G) {
+    if (G < 1 || 128 % G != 0) return false;
+    const long long st[3] = {p->q_stride_h, p->q_stride_t, p->q_stride_b};
+    for (long long v : st)
+        if (v <= 0 || (v * 2) % 16 != 0 || v * 2 * G >= (1ll << 40)) return false;
+    return (reinterpret_cast<uintptr_t>(p->Q) & 15) == 0;
+}
+
 }  // namespace
 
 int graft_attn_tc_init() {
@@ -1034,13 +1080,18 @@ int graft_attn_tc_launch(graft_ctx* ctx, const graft_attn_params* p, cudaStream_
     CUtensorMap kmap, vmap;
     int rc = make_kv_map(&kmap, p->Kc, p);
     if (rc == GRAFT_OK) rc = make_kv_map(&vmap, p->Vc, p);
+    const int G = p->Hq / p->Hkv;
+    CUtensorMap qmap = kmap;                 // unused placeholder unless Q goes by TMA
+    const bool q_tma = q_map_possible(p, G);
+    if (rc == GRAFT_OK && q_tma) rc = make_q_map(&qmap, p, G);
     if (rc != GRAFT_OK) return rc;
     TcArgs a;
     a.p = *p;
     a.desc = reinterpret_cast<int*>(reinterpret_cast<char*>(ctx->ws) + GRAFT_WS_HEADER);
     a.cut = reinterpret_cast<CutHeader*>(reinterpret_cast<char*>(ctx->ws) + GRAFT_WS_HEADER + kDescBytes);
     a.partial = reinterpret_cast<float*>(reinterpret_cast<char*>(ctx->ws) + GRAFT_WS_HEADER + kDescBytes + cut_bytes(p->B));
-    a.G = p->Hq / p->Hkv;
+    a.G = G;
+    a.q_tma = q_tma ? 1 : 0;
     a.prof_cta = 0;
 #ifdef GRAFT_TC_EXPERIMENTS
     if (getenv("GRAFT_TC_PROF_CTA")) a.prof_cta = atoi(getenv("GRAFT_TC_PROF_CTA"));
@@ -1049,7 +1100,7 @@ int graft_attn_tc_launch(graft_ctx* ctx, const graft_attn_params* p, cudaStream_
 #ifdef GRAFT_TC_EXPERIMENTS
     if (getenv("GRAFT_TC_GRID")) grid = atoi(getenv("GRAFT_TC_GRID"));
 #endif
-    attn_tc_kernel<<<grid, NTHREADS, SMEM_DYN, stream>>>(kmap, vmap, a, ctx->status);
+    attn_tc_kernel<<<grid, NTHREADS, SMEM_DYN, stream>>>(kmap, vmap, qmap, a, ctx->status);
     GRAFT_CHECK_CUDA(cudaGetLastError());
     // few rows: one row per warp (the merge is latency-bound); many rows: four, to keep the CTA count down
     const int rows_pad = p->T_max * a.G;
