@@ -62,7 +62,8 @@ enum {
     GRAFT_FLAG_BAD_TEMPLATE = 32, /* template parent or rank out of range: node hangs off the root, token -1 */
     GRAFT_FLAG_NAN_SCORE = 64,    /* NaN score: treated as -inf                                             */
     GRAFT_FLAG_BAD_PATH = 128,    /* compaction: n_acc or a path entry out of range: sequence left untouched */
-    GRAFT_FLAG_WAIT_TIMEOUT = 256 /* a bounded wait inside a kernel gave up (output of that launch invalid) */
+    GRAFT_FLAG_WAIT_TIMEOUT = 256,/* a bounded wait inside a kernel gave up (output of that launch invalid) */
+    GRAFT_FLAG_INTERNAL = 512     /* a kernel found its own set-up inconsistent and did not run (output invalid) */
 };
 
 /* prune modes of graft_build_tree */
@@ -78,7 +79,9 @@ enum {
 enum {
     GRAFT_ATTN_AUTO = 0,
     GRAFT_ATTN_MMA_SYNC = 1,   /* register-tile kernel (any supported shape; the low-row path)    */
-    GRAFT_ATTN_TCGEN05 = 2     /* TMA + tcgen05/TMEM kernel (d = 128, contiguous cache rows)        */
+    GRAFT_ATTN_TCGEN05 = 2,    /* TMA + tcgen05/TMEM kernels (d = 128): one of the two below        */
+    GRAFT_ATTN_TCGEN05_1SM = 3,/* ... one CTA per SM holds both 128-row blocks of an item           */
+    GRAFT_ATTN_TCGEN05_2SM = 4 /* ... a pair of SMs shares every tile                              */
 };
 
 /* ---- context --------------------------------------------------------------------------------- */

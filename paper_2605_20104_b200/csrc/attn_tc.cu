@@ -217,6 +217,117 @@ struct Seg {
 };
 
 // ---------------------------------------------------------------------------------------------------
+// per-worker plan: a worker (a CTA, or a pair of CTAs) owns a range of the cut axis and walks it in rounds
+// ---------------------------------------------------------------------------------------------------
+struct Plan {
+    Seg seg[MAXSEG];
+    long long gnext, ghi;    // stream-K: next unit to plan, end of the worker's range
+    int nseg, npartial;
+};
+
+// Fills pl.seg with the next <= MAXSEG segments of the unit range [g, g_hi) (warp-cooperative).  A tile
+// belongs to the range that holds its first unit.  Partial results go to slots 2*worker and 2*worker + 1.
+__device__ __forceinline__ void plan_round(const TcArgs& a, int G, int worker, bool write_desc, Plan& pl, long long g, long long g_hi) {
+    const graft_attn_params& p = a.p;
+    const int lane = threadIdx.x & 31;
+    int n = 0;
+    int n_partial = pl.npartial;
+    while (g < g_hi && n < MAXSEG) {
+        long long total, tiles;
+        const SeqInfo si = scan_sequences(p, G, g, -1, total, tiles, 0);
+        if (!si.found) { g = g_hi; break; }
+        const long long hu = head_units(si.ntiles, si.nrb, si.wlast);
+        const long long seq_end = si.base + (long long)p.Hkv * hu;
+        // walk the items of this sequence from the one that holds unit g
+        int h = (int)((g - si.base) / hu);
+        const long long rem = (g - si.base) % hu;
+        int rb = (int)(rem / ((long long)si.ntiles * kW2));
+        if (rb > si.nrb - 1) rb = si.nrb - 1;
+        while (g < g_hi && g < seq_end && n < MAXSEG) {
+            long long U;
+            int w;
+            item_span(si, h, rb, U, w);
+            const long long item_end = U + (long long)si.ntiles * w;
+            long long t_lo = (g - U + w - 1) / w, t_hi = (g_hi - U + w - 1) / w;
+            if (t_lo < 0) t_lo = 0;
+            if (t_hi > si.ntiles) t_hi = si.ntiles;
+            if (t_lo < t_hi) {
+                const bool whole = t_lo == 0 && t_hi == si.ntiles;
+                if (lane == 0) {
+                    Seg sg;
+                    sg.b = si.b;
+                    sg.h = h;
+                    sg.rb = rb;
+                    sg.tile_lo = (int)t_lo;
+                    sg.tile_hi = (int)t_hi;
+                    sg.L = si.L;
+                    sg.T = si.T;
+                    sg.slot = whole ? -1 : 2 * worker + (n_partial < 1 ? n_partial : 1);
+                    pl.seg[n] = sg;
+                    if (!whole && write_desc) a.desc[sg.slot] = item_id(p, si.b, h, rb);
+                }
+                if (!whole) ++n_partial;
+                ++n;
+            }
+            g = item_end < g_hi ? item_end : g_hi;
+            if (++rb == si.nrb) { rb = 0; ++h; }
+        }
+    }
+    if (lane == 0) { pl.nseg = n; pl.gnext = g; pl.npartial = n_partial; }
+}
+
+// The worker's share of the batch and its first round (warp-cooperative).  `record`: this worker writes
+// the cut for the merge kernel.
+__device__ __forceinline__ void plan_first(const TcArgs& a, int G, int worker, int nworkers, bool record, bool write_desc, Plan& pl) {
+    const graft_attn_params& p = a.p;
+    const int lane = threadIdx.x & 31;
+    long long total, per;
+    bool pieces;
+    choose_cut(p, G, nworkers, total, per, pieces, record ? a.cut : nullptr);
+    if (lane == 0) {
+        pl.npartial = 0;
+        if (write_desc) {
+            a.desc[2 * worker] = -1;           // this call's slot descriptors
+            a.desc[2 * worker + 1] = -1;
+        }
+    }
+    __syncwarp();
+    if (pieces) {
+        // exactly one piece of one item for this worker
+        long long units, tiles;
+        const SeqInfo si = scan_sequences(p, G, worker, -1, units, tiles, per);
+        if (lane == 0) {
+            pl.nseg = 0;
+            pl.gnext = pl.ghi = 0;
+            if (si.found) {
+                int nsplit, plen;
+                piece_shape(si.ntiles, per, nsplit, plen);
+                const int local = (int)(worker - si.base);
+                const int k = local / nsplit, sp = local % nsplit;
+                Seg sg;
+                sg.b = si.b;
+                sg.h = k / si.nrb;
+                sg.rb = k % si.nrb;
+                sg.tile_lo = sp * plen;
+                sg.tile_hi = min(si.ntiles, sg.tile_lo + plen);
+                sg.L = si.L;
+                sg.T = si.T;
+                sg.slot = nsplit == 1 ? -1 : 2 * worker;
+                pl.seg[0] = sg;
+                pl.nseg = 1;
+            }
+        }
+    } else {
+        long long g_lo = per * worker;
+        long long g_hi = g_lo + per;
+        if (g_hi > total) g_hi = total;
+        if (g_lo > total) g_lo = total;
+        if (lane == 0) pl.ghi = g_hi;
+        plan_round(a, G, worker, write_desc, pl, g_lo, g_hi);
+    }
+}
+
+// ---------------------------------------------------------------------------------------------------
 // PTX helpers
 // ---------------------------------------------------------------------------------------------------
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
@@ -357,10 +468,9 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap kmap, const __grid_constant__
     __shared__ __align__(8) uint64_t s_bar[BAR_COUNT];
     __shared__ uint32_t s_tmem;
     __shared__ int s_abort;
-    __shared__ Seg s_seg[MAXSEG];
-    __shared__ int s_nseg;
-    __shared__ long long s_gnext, s_ghi;
-    __shared__ int s_npartial;
+    __shared__ Plan s_plan;
+    Seg* const s_seg = s_plan.seg;
+    int& s_nseg = s_plan.nseg;
 
     const graft_attn_params& p = a.p;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -378,57 +488,6 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap kmap, const __grid_constant__
     const uint32_t bar0 = smem_u32(s_bar);
     auto bar = [&](int i) { return bar0 + 8u * (uint32_t)i; };
     volatile int* abort_flag = &s_abort;
-
-    // ---- this CTA's range, and the first round of segments
-    // plan_round (warp 0): fills s_seg with the next <= MAXSEG segments of the unit range [g, g_hi); g_lo is the
-    // start of the CTA's range (a tile belongs to the range that holds its first unit)
-    auto plan_round = [&](long long g, long long g_lo, long long g_hi) {
-        int n = 0;
-        int n_partial = s_npartial;
-        while (g < g_hi && n < MAXSEG) {
-            long long total, tiles;
-            const SeqInfo si = scan_sequences(p, G, g, -1, total, tiles, 0);
-            if (!si.found) { g = g_hi; break; }
-            const long long hu = head_units(si.ntiles, si.nrb, si.wlast);
-            const long long seq_end = si.base + (long long)p.Hkv * hu;
-            // walk the items of this sequence from the one that holds unit g
-            int h = (int)((g - si.base) / hu);
-            const long long rem = (g - si.base) % hu;
-            int rb = (int)(rem / ((long long)si.ntiles * kW2));
-            if (rb > si.nrb - 1) rb = si.nrb - 1;
-            while (g < g_hi && g < seq_end && n < MAXSEG) {
-                long long U;
-                int w;
-                item_span(si, h, rb, U, w);
-                const long long item_end = U + (long long)si.ntiles * w;
-                long long t_lo = (g - U + w - 1) / w, t_hi = (g_hi - U + w - 1) / w;
-                if (t_lo < 0) t_lo = 0;
-                if (t_hi > si.ntiles) t_hi = si.ntiles;
-                if (t_lo < t_hi) {
-                    const bool whole = t_lo == 0 && t_hi == si.ntiles;
-                    if (lane == 0) {
-                        Seg sg;
-                        sg.b = si.b;
-                        sg.h = h;
-                        sg.rb = rb;
-                        sg.tile_lo = (int)t_lo;
-                        sg.tile_hi = (int)t_hi;
-                        sg.L = si.L;
-                        sg.T = si.T;
-                        sg.slot = whole ? -1 : 2 * (int)blockIdx.x + (n_partial < 1 ? n_partial : 1);
-                        s_seg[n] = sg;
-                        if (!whole) a.desc[sg.slot] = item_id(p, si.b, h, rb);
-                    }
-                    if (!whole) ++n_partial;
-                    ++n;
-                }
-                g = item_end < g_hi ? item_end : g_hi;
-                if (++rb == si.nrb) { rb = 0; ++h; }
-            }
-        }
-        (void)g_lo;
-        if (lane == 0) { s_nseg = n; s_gnext = g; s_npartial = n_partial; }
-    };
 
     // Q rows of an item into shared memory, K-major with the 128-byte swizzle (16-byte chunk c of row r at
     // c ^ (r & 7)), by `nthr` threads numbered tid = 0 .. nthr-1; 16 independent global loads per thread and round
@@ -474,52 +533,8 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap kmap, const __grid_constant__
                 tma_load_5d(sQ + blk * TILE_BYTES + half * HALF_BYTES, &qmap, half * 64, 0, (row0 + blk * 128) / G, sg.h, sg.b, bar(BAR_Q));
     };
 
-    long long g_lo_cta = 0;
-    if (warp == 0) {
-        long long total, per;
-        bool pieces;
-        choose_cut(p, G, (int)gridDim.x, total, per, pieces, blockIdx.x == 0 ? a.cut : nullptr);
-        if (lane == 0) {
-            s_abort = 0;
-            s_npartial = 0;
-            a.desc[2 * blockIdx.x] = -1;           // this call's slot descriptors
-            a.desc[2 * blockIdx.x + 1] = -1;
-        }
-        __syncwarp();
-        if (pieces) {
-            // exactly one piece of one item for this CTA
-            long long units, tiles;
-            const SeqInfo si = scan_sequences(p, G, blockIdx.x, -1, units, tiles, per);
-            if (lane == 0) {
-                s_nseg = 0;
-                s_gnext = s_ghi = 0;
-                if (si.found) {
-                    int nsplit, plen;
-                    piece_shape(si.ntiles, per, nsplit, plen);
-                    const int local = (int)(blockIdx.x - si.base);
-                    const int k = local / nsplit, sp = local % nsplit;
-                    Seg sg;
-                    sg.b = si.b;
-                    sg.h = k / si.nrb;
-                    sg.rb = k % si.nrb;
-                    sg.tile_lo = sp * plen;
-                    sg.tile_hi = min(si.ntiles, sg.tile_lo + plen);
-                    sg.L = si.L;
-                    sg.T = si.T;
-                    sg.slot = nsplit == 1 ? -1 : 2 * (int)blockIdx.x;
-                    s_seg[0] = sg;
-                    s_nseg = 1;
-                }
-            }
-        } else {
-            g_lo_cta = per * blockIdx.x;
-            long long g_hi = g_lo_cta + per;
-            if (g_hi > total) g_hi = total;
-            if (g_lo_cta > total) g_lo_cta = total;
-            if (lane == 0) s_ghi = g_hi;
-            plan_round(g_lo_cta, g_lo_cta, g_hi);
-        }
-    }
+    if (warp == 0) plan_first(a, G, (int)blockIdx.x, (int)gridDim.x, blockIdx.x == 0, true, s_plan);
+    if (threadIdx.x == 0) s_abort = 0;
     __syncthreads();
     if (s_nseg == 0) return;                      // nothing for this CTA (short batch)
 
@@ -865,10 +880,10 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap kmap, const __grid_constant__
 
         // ---- next round (only batches with very many short sequences need more than one)
         __syncthreads();
-        const long long g_next = s_gnext, g_hi = s_ghi;
+        const long long g_next = s_plan.gnext, g_hi = s_plan.ghi;
         if (g_next >= g_hi) break;
         __syncthreads();
-        if (warp == 0) plan_round(g_next, g_lo_cta, g_hi);
+        if (warp == 0) plan_round(a, G, (int)blockIdx.x, true, s_plan, g_next, g_hi);
         __syncthreads();
         if (s_nseg == 0) break;
     }
@@ -885,6 +900,482 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap kmap, const __grid_constant__
     if (warp == 1) {
         tc_fence_after();
         asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(512u) : "memory");
+    }
+}
+
+// ---------------------------------------------------------------------------------------------------
+// the pair kernel: two CTAs (a cluster of two SMs) share every tile
+// ---------------------------------------------------------------------------------------------------
+// One tcgen05.mma.cta_group::2 multiplies 256 rows at once: CTA 0 of the pair owns rows 0..127 of the item,
+// CTA 1 rows 128..255, each in its own tensor memory.  The B operand is split between the two shared
+// memories: of a K tile each CTA fetches 64 of the 128 keys (all of d), of a V tile all 128 keys and 64 of
+// the d columns, so every byte of the cache still crosses into the pair once.  With one row block per SM
+// the score tile is double-buffered in tensor memory (columns 0..127 and 128..255, O at 256..383): the
+// tensor pipe computes S of tile j+1 while the softmax warps work on tile j.
+//
+// Barriers live at the same offset in both shared memories.  Copies of both CTAs complete on the leader's
+// (CTA 0's) FULL and Q barriers; the softmax warps of both arrive on the leader's P barriers; everything
+// the MMA thread commits is multicast to both CTAs (slot free, S ready, PV done, O final, Q free).
+//
+// The last tile of an item is fetched at keys [L+T-128, L+T) instead of a tile-aligned position: it never
+// reaches past the sequence's keys (rows before key 0 are zero-filled by the copy), and the columns that
+// the previous tile already covered are masked like non-ancestors.
+constexpr int P_NTHREADS = 256;
+constexpr int P_SLOT_BYTES = TILE_BYTES / 2;      // half a K tile or half a V tile
+constexpr int P_NSLOT = 12;
+constexpr int kCtrlBytes = 1024;
+constexpr int P_SMEM_DYN = kCtrlBytes + TILE_BYTES + P_NSLOT * P_SLOT_BYTES;      // control, Q (128 rows), ring
+enum { PB_FULL = 0, PB_EMPTY = P_NSLOT, PB_S = 2 * P_NSLOT, PB_P = 2 * P_NSLOT + 2, PB_Q = 2 * P_NSLOT + 4, PB_O = 2 * P_NSLOT + 5,
+       PB_QFREE = 2 * P_NSLOT + 6, PB_PVD = 2 * P_NSLOT + 7, PB_COUNT = 2 * P_NSLOT + 8 };
+struct PairCtrl {
+    uint64_t bar[PB_COUNT];
+    Plan plan;
+    uint32_t tmem;
+    int abort;
+};
+static_assert(sizeof(PairCtrl) <= kCtrlBytes, "control block too large");
+
+__device__ __forceinline__ uint32_t cluster_ctarank() {
+    uint32_t r;
+    asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
+    return r;
+}
+__device__ __forceinline__ void cluster_sync_all() {
+    asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
+    asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+// address of this CTA's shared-memory location `addr` as seen in CTA `cta` of the cluster
+__device__ __forceinline__ uint32_t map_to_cta(uint32_t addr, uint32_t cta) {
+    uint32_t r;
+    asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(addr), "r"(cta));
+    return r;
+}
+// arrival on a barrier of the pair's leader.  The plain form orders tensor-memory traffic (together with the
+// tcgen05 fences on both sides); the cluster-scope release also publishes ordinary shared-memory writes, at
+// the price of a full memory fence (over a thousand cycles when measured), so only the Q stagers use it.
+__device__ __forceinline__ void mbar_arrive_remote(uint32_t cluster_addr) {
+    asm volatile("mbarrier.arrive.shared::cluster.b64 _, [%0];" ::"r"(cluster_addr) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive_cluster(uint32_t cluster_addr) {
+    asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(cluster_addr) : "memory");
+}
+// bounded wait on a barrier that threads of the partner CTA arrive on
+__device__ __forceinline__ bool mbar_try_wait_cluster(uint32_t bar, uint32_t parity) {
+    uint32_t ok;
+    asm volatile("{\n\t.reg .pred p;\n\tmbarrier.try_wait.parity.acquire.cluster.shared::cta.b64 p, [%1], %2;\n\tselp.u32 %0, 1, 0, p;\n\t}"
+                 : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+    return ok != 0;
+}
+__device__ __forceinline__ void mbar_wait_cluster(uint32_t bar, uint32_t parity, volatile int* abort_flag, unsigned* status) {
+    if (mbar_try_wait_cluster(bar, parity)) return;
+    if (*abort_flag) return;
+    const long long t0 = clock64();
+    while (!mbar_try_wait_cluster(bar, parity)) {
+        if (*abort_flag) return;
+        if (clock64() - t0 > kWaitCycles) {
+            *abort_flag = 1;
+            atomicOr(status, (unsigned)GRAFT_FLAG_WAIT_TIMEOUT);
+            return;
+        }
+    }
+}
+// copies whose completion is counted on a barrier of the pair's leader
+__device__ __forceinline__ void tma_pair_4d(uint32_t dst, const CUtensorMap* map, int x, int y, int z, int w, uint32_t cluster_bar) {
+    asm volatile("cp.async.bulk.tensor.4d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4, %5}], [%6];"
+                 ::"r"(dst), "l"(map), "r"(x), "r"(y), "r"(z), "r"(w), "r"(cluster_bar) : "memory");
+}
+__device__ __forceinline__ void tma_pair_5d(uint32_t dst, const CUtensorMap* map, int x, int y, int z, int w, int v, uint32_t cluster_bar) {
+    asm volatile("cp.async.bulk.tensor.5d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4, %5, %6}], [%7];"
+                 ::"r"(dst), "l"(map), "r"(x), "r"(y), "r"(z), "r"(w), "r"(v), "r"(cluster_bar) : "memory");
+}
+// D[tmem of both CTAs] (+)= A * B over the pair; issued by one thread of the leader
+__device__ __forceinline__ void mma_pair_ss(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc, uint32_t accumulate) {
+    asm volatile("{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
+                 "tcgen05.mma.cta_group::2.kind::f16 [%0], %1, %2, %3, {%5, %5, %5, %5, %5, %5, %5, %5}, p;\n\t}"
+                 ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate), "r"(0u) : "memory");
+}
+__device__ __forceinline__ void mma_pair_ts(uint32_t d_tmem, uint32_t a_tmem, uint64_t b_desc, uint32_t idesc, uint32_t accumulate) {
+    asm volatile("{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
+                 "tcgen05.mma.cta_group::2.kind::f16 [%0], [%1], %2, %3, {%5, %5, %5, %5, %5, %5, %5, %5}, p;\n\t}"
+                 ::"r"(d_tmem), "r"(a_tmem), "l"(b_desc), "r"(idesc), "r"(accumulate), "r"(0u) : "memory");
+}
+// arrive on the barrier at this offset in both CTAs once every MMA issued so far is complete
+__device__ __forceinline__ void tc_commit_pair(uint32_t bar) {
+    asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], %1;"
+                 ::"r"(bar), "h"((unsigned short)3) : "memory");
+}
+// M = 256 over the pair, N = 128
+constexpr uint32_t kIdescPairBase = (1u << 4) | (1u << 7) | (1u << 10) | ((128u >> 3) << 17) | ((256u >> 4) << 24);
+constexpr uint32_t kIdescPairQK = kIdescPairBase;
+constexpr uint32_t kIdescPairPV = kIdescPairBase | (1u << 16);
+
+__global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(P_NTHREADS, 1)
+attn_tc_pair_kernel(const __grid_constant__ CUtensorMap kmap, const __grid_constant__ CUtensorMap vmap, const __grid_constant__ CUtensorMap qmap,
+                    TcArgs a, unsigned* status) {
+    extern __shared__ __align__(1024) unsigned char smem_raw[];
+    PairCtrl& ctrl = *reinterpret_cast<PairCtrl*>(smem_raw);
+    Plan& plan = ctrl.plan;
+    const graft_attn_params& p = a.p;
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int G = a.G;
+    const uint32_t rank = cluster_ctarank();          // 0: leader (issues the MMAs), 1: peer
+#ifdef GRAFT_TC_EXPERIMENTS
+    const long long t_entry = clock64();
+    const bool prof = (int)blockIdx.x == a.prof_cta;
+#define PSTAMP(cond, idx) do { if (prof && (cond)) a.desc[(idx)] = (int)(clock64() - t_entry); } while (0)
+#else
+#define PSTAMP(cond, idx) do { } while (0)
+#endif
+    const int worker = (int)(blockIdx.x >> 1), nworkers = (int)(gridDim.x >> 1);
+
+    if ((smem_u32(smem_raw) & 1023u) != 0) {          // the tiles would miss their alignment: refuse to run (both CTAs alike)
+        if (threadIdx.x == 0) atomicOr(status, (unsigned)GRAFT_FLAG_INTERNAL);
+        return;
+    }
+    const uint32_t sQ = smem_u32(smem_raw) + kCtrlBytes;
+    const uint32_t sRing = sQ + TILE_BYTES;
+    const uint32_t bar0 = smem_u32(ctrl.bar);
+    auto bar = [&](int i) { return bar0 + 8u * (uint32_t)i; };
+    auto leader_bar = [&](int i) { return map_to_cta(bar(i), 0u); };
+    volatile int* abort_flag = &ctrl.abort;
+
+    // both CTAs of a pair derive the same plan
+    if (warp == 0) plan_first(a, G, worker, nworkers, blockIdx.x == 0, rank == 0, plan);
+    if (threadIdx.x == 0) ctrl.abort = 0;
+    __syncthreads();
+    if (plan.nseg == 0) return;                       // nothing for this pair (short batch); no cluster operation was started
+
+    if (threadIdx.x == 0) {
+        for (int i = 0; i < P_NSLOT; ++i) { mbar_init(bar(PB_FULL + i), 1); mbar_init(bar(PB_EMPTY + i), 1); }
+        for (int i = 0; i < 2; ++i) { mbar_init(bar(PB_S + i), 1); mbar_init(bar(PB_P + i), 8); }      // 4 softmax warps in each CTA
+        mbar_init(bar(PB_Q), a.q_tma ? 2 : 4);      // by TMA: one arrival per CTA; staged by threads: one per stager warp
+        mbar_init(bar(PB_O), 1);
+        mbar_init(bar(PB_QFREE), 1);
+        mbar_init(bar(PB_PVD), 1);
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    if (warp == 1) {
+        asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&ctrl.tmem)), "r"(512u) : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
+    }
+    tc_fence_before();
+    __syncthreads();
+    cluster_sync_all();                               // the partner's barriers exist before anything signals them
+    tc_fence_after();
+    const uint32_t tmem = ctrl.tmem;
+
+    // first key and number of already-covered columns of tile t of an item
+    auto tile_key0 = [&](const Seg& sg, int t, int& overlap) {
+        const int n_keys = sg.L + sg.T;
+        const int ntiles = (n_keys + BN - 1) / BN;
+        overlap = 0;
+        if (t < ntiles - 1) return t * BN;
+        overlap = ntiles * BN - n_keys;
+        return n_keys - BN;
+    };
+
+    // running counters that persist across segments and rounds (each role keeps its own copy)
+    int n_load = 0;            // ring loads issued / consumed so far (2 per tile)
+    int jt = 0;                // tiles processed so far (S, P and PV-done barrier phases)
+    int n_seg_done = 0;        // segments finished (Q, Q-free and O barrier phases)
+
+    for (;;) {                 // rounds of <= MAXSEG segments
+        const int nseg = plan.nseg;
+
+        if (warp == 0) {
+            // =============================== K/V producer (both CTAs) ===============================
+            if (lane == 0) {
+                for (int si = 0; si < nseg; ++si) {
+                    const Seg sg = plan.seg[si];
+                    for (int t = sg.tile_lo; t < sg.tile_hi; ++t) {
+                        int overlap;
+                        const int key0 = tile_key0(sg, t, overlap);
+                        for (int which = 0; which < 2; ++which, ++n_load) {
+                            const int slot = n_load % P_NSLOT, use = n_load / P_NSLOT;
+                            if (use > 0) mbar_wait(bar(PB_EMPTY + slot), (use - 1) & 1, abort_flag, status);
+                            if (rank == 0) mbar_expect_tx(bar(PB_FULL + slot), 2 * P_SLOT_BYTES);      // both halves
+                            const uint32_t dst = sRing + slot * P_SLOT_BYTES;
+                            const uint32_t fb = leader_bar(PB_FULL + slot);
+                            if (which == 0) {      // 64 keys of the K tile, all of d (two 64-column boxes)
+                                tma_pair_4d(dst, &kmap, 0, key0 + 64 * (int)rank, sg.h, sg.b, fb);
+                                tma_pair_4d(dst + P_SLOT_BYTES / 2, &kmap, 64, key0 + 64 * (int)rank, sg.h, sg.b, fb);
+                            } else {               // all keys of the V tile, 64 columns of d
+                                tma_pair_4d(dst, &vmap, 64 * (int)rank, key0, sg.h, sg.b, fb);
+                            }
+                        }
+                    }
+                }
+            }
+        } else if (warp == 1) {
+            // =============================== MMA issuer (leader only) ===============================
+            if (lane == 0 && rank == 0) {
+                auto wait_full = [&](int n) { mbar_wait(bar(PB_FULL + n % P_NSLOT), (n / P_NSLOT) & 1, abort_flag, status); };
+                for (int si = 0; si < nseg; ++si) {
+                    const Seg sg = plan.seg[si];
+                    const int nt = sg.tile_hi - sg.tile_lo;
+                    // S[buffer gt & 1] = Q K^T with the K tile of ring load n
+                    auto issue_qk = [&](int gt, int n) {
+                        wait_full(n);
+                        PSTAMP(gt >= 40 && gt < 48, 343 + (gt - 40) * 4);
+                        tc_fence_after();
+                        const uint32_t sK16 = (sRing + (n % P_NSLOT) * P_SLOT_BYTES) >> 4;
+                        const uint32_t sQ16 = sQ >> 4;
+#pragma unroll
+                        for (int k = 0; k < D / 16; ++k) {
+                            const uint32_t offQ = ((k >> 2) * HALF_BYTES + (k & 3) * 32) >> 4;
+                            const uint32_t offK = ((k >> 2) * (P_SLOT_BYTES / 2) + (k & 3) * 32) >> 4;
+                            mma_pair_ss(tmem + (gt & 1) * 128, smem_desc(kDescKMajor, sQ16 + offQ), smem_desc(kDescKMajor, sK16 + offK), kIdescPairQK, k > 0);
+                        }
+                        tc_commit_pair(bar(PB_S + (gt & 1)));
+                        tc_commit_pair(bar(PB_EMPTY + n % P_NSLOT));          // K tile fully read
+                    };
+                    mbar_wait_cluster(bar(PB_Q), n_seg_done & 1, abort_flag, status);   // Q of this segment is in place in both CTAs
+                    issue_qk(jt, n_load);
+                    if (nt == 1) tc_commit_pair(bar(PB_QFREE));      // the segment's last Q K^T is in the pipe
+                    for (int j = 0; j < nt; ++j) {
+                        const int gt = jt + j;
+                        if (j + 1 < nt) {
+                            issue_qk(gt + 1, n_load + 2 * (j + 1));             // runs while the softmax warps work on tile j
+                            if (j + 2 == nt) tc_commit_pair(bar(PB_QFREE));
+                        }
+                        const int nV = n_load + 2 * j + 1;
+                        PSTAMP(gt >= 40 && gt < 48, 340 + (gt - 40) * 4);
+                        mbar_wait_cluster(bar(PB_P + (gt & 1)), (gt >> 1) & 1, abort_flag, status);
+                        PSTAMP(gt >= 40 && gt < 48, 341 + (gt - 40) * 4);
+                        wait_full(nV);
+                        tc_fence_after();
+                        const uint32_t sV16 = (sRing + (nV % P_NSLOT) * P_SLOT_BYTES) >> 4;
+#pragma unroll
+                        for (int k = 0; k < BN / 16; ++k)
+                            mma_pair_ts(tmem + 256, tmem + (gt & 1) * 128 + k * 8, smem_desc(kDescVMajor, sV16 + k * (2048 >> 4)), kIdescPairPV,
+                                        (j > 0 || k > 0) ? 1u : 0u);
+                        tc_commit_pair(bar(PB_EMPTY + nV % P_NSLOT));         // V tile fully read
+                        tc_commit_pair(bar(PB_PVD));                          // O holds tiles 0..j
+                        PSTAMP(gt >= 40 && gt < 48, 342 + (gt - 40) * 4);
+                    }
+                    tc_commit_pair(bar(PB_O));
+                    n_load += 2 * nt;
+                    jt += nt;
+                    ++n_seg_done;
+                }
+            }
+        } else if (warp == 2 || warp == 3) {
+            // =============================== Q loaders (both CTAs) ===============================
+            for (int si = 0; si < nseg; ++si) {
+                const Seg sg = plan.seg[si];
+                // Q may be overwritten once the previous segment's last Q K^T is complete
+                if (n_seg_done > 0) mbar_wait(bar(PB_QFREE), (n_seg_done - 1) & 1, abort_flag, status);
+                const uint32_t qb = leader_bar(PB_Q);
+                const int row0 = sg.rb * BR + (int)rank * 128;
+                if (a.q_tma) {
+                    if (warp == 2 && lane == 0) {
+                        if (rank == 0) mbar_expect_tx(bar(PB_Q), 2 * TILE_BYTES);           // 128 rows in each CTA
+                        else mbar_arrive_remote(qb);
+                        tma_pair_5d(sQ, &qmap, 0, 0, row0 / G, sg.h, sg.b, qb);
+                        tma_pair_5d(sQ + HALF_BYTES, &qmap, 64, 0, row0 / G, sg.h, sg.b, qb);
+                    }
+                } else {
+                    // 16-byte asynchronous copies by the 64 threads, K-major with the 128-byte swizzle; rows past the tree read as zero
+                    const int tid = threadIdx.x - 64;
+                    const int R = sg.T * G;
+                    const __nv_bfloat16* Qg = reinterpret_cast<const __nv_bfloat16*>(p.Q) + (size_t)sg.b * p.q_stride_b +
+                                              (size_t)sg.h * G * p.q_stride_h;
+                    const int ch = tid & 15;
+                    int r = row0 + (tid >> 4);
+                    int g = r % G;
+                    const int dt = 4 / G, dg = 4 - dt * G;                 // four rows per pass
+                    const __nv_bfloat16* src_t = Qg + (size_t)(r / G) * p.q_stride_t + ch * 8;
+                    const size_t inc_t = (size_t)dt * p.q_stride_t;
+                    for (int qr = tid >> 4; qr < 128; qr += 4) {
+                        const bool valid = r < R;
+                        const __nv_bfloat16* src = valid ? src_t + (size_t)g * p.q_stride_h : Qg;
+                        const uint32_t dst = sQ + (ch >> 3) * HALF_BYTES + qr * 128 + (((ch & 7) ^ (qr & 7)) << 4);
+                        asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"(dst), "l"(src), "r"(valid ? 16 : 0) : "memory");
+                        r += 4;
+                        g += dg;
+                        src_t += inc_t;
+                        if (g >= G) { g -= G; src_t += p.q_stride_t; }
+                    }
+                    asm volatile("cp.async.wait_all;" ::: "memory");
+                    fence_async_smem();
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive_cluster(qb);
+                }
+                ++n_seg_done;
+            }
+        } else if (warp >= 4) {
+            // =============================== softmax, results (both CTAs) ===============================
+            const int rl = ((warp & 3) << 5) + lane;            // row inside this CTA's block = TMEM lane
+            const uint32_t lane_bits = (uint32_t)((warp & 3) << 5) << 16;
+            const uint32_t tO = tmem + lane_bits + 256;
+            const float sl2 = p.scale * kLog2e;
+            for (int si = 0; si < nseg; ++si) {
+                const Seg sg = plan.seg[si];
+                const int nt = sg.tile_hi - sg.tile_lo;
+                const int R = sg.T * G;
+                const int r = sg.rb * BR + (int)rank * 128 + rl;
+                const bool row_valid = r < R;
+                const int t = row_valid ? r / G : 0, g = row_valid ? r % G : 0;
+                const unsigned long long anc = row_valid ? p.tree_anc[(size_t)sg.b * p.T_max + t] : 0ull;
+                const unsigned long long allowed = sg.T >= 64 ? anc : (anc & ((1ull << sg.T) - 1ull));
+                float m_ref = -CUDART_INF_F, l = 0.f;
+
+                for (int j = 0; j < nt; ++j) {
+                    const int gt = jt + j;
+                    const uint32_t tS = tmem + lane_bits + (gt & 1) * 128;
+                    int overlap;
+                    const int key0 = tile_key0(sg, sg.tile_lo + j, overlap);
+                    const bool masked = key0 + BN > sg.L || overlap > 0;
+                    mbar_wait(bar(PB_S + (gt & 1)), (gt >> 1) & 1, abort_flag, status);
+                    tc_fence_after();
+                    PSTAMP(threadIdx.x == 128 && gt >= 40 && gt < 48, 300 + (gt - 40) * 4);
+                    uint32_t x[4][32];
+#pragma unroll
+                    for (int c = 0; c < 4; ++c) tmem_ld32(tS + c * 32, x[c]);
+                    tmem_wait_ld();
+                    if (masked) {
+                        // per 32-column chunk one word of allowed columns: cached keys not yet covered, ancestors in the tree
+#pragma unroll
+                        for (int c = 0; c < 4; ++c) {
+                            const int u0 = key0 + c * 32 - sg.L;         // tree index of the chunk's first column
+                            uint32_t w;
+                            if (u0 >= 64) w = 0u;
+                            else if (u0 >= 0) w = (uint32_t)(allowed >> u0);
+                            else if (u0 <= -32) w = 0xffffffffu;
+                            else w = (uint32_t)((allowed << (-u0)) | ((1ull << (-u0)) - 1ull));
+                            const int cov = overlap - c * 32;            // columns of this chunk that the previous tile covered
+                            if (cov >= 32) w = 0u;
+                            else if (cov > 0) w &= ~((1u << cov) - 1u);
+#pragma unroll
+                            for (int q = 0; q < 32; ++q)
+                                if (!((w >> q) & 1u)) x[c][q] = 0xff800000u;   // -inf
+                        }
+                    }
+                    float mx0 = -CUDART_INF_F, mx1 = -CUDART_INF_F;
+#pragma unroll
+                    for (int c = 0; c < 4; ++c)
+#pragma unroll
+                        for (int q = 0; q < 32; q += 4) {
+                            mx0 = fmax3(mx0, __uint_as_float(x[c][q]), __uint_as_float(x[c][q + 1]));
+                            mx1 = fmax3(mx1, __uint_as_float(x[c][q + 2]), __uint_as_float(x[c][q + 3]));
+                        }
+                    const float mx = fmaxf(mx0, mx1);
+                    PSTAMP(threadIdx.x == 128 && gt >= 40 && gt < 48, 301 + (gt - 40) * 4);
+                    // reference maximum: move it only when the scores outgrow it by more than the threshold
+                    if (mx != -CUDART_INF_F && (m_ref == -CUDART_INF_F || (mx - m_ref) * sl2 > kRescaleThreshold)) {
+                        if (m_ref != -CUDART_INF_F) {
+                            // O must hold every earlier tile of the segment before it is rescaled (j > 0 here)
+                            mbar_wait(bar(PB_PVD), (gt - 1) & 1, abort_flag, status);
+                            tc_fence_after();
+                            const float alpha = exp2f((m_ref - mx) * sl2);
+                            l *= alpha;
+#pragma unroll 1
+                            for (int c = 0; c < 4; ++c) {
+                                uint32_t o[32];
+                                tmem_ld32(tO + c * 32, o);
+                                tmem_wait_ld();
+#pragma unroll
+                                for (int q = 0; q < 32; ++q) o[q] = __float_as_uint(__uint_as_float(o[q]) * alpha);
+                                tmem_st32(tO + c * 32, o);
+                            }
+                            tmem_wait_st();
+                        }
+                        m_ref = mx;
+                    }
+                    const float off = m_ref == -CUDART_INF_F ? 0.f : m_ref * sl2;
+                    // P = 2^(s*scale*log2e - off) as bf16 into the first 64 columns of this S buffer
+                    float sum0 = 0.f, sum1 = 0.f;
+#pragma unroll
+                    for (int c = 0; c < 4; ++c) {
+                        uint32_t pk[16];
+#pragma unroll
+                        for (int q = 0; q < 32; q += 2) {
+                            const float p0 = ex2(fmaf(__uint_as_float(x[c][q]), sl2, -off));
+                            const float p1 = ex2(fmaf(__uint_as_float(x[c][q + 1]), sl2, -off));
+                            sum0 += p0;
+                            sum1 += p1;
+                            pk[q >> 1] = pack_bf16(p0, p1);
+                        }
+                        tmem_st16(tS + c * 16, pk);
+                    }
+                    l += sum0 + sum1;
+                    PSTAMP(threadIdx.x == 128 && gt >= 40 && gt < 48, 380 + (gt - 40) * 2);
+                    tmem_wait_st();
+                    PSTAMP(threadIdx.x == 128 && gt >= 40 && gt < 48, 381 + (gt - 40) * 2);
+                    tc_fence_before();
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive_remote(leader_bar(PB_P + (gt & 1)));       // one arrival per warp
+                    PSTAMP(threadIdx.x == 128 && gt >= 40 && gt < 48, 302 + (gt - 40) * 4);
+                }
+
+                // ---- results of the segment: O row from TMEM, final rows or a partial
+                mbar_wait(bar(PB_O), n_seg_done & 1, abort_flag, status);     // every MMA of the segment is complete
+                tc_fence_after();
+                if (sg.slot < 0) {
+                    const float inv = l > 0.f ? 1.f / l : 0.f;
+                    __nv_bfloat16* orow = reinterpret_cast<__nv_bfloat16*>(p.O) + (size_t)sg.b * p.o_stride_b + (size_t)t * p.o_stride_t +
+                                          (size_t)(sg.h * G + g) * p.o_stride_h;
+#pragma unroll 1
+                    for (int c = 0; c < 4; ++c) {
+                        uint32_t v[32];
+                        tmem_ld32(tO + c * 32, v);
+                        tmem_wait_ld();
+                        if (row_valid) {
+#pragma unroll
+                            for (int q = 0; q < 4; ++q) {      // 16-byte stores: O strides are only guaranteed 16-byte aligned
+                                uint4 o4;
+                                o4.x = pack_bf16(__uint_as_float(v[q * 8 + 0]) * inv, __uint_as_float(v[q * 8 + 1]) * inv);
+                                o4.y = pack_bf16(__uint_as_float(v[q * 8 + 2]) * inv, __uint_as_float(v[q * 8 + 3]) * inv);
+                                o4.z = pack_bf16(__uint_as_float(v[q * 8 + 4]) * inv, __uint_as_float(v[q * 8 + 5]) * inv);
+                                o4.w = pack_bf16(__uint_as_float(v[q * 8 + 6]) * inv, __uint_as_float(v[q * 8 + 7]) * inv);
+                                *reinterpret_cast<uint4*>(orow + c * 32 + q * 8) = o4;
+                            }
+                        }
+                    }
+                    if (row_valid && p.LSE)
+                        p.LSE[((size_t)sg.b * p.Hq + sg.h * G + g) * p.T_max + t] =
+                            l > 0.f ? (m_ref * sl2 + log2f(l)) * kLn2 : -CUDART_INF_F;
+                } else {
+                    float* base = a.partial + (size_t)sg.slot * SLOT_FLOATS;
+                    const int lr = (int)rank * 128 + rl;
+                    float* prow = base + (size_t)lr * D;
+#pragma unroll 1
+                    for (int c = 0; c < 4; ++c) {
+                        uint32_t v[32];
+                        tmem_ld32(tO + c * 32, v);
+                        tmem_wait_ld();
+#pragma unroll
+                        for (int q = 0; q < 4; ++q)      // 32-byte stores: every store fills a whole sector
+                            st_global_v8(prow + c * 32 + q * 8, v[q * 8], v[q * 8 + 1], v[q * 8 + 2], v[q * 8 + 3], v[q * 8 + 4],
+                                         v[q * 8 + 5], v[q * 8 + 6], v[q * 8 + 7]);
+                    }
+                    base[BR * D + lr] = m_ref == -CUDART_INF_F ? -CUDART_INF_F : m_ref * sl2;
+                    base[BR * D + BR + lr] = l;
+                }
+                tc_fence_before();                 // TMEM reads done before the next segment's MMAs are released
+                jt += nt;
+                ++n_seg_done;
+            }
+        }
+
+        // ---- next round (only batches with very many short sequences need more than one)
+        const long long g_next = plan.gnext, g_hi = plan.ghi;
+        if (g_next >= g_hi) break;
+        __syncthreads();
+        if (warp == 0) plan_round(a, G, worker, rank == 0, plan, g_next, g_hi);
+        __syncthreads();
+        if (plan.nseg == 0) break;
+    }
+
+    PSTAMP(threadIdx.x == 128, 299);
+    // ---- teardown: nobody leaves while its partner may still read its shared memory or signal its barriers;
+    // both CTAs free the tensor memory of the pair
+    tc_fence_before();
+    __syncthreads();
+    cluster_sync_all();
+    if (warp == 1) {
+        tc_fence_after();
+        asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(512u) : "memory");
     }
 }
 
@@ -1013,11 +1504,13 @@ typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t,
                                   const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
                                   CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
 EncodeTiledFn g_encode = nullptr;
+constexpr int kMaxDevices = 64;
+int g_pair_clusters[kMaxDevices] = {0};      // resident 2-CTA clusters of the pair kernel per device (0: not asked yet)
 
-int make_kv_map(CUtensorMap* map, const void* base, const graft_attn_params* p) {
+int make_kv_map(CUtensorMap* map, const void* base, const graft_attn_params* p, int box_rows = BN) {
     const cuuint64_t dims[4] = {(cuuint64_t)p->d, (cuuint64_t)p->S_cap, (cuuint64_t)p->Hkv, (cuuint64_t)p->B};
     const cuuint64_t strides[3] = {(cuuint64_t)p->kv_stride_s * 2, (cuuint64_t)p->kv_stride_h * 2, (cuuint64_t)p->kv_stride_b * 2};
-    const cuuint32_t box[4] = {64, (cuuint32_t)BN, 1, 1};
+    const cuuint32_t box[4] = {64, (cuuint32_t)box_rows, 1, 1};
     const cuuint32_t estr[4] = {1, 1, 1, 1};
     const CUresult rc = g_encode(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void*>(base), dims, strides, box, estr,
                                  CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
@@ -1059,7 +1552,42 @@ int graft_attn_tc_init() {
         g_encode = reinterpret_cast<EncodeTiledFn>(fn);
     }
     GRAFT_CHECK_CUDA(cudaFuncSetAttribute(attn_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_DYN));
+    // pair kernel: how many 2-CTA clusters fit on the device at once (SMs that cannot be paired stay idle)
+    GRAFT_CHECK_CUDA(cudaFuncSetAttribute(attn_tc_pair_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, P_SMEM_DYN));
+    int dev = 0;
+    GRAFT_CHECK_CUDA(cudaGetDevice(&dev));
+    if (dev >= 0 && dev < kMaxDevices && g_pair_clusters[dev] == 0) {
+        int sms = 0;
+        GRAFT_CHECK_CUDA(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev));
+        cudaLaunchConfig_t cfg = {};
+        cfg.gridDim = dim3((unsigned)(sms & ~1));
+        cfg.blockDim = dim3(P_NTHREADS);
+        cfg.dynamicSmemBytes = P_SMEM_DYN;
+        cudaLaunchAttribute attr;
+        attr.id = cudaLaunchAttributeClusterDimension;
+        attr.val.clusterDim.x = 2;
+        attr.val.clusterDim.y = 1;
+        attr.val.clusterDim.z = 1;
+        cfg.attrs = &attr;
+        cfg.numAttrs = 1;
+        int n = 0;
+        if (cudaOccupancyMaxActiveClusters(&n, attn_tc_pair_kernel, &cfg) != cudaSuccess) { (void)cudaGetLastError(); n = 0; }
+        g_pair_clusters[dev] = n > 0 ? (n < sms / 2 ? n : sms / 2) : -1;      // -1: the pair kernel cannot run here
+    }
     return GRAFT_OK;
+}
+
+// number of resident CTA pairs of the pair kernel on the current device (0 if it cannot run)
+static int pair_clusters() {
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return 0;
+    return g_pair_clusters[dev] > 0 ? g_pair_clusters[dev] : 0;
+}
+
+// The pair kernel pays off when items carry more than 128 rows (the second SM of a pair would otherwise idle).
+bool graft_attn_tc_pair_supported(const graft_ctx* ctx, const graft_attn_params* p) {
+    if (!graft_attn_tc_supported(ctx, p)) return false;
+    return pair_clusters() > 0;
 }
 
 bool graft_attn_tc_supported(const graft_ctx* ctx, const graft_attn_params* p) {
@@ -1076,11 +1604,15 @@ size_t graft_attn_tc_ws_bytes(int num_sms, int B, int, int, int d, int) {
     return kDescBytes + cut_bytes(B) + (size_t)num_sms * 2 * SLOT_FLOATS * sizeof(float);
 }
 
-int graft_attn_tc_launch(graft_ctx* ctx, const graft_attn_params* p, cudaStream_t stream) {
-    CUtensorMap kmap, vmap;
-    int rc = make_kv_map(&kmap, p->Kc, p);
-    if (rc == GRAFT_OK) rc = make_kv_map(&vmap, p->Vc, p);
+int graft_attn_tc_launch(graft_ctx* ctx, const graft_attn_params* p, cudaStream_t stream, int pair) {
     const int G = p->Hq / p->Hkv;
+    // pair < 0: choose.  The pair kernel measured faster on every benchmark configuration (3 % at 64K context
+    // with 240-row items up to 20 % on batches of short sequences), so it runs wherever clusters of two fit.
+    const bool use_pair = pair > 0 || (pair < 0 && graft_attn_tc_pair_supported(ctx, p));
+    if (use_pair && !graft_attn_tc_pair_supported(ctx, p)) return GRAFT_ERR_UNSUPPORTED;
+    CUtensorMap kmap, vmap;
+    int rc = make_kv_map(&kmap, p->Kc, p, use_pair ? 64 : BN);
+    if (rc == GRAFT_OK) rc = make_kv_map(&vmap, p->Vc, p);
     CUtensorMap qmap = kmap;                 // unused placeholder unless Q goes by TMA
     const bool q_tma = q_map_possible(p, G);
     if (rc == GRAFT_OK && q_tma) rc = make_q_map(&qmap, p, G);
@@ -1100,6 +1632,11 @@ int graft_attn_tc_launch(graft_ctx* ctx, const graft_attn_params* p, cudaStream_
 #ifdef GRAFT_TC_EXPERIMENTS
     if (getenv("GRAFT_TC_GRID")) grid = atoi(getenv("GRAFT_TC_GRID"));
 #endif
+    if (use_pair) {
+        int pairs = pair_clusters();
+        if (pairs > ctx->num_sms / 2) pairs = ctx->num_sms / 2;       // the workspace has two slots per SM
+        attn_tc_pair_kernel<<<2 * pairs, P_NTHREADS, P_SMEM_DYN, stream>>>(kmap, vmap, qmap, a, ctx->status);
+    } else
     attn_tc_kernel<<<grid, NTHREADS, SMEM_DYN, stream>>>(kmap, vmap, qmap, a, ctx->status);
     GRAFT_CHECK_CUDA(cudaGetLastError());
     // few rows: one row per warp (the merge is latency-bound); many rows: four, to keep the CTA count down

@@ -27,11 +27,14 @@ def Step():
     return VerifyStep
 
 
-VARIANTS = ["mma", "auto"]
+VARIANTS = ["mma", "auto", "one", "pair"]      # "one"/"pair": the one-SM and the two-SM tcgen05 kernel, forced
 
 
-def variant_id(G, name):
-    return {"mma": G.ATTN_MMA_SYNC, "auto": G.ATTN_AUTO, "tc": G.ATTN_TCGEN05}[name]
+def variant_id(G, name, w=None):
+    if name in ("one", "pair") and w is not None and w.d != 128:
+        pytest.skip("the tcgen05 kernels take d = 128 only")
+    return {"mma": G.ATTN_MMA_SYNC, "auto": G.ATTN_AUTO, "tc": G.ATTN_TCGEN05, "one": G.ATTN_TCGEN05_1SM,
+            "pair": G.ATTN_TCGEN05_2SM}[name]
 
 
 def check_tree(vs, tree):
@@ -90,7 +93,7 @@ def full_case(orc, G, Step, w, variant, rows=None, poison=True):
     vs = Step(w)
     vs.build()
     check_tree(vs, tree)
-    vs.attn(variant_id(G, variant))
+    vs.attn(variant_id(G, variant, w))
     torch.cuda.synchronize()
     e = check_attn(orc, w, vs, tree, rows)
     assert vs.ctx.device_status() == 0
@@ -157,7 +160,7 @@ def test_strided_cache_and_no_lse(orc, G, Step, variant):
     Vt = vs.Vc.permute(0, 2, 1, 3).contiguous().permute(0, 2, 1, 3)
     vs.LSE.fill_(7.0)
     G.graft_tree_verify_attn(vs.ctx, Q=vs.Q, Kc=Kt, Vc=Vt, O=vs.O, seq_len=vs.seq_len, tree_size=vs.tree_size,
-                             tree_anc=vs.tree_anc, scale=w.scale, LSE=None, variant=variant_id(G, variant))
+                             tree_anc=vs.tree_anc, scale=w.scale, LSE=None, variant=variant_id(G, variant, w))
     torch.cuda.synchronize()
     assert (vs.LSE == 7.0).all()
     out = orc.tree_attn(W.bf16_bits(w.Q), W.bf16_bits(w.Kc), W.bf16_bits(w.Vc), w.seq_len, tree["tree_size"],
@@ -177,12 +180,12 @@ def test_mask_locality_on_device(orc, G, Step, variant):
     W.make_qkv(w, tree["tree_size"], poison=True)
     vs = Step(w)
     vs.build()
-    vs.attn(variant_id(G, variant))
+    vs.attn(variant_id(G, variant, w))
     base = vs.O.clone()
     u = 11
     vs.Vc[0, :, 200 + u] += 2.0
     vs.Kc[0, :, 200 + u] *= -1.0
-    vs.attn(variant_id(G, variant))
+    vs.attn(variant_id(G, variant, w))
     changed = (vs.O != base).flatten(2).any(-1)[0].cpu().numpy()          # [T_max]
     anc = tree["tree_anc"][0]
     for t in range(30):
@@ -347,7 +350,7 @@ def test_invalid_sequence_inside_a_batch(orc, G, Step):
     vs.tree_size[1] = 33                                   # larger than T_max: invalid
     for variant in VARIANTS:
         vs.O.fill_(float("nan"))
-        vs.attn(variant_id(G, variant))
+        vs.attn(variant_id(G, variant, w))
         torch.cuda.synchronize()
         assert vs.ctx.device_status() == G.FLAG_BAD_SIZE
         O = vs.O.cpu().to(torch.float64).numpy()
