@@ -921,12 +921,13 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap kmap, const __grid_constant__
 // reaches past the sequence's keys (rows before key 0 are zero-filled by the copy), and the columns that
 // the previous tile already covered are masked like non-ancestors.
 constexpr int P_NTHREADS = 256;
-constexpr int P_SLOT_BYTES = TILE_BYTES / 2;      // half a K tile or half a V tile
-constexpr int P_NSLOT = 12;
+constexpr int P_HALF_TILE = TILE_BYTES / 2;       // this CTA's half of a K tile or of a V tile
+constexpr int P_SLOT_BYTES = 2 * P_HALF_TILE;     // one ring slot: the K half, then the V half of a tile
+constexpr int P_NSLOT = 6;
 constexpr int kCtrlBytes = 1024;
 constexpr int P_SMEM_DYN = kCtrlBytes + TILE_BYTES + P_NSLOT * P_SLOT_BYTES;      // control, Q (128 rows), ring
 enum { PB_FULL = 0, PB_EMPTY = P_NSLOT, PB_S = 2 * P_NSLOT, PB_P = 2 * P_NSLOT + 2, PB_Q = 2 * P_NSLOT + 4, PB_O = 2 * P_NSLOT + 5,
-       PB_QFREE = 2 * P_NSLOT + 6, PB_PVD = 2 * P_NSLOT + 7, PB_COUNT = 2 * P_NSLOT + 8 };
+       PB_QFREE = 2 * P_NSLOT + 6, PB_COUNT = 2 * P_NSLOT + 7 };
 struct PairCtrl {
     uint64_t bar[PB_COUNT];
     Plan plan;
@@ -934,6 +935,11 @@ struct PairCtrl {
     int abort;
 };
 static_assert(sizeof(PairCtrl) <= kCtrlBytes, "control block too large");
+#ifdef GRAFT_TC_EXPERIMENTS
+constexpr int kProfBytes = 1024;      // time stamps of one CTA
+#else
+constexpr int kProfBytes = 0;
+#endif
 
 __device__ __forceinline__ uint32_t cluster_ctarank() {
     uint32_t r;
@@ -1022,7 +1028,8 @@ attn_tc_pair_kernel(const __grid_constant__ CUtensorMap kmap, const __grid_const
 #ifdef GRAFT_TC_EXPERIMENTS
     const long long t_entry = clock64();
     const bool prof = (int)blockIdx.x == a.prof_cta;
-#define PSTAMP(cond, idx) do { if (prof && (cond)) a.desc[(idx)] = (int)(clock64() - t_entry); } while (0)
+    volatile int* s_prof = reinterpret_cast<volatile int*>(smem_raw + P_SMEM_DYN);       // experiments: 1 KB more is requested
+#define PSTAMP(cond, idx) do { if (prof && (cond)) s_prof[(idx) - 256] = (int)(clock() - (int)t_entry); } while (0)
 #else
 #define PSTAMP(cond, idx) do { } while (0)
 #endif
@@ -1051,7 +1058,6 @@ attn_tc_pair_kernel(const __grid_constant__ CUtensorMap kmap, const __grid_const
         mbar_init(bar(PB_Q), a.q_tma ? 2 : 4);      // by TMA: one arrival per CTA; staged by threads: one per stager warp
         mbar_init(bar(PB_O), 1);
         mbar_init(bar(PB_QFREE), 1);
-        mbar_init(bar(PB_PVD), 1);
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     if (warp == 1) {
@@ -1075,8 +1081,7 @@ attn_tc_pair_kernel(const __grid_constant__ CUtensorMap kmap, const __grid_const
     };
 
     // running counters that persist across segments and rounds (each role keeps its own copy)
-    int n_load = 0;            // ring loads issued / consumed so far (2 per tile)
-    int jt = 0;                // tiles processed so far (S, P and PV-done barrier phases)
+    int jt = 0;                // tiles issued / processed so far: ring slot and use, S and P barrier phases
     int n_seg_done = 0;        // segments finished (Q, Q-free and O barrier phases)
 
     for (;;) {                 // rounds of <= MAXSEG segments
@@ -1087,74 +1092,60 @@ attn_tc_pair_kernel(const __grid_constant__ CUtensorMap kmap, const __grid_const
             if (lane == 0) {
                 for (int si = 0; si < nseg; ++si) {
                     const Seg sg = plan.seg[si];
-                    for (int t = sg.tile_lo; t < sg.tile_hi; ++t) {
+                    for (int t = sg.tile_lo; t < sg.tile_hi; ++t, ++jt) {
                         int overlap;
                         const int key0 = tile_key0(sg, t, overlap);
-                        for (int which = 0; which < 2; ++which, ++n_load) {
-                            const int slot = n_load % P_NSLOT, use = n_load / P_NSLOT;
-                            if (use > 0) mbar_wait(bar(PB_EMPTY + slot), (use - 1) & 1, abort_flag, status);
-                            if (rank == 0) mbar_expect_tx(bar(PB_FULL + slot), 2 * P_SLOT_BYTES);      // both halves
-                            const uint32_t dst = sRing + slot * P_SLOT_BYTES;
-                            const uint32_t fb = leader_bar(PB_FULL + slot);
-                            if (which == 0) {      // 64 keys of the K tile, all of d (two 64-column boxes)
-                                tma_pair_4d(dst, &kmap, 0, key0 + 64 * (int)rank, sg.h, sg.b, fb);
-                                tma_pair_4d(dst + P_SLOT_BYTES / 2, &kmap, 64, key0 + 64 * (int)rank, sg.h, sg.b, fb);
-                            } else {               // all keys of the V tile, 64 columns of d
-                                tma_pair_4d(dst, &vmap, 64 * (int)rank, key0, sg.h, sg.b, fb);
-                            }
-                        }
+                        const int slot = jt % P_NSLOT, use = jt / P_NSLOT;
+                        if (use > 0) mbar_wait(bar(PB_EMPTY + slot), (use - 1) & 1, abort_flag, status);
+                        if (rank == 0) mbar_expect_tx(bar(PB_FULL + slot), 2 * P_SLOT_BYTES);      // K and V halves of both CTAs
+                        const uint32_t dst = sRing + slot * P_SLOT_BYTES;
+                        const uint32_t fb = leader_bar(PB_FULL + slot);
+                        // 64 keys of the K tile, all of d (two 64-column boxes); all keys of the V tile, 64 columns of d
+                        tma_pair_4d(dst, &kmap, 0, key0 + 64 * (int)rank, sg.h, sg.b, fb);
+                        tma_pair_4d(dst + P_HALF_TILE / 2, &kmap, 64, key0 + 64 * (int)rank, sg.h, sg.b, fb);
+                        tma_pair_4d(dst + P_HALF_TILE, &vmap, 64 * (int)rank, key0, sg.h, sg.b, fb);
                     }
                 }
             }
         } else if (warp == 1) {
             // =============================== MMA issuer (leader only) ===============================
             if (lane == 0 && rank == 0) {
-                auto wait_full = [&](int n) { mbar_wait(bar(PB_FULL + n % P_NSLOT), (n / P_NSLOT) & 1, abort_flag, status); };
                 for (int si = 0; si < nseg; ++si) {
                     const Seg sg = plan.seg[si];
                     const int nt = sg.tile_hi - sg.tile_lo;
-                    // S[buffer gt & 1] = Q K^T with the K tile of ring load n
-                    auto issue_qk = [&](int gt, int n) {
-                        wait_full(n);
-                        PSTAMP(gt >= 40 && gt < 48, 343 + (gt - 40) * 4);
+                    // S[buffer gt & 1] = Q K^T with the K half-tiles of ring slot gt % P_NSLOT (V of the same tile lands with it)
+                    auto issue_qk = [&](int gt) {
+                        mbar_wait(bar(PB_FULL + gt % P_NSLOT), (gt / P_NSLOT) & 1, abort_flag, status);
                         tc_fence_after();
-                        const uint32_t sK16 = (sRing + (n % P_NSLOT) * P_SLOT_BYTES) >> 4;
+                        const uint32_t sK16 = (sRing + (gt % P_NSLOT) * P_SLOT_BYTES) >> 4;
                         const uint32_t sQ16 = sQ >> 4;
 #pragma unroll
                         for (int k = 0; k < D / 16; ++k) {
                             const uint32_t offQ = ((k >> 2) * HALF_BYTES + (k & 3) * 32) >> 4;
-                            const uint32_t offK = ((k >> 2) * (P_SLOT_BYTES / 2) + (k & 3) * 32) >> 4;
+                            const uint32_t offK = ((k >> 2) * (P_HALF_TILE / 2) + (k & 3) * 32) >> 4;
                             mma_pair_ss(tmem + (gt & 1) * 128, smem_desc(kDescKMajor, sQ16 + offQ), smem_desc(kDescKMajor, sK16 + offK), kIdescPairQK, k > 0);
                         }
                         tc_commit_pair(bar(PB_S + (gt & 1)));
-                        tc_commit_pair(bar(PB_EMPTY + n % P_NSLOT));          // K tile fully read
                     };
                     mbar_wait_cluster(bar(PB_Q), n_seg_done & 1, abort_flag, status);   // Q of this segment is in place in both CTAs
-                    issue_qk(jt, n_load);
+                    issue_qk(jt);
                     if (nt == 1) tc_commit_pair(bar(PB_QFREE));      // the segment's last Q K^T is in the pipe
                     for (int j = 0; j < nt; ++j) {
                         const int gt = jt + j;
                         if (j + 1 < nt) {
-                            issue_qk(gt + 1, n_load + 2 * (j + 1));             // runs while the softmax warps work on tile j
+                            issue_qk(gt + 1);                                   // runs while the softmax warps work on tile j
                             if (j + 2 == nt) tc_commit_pair(bar(PB_QFREE));
                         }
-                        const int nV = n_load + 2 * j + 1;
-                        PSTAMP(gt >= 40 && gt < 48, 340 + (gt - 40) * 4);
                         mbar_wait_cluster(bar(PB_P + (gt & 1)), (gt >> 1) & 1, abort_flag, status);
-                        PSTAMP(gt >= 40 && gt < 48, 341 + (gt - 40) * 4);
-                        wait_full(nV);
                         tc_fence_after();
-                        const uint32_t sV16 = (sRing + (nV % P_NSLOT) * P_SLOT_BYTES) >> 4;
+                        const uint32_t sV16 = (sRing + (gt % P_NSLOT) * P_SLOT_BYTES + P_HALF_TILE) >> 4;
 #pragma unroll
                         for (int k = 0; k < BN / 16; ++k)
                             mma_pair_ts(tmem + 256, tmem + (gt & 1) * 128 + k * 8, smem_desc(kDescVMajor, sV16 + k * (2048 >> 4)), kIdescPairPV,
                                         (j > 0 || k > 0) ? 1u : 0u);
-                        tc_commit_pair(bar(PB_EMPTY + nV % P_NSLOT));         // V tile fully read
-                        tc_commit_pair(bar(PB_PVD));                          // O holds tiles 0..j
-                        PSTAMP(gt >= 40 && gt < 48, 342 + (gt - 40) * 4);
+                        tc_commit_pair(bar(PB_EMPTY + gt % P_NSLOT));         // the tile's K and V are read, O holds tiles 0..j
                     }
                     tc_commit_pair(bar(PB_O));
-                    n_load += 2 * nt;
                     jt += nt;
                     ++n_seg_done;
                 }
@@ -1265,7 +1256,7 @@ attn_tc_pair_kernel(const __grid_constant__ CUtensorMap kmap, const __grid_const
                     if (mx != -CUDART_INF_F && (m_ref == -CUDART_INF_F || (mx - m_ref) * sl2 > kRescaleThreshold)) {
                         if (m_ref != -CUDART_INF_F) {
                             // O must hold every earlier tile of the segment before it is rescaled (j > 0 here)
-                            mbar_wait(bar(PB_PVD), (gt - 1) & 1, abort_flag, status);
+                            mbar_wait(bar(PB_EMPTY + (gt - 1) % P_NSLOT), ((gt - 1) / P_NSLOT) & 1, abort_flag, status);
                             tc_fence_after();
                             const float alpha = exp2f((m_ref - mx) * sl2);
                             l *= alpha;
@@ -1368,6 +1359,10 @@ attn_tc_pair_kernel(const __grid_constant__ CUtensorMap kmap, const __grid_const
     }
 
     PSTAMP(threadIdx.x == 128, 299);
+#ifdef GRAFT_TC_EXPERIMENTS
+    __syncthreads();
+    if (prof && threadIdx.x < 256) a.desc[256 + threadIdx.x] = s_prof[threadIdx.x];
+#endif
     // ---- teardown: nobody leaves while its partner may still read its shared memory or signal its barriers;
     // both CTAs free the tensor memory of the pair
     tc_fence_before();
@@ -1553,7 +1548,7 @@ int graft_attn_tc_init() {
     }
     GRAFT_CHECK_CUDA(cudaFuncSetAttribute(attn_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_DYN));
     // pair kernel: how many 2-CTA clusters fit on the device at once (SMs that cannot be paired stay idle)
-    GRAFT_CHECK_CUDA(cudaFuncSetAttribute(attn_tc_pair_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, P_SMEM_DYN));
+    GRAFT_CHECK_CUDA(cudaFuncSetAttribute(attn_tc_pair_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, P_SMEM_DYN + kProfBytes));
     int dev = 0;
     GRAFT_CHECK_CUDA(cudaGetDevice(&dev));
     if (dev >= 0 && dev < kMaxDevices && g_pair_clusters[dev] == 0) {
@@ -1562,7 +1557,7 @@ int graft_attn_tc_init() {
         cudaLaunchConfig_t cfg = {};
         cfg.gridDim = dim3((unsigned)(sms & ~1));
         cfg.blockDim = dim3(P_NTHREADS);
-        cfg.dynamicSmemBytes = P_SMEM_DYN;
+        cfg.dynamicSmemBytes = P_SMEM_DYN + kProfBytes;
         cudaLaunchAttribute attr;
         attr.id = cudaLaunchAttributeClusterDimension;
         attr.val.clusterDim.x = 2;
@@ -1635,7 +1630,7 @@ int graft_attn_tc_launch(graft_ctx* ctx, const graft_attn_params* p, cudaStream_
     if (use_pair) {
         int pairs = pair_clusters();
         if (pairs > ctx->num_sms / 2) pairs = ctx->num_sms / 2;       // the workspace has two slots per SM
-        attn_tc_pair_kernel<<<2 * pairs, P_NTHREADS, P_SMEM_DYN, stream>>>(kmap, vmap, qmap, a, ctx->status);
+        attn_tc_pair_kernel<<<2 * pairs, P_NTHREADS, P_SMEM_DYN + kProfBytes, stream>>>(kmap, vmap, qmap, a, ctx->status);
     } else
     attn_tc_kernel<<<grid, NTHREADS, SMEM_DYN, stream>>>(kmap, vmap, qmap, a, ctx->status);
     GRAFT_CHECK_CUDA(cudaGetLastError());
