@@ -26,6 +26,7 @@ def build(force: bool = False, verbose: bool = False) -> str:
     flags = list(NVCC_FLAGS)
     if os.environ.get("GRAFT_TC_EXPERIMENTS"):      # ablation switches and phase timers of the tcgen05 kernel
         flags.append("-DGRAFT_TC_EXPERIMENTS")
+        flags += ["-D" + d for d in os.environ.get("GRAFT_TC_DEFINES", "").split()]      # further experiment macros
         force = True
     if not force and os.path.exists(LIB) and os.path.getmtime(LIB) >= _newest_source():
         return LIB

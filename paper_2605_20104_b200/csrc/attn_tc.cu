@@ -910,12 +910,16 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap kmap, const __grid_constant__
 // CTA 1 rows 128..255, each in its own tensor memory.  The B operand is split between the two shared
 // memories: of a K tile each CTA fetches 64 of the 128 keys (all of d), of a V tile all 128 keys and 64 of
 // the d columns, so every byte of the cache still crosses into the pair once.  With one row block per SM
-// the score tile is double-buffered in tensor memory (columns 0..127 and 128..255, O at 256..383): the
-// tensor pipe computes S of tile j+1 while the softmax warps work on tile j.
+// there is room for three score buffers in tensor memory (columns 0..383, O at 384..511): Q K^T runs two
+// tiles ahead of P V, so the tensor pipe never waits for the buffer that holds P of the tile in the softmax.
 //
 // Barriers live at the same offset in both shared memories.  Copies of both CTAs complete on the leader's
 // (CTA 0's) FULL and Q barriers; the softmax warps of both arrive on the leader's P barriers; everything
-// the MMA thread commits is multicast to both CTAs (slot free, S ready, PV done, O final, Q free).
+// the MMA thread commits is multicast to both CTAs (slot free, S ready, O final, Q free).
+//
+// Measured on the 64K-context configuration (per 128-key tile and pair): the sixteen 256-row MMAs take about
+// 1500 cycles with the softmax arithmetic switched off and about 1850 with it, the softmax of one tile about
+// 1600; the kernel is bound by the tensor pipe in this mode.
 //
 // The last tile of an item is fetched at keys [L+T-128, L+T) instead of a tile-aligned position: it never
 // reaches past the sequence's keys (rows before key 0 are zero-filled by the copy), and the columns that
@@ -926,8 +930,9 @@ constexpr int P_SLOT_BYTES = 2 * P_HALF_TILE;     // one ring slot: the K half, 
 constexpr int P_NSLOT = 6;
 constexpr int kCtrlBytes = 1024;
 constexpr int P_SMEM_DYN = kCtrlBytes + TILE_BYTES + P_NSLOT * P_SLOT_BYTES;      // control, Q (128 rows), ring
-enum { PB_FULL = 0, PB_EMPTY = P_NSLOT, PB_S = 2 * P_NSLOT, PB_P = 2 * P_NSLOT + 2, PB_Q = 2 * P_NSLOT + 4, PB_O = 2 * P_NSLOT + 5,
-       PB_QFREE = 2 * P_NSLOT + 6, PB_COUNT = 2 * P_NSLOT + 7 };
+constexpr int P_NSBUF = 3;                        // score buffers in tensor memory (128 columns each), O behind them
+enum { PB_FULL = 0, PB_EMPTY = P_NSLOT, PB_S = 2 * P_NSLOT, PB_P = PB_S + P_NSBUF, PB_Q = PB_P + P_NSBUF, PB_O = PB_Q + 1,
+       PB_QFREE = PB_O + 1, PB_COUNT = PB_QFREE + 1 };
 struct PairCtrl {
     uint64_t bar[PB_COUNT];
     Plan plan;
@@ -972,6 +977,13 @@ __device__ __forceinline__ bool mbar_try_wait_cluster(uint32_t bar, uint32_t par
                  : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
     return ok != 0;
 }
+// non-blocking test; issued ahead of a run of MMAs so that its latency hides behind them
+__device__ __forceinline__ bool mbar_test(uint32_t bar, uint32_t parity) {
+    uint32_t ok;
+    asm volatile("{\n\t.reg .pred p;\n\tmbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2;\n\tselp.u32 %0, 1, 0, p;\n\t}"
+                 : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+    return ok != 0;
+}
 __device__ __forceinline__ void mbar_wait_cluster(uint32_t bar, uint32_t parity, volatile int* abort_flag, unsigned* status) {
     if (mbar_try_wait_cluster(bar, parity)) return;
     if (*abort_flag) return;
@@ -997,13 +1009,13 @@ __device__ __forceinline__ void tma_pair_5d(uint32_t dst, const CUtensorMap* map
 // D[tmem of both CTAs] (+)= A * B over the pair; issued by one thread of the leader
 __device__ __forceinline__ void mma_pair_ss(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc, uint32_t accumulate) {
     asm volatile("{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
-                 "tcgen05.mma.cta_group::2.kind::f16 [%0], %1, %2, %3, {%5, %5, %5, %5, %5, %5, %5, %5}, p;\n\t}"
-                 ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate), "r"(0u) : "memory");
+                 "tcgen05.mma.cta_group::2.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+                 ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate) : "memory");
 }
 __device__ __forceinline__ void mma_pair_ts(uint32_t d_tmem, uint32_t a_tmem, uint64_t b_desc, uint32_t idesc, uint32_t accumulate) {
     asm volatile("{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
-                 "tcgen05.mma.cta_group::2.kind::f16 [%0], [%1], %2, %3, {%5, %5, %5, %5, %5, %5, %5, %5}, p;\n\t}"
-                 ::"r"(d_tmem), "r"(a_tmem), "l"(b_desc), "r"(idesc), "r"(accumulate), "r"(0u) : "memory");
+                 "tcgen05.mma.cta_group::2.kind::f16 [%0], [%1], %2, %3, p;\n\t}"
+                 ::"r"(d_tmem), "r"(a_tmem), "l"(b_desc), "r"(idesc), "r"(accumulate) : "memory");
 }
 // arrive on the barrier at this offset in both CTAs once every MMA issued so far is complete
 __device__ __forceinline__ void tc_commit_pair(uint32_t bar) {
@@ -1054,7 +1066,7 @@ attn_tc_pair_kernel(const __grid_constant__ CUtensorMap kmap, const __grid_const
 
     if (threadIdx.x == 0) {
         for (int i = 0; i < P_NSLOT; ++i) { mbar_init(bar(PB_FULL + i), 1); mbar_init(bar(PB_EMPTY + i), 1); }
-        for (int i = 0; i < 2; ++i) { mbar_init(bar(PB_S + i), 1); mbar_init(bar(PB_P + i), 8); }      // 4 softmax warps in each CTA
+        for (int i = 0; i < P_NSBUF; ++i) { mbar_init(bar(PB_S + i), 1); mbar_init(bar(PB_P + i), 8); }      // 4 softmax warps in each CTA
         mbar_init(bar(PB_Q), a.q_tma ? 2 : 4);      // by TMA: one arrival per CTA; staged by threads: one per stager warp
         mbar_init(bar(PB_O), 1);
         mbar_init(bar(PB_QFREE), 1);
@@ -1113,9 +1125,10 @@ attn_tc_pair_kernel(const __grid_constant__ CUtensorMap kmap, const __grid_const
                 for (int si = 0; si < nseg; ++si) {
                     const Seg sg = plan.seg[si];
                     const int nt = sg.tile_hi - sg.tile_lo;
-                    // S[buffer gt & 1] = Q K^T with the K half-tiles of ring slot gt % P_NSLOT (V of the same tile lands with it)
-                    auto issue_qk = [&](int gt) {
-                        mbar_wait(bar(PB_FULL + gt % P_NSLOT), (gt / P_NSLOT) & 1, abort_flag, status);
+                    // S[buffer gt % 3] = Q K^T with the K half-tiles of ring slot gt % P_NSLOT (V of the same tile lands with it)
+                    // `landed`: the slot's barrier was already seen complete by an earlier test
+                    auto issue_qk = [&](int gt, bool landed) {
+                        if (!landed) mbar_wait(bar(PB_FULL + gt % P_NSLOT), (gt / P_NSLOT) & 1, abort_flag, status);
                         tc_fence_after();
                         const uint32_t sK16 = (sRing + (gt % P_NSLOT) * P_SLOT_BYTES) >> 4;
                         const uint32_t sQ16 = sQ >> 4;
@@ -1123,25 +1136,32 @@ attn_tc_pair_kernel(const __grid_constant__ CUtensorMap kmap, const __grid_const
                         for (int k = 0; k < D / 16; ++k) {
                             const uint32_t offQ = ((k >> 2) * HALF_BYTES + (k & 3) * 32) >> 4;
                             const uint32_t offK = ((k >> 2) * (P_HALF_TILE / 2) + (k & 3) * 32) >> 4;
-                            mma_pair_ss(tmem + (gt & 1) * 128, smem_desc(kDescKMajor, sQ16 + offQ), smem_desc(kDescKMajor, sK16 + offK), kIdescPairQK, k > 0);
+                            mma_pair_ss(tmem + (gt % P_NSBUF) * 128, smem_desc(kDescKMajor, sQ16 + offQ), smem_desc(kDescKMajor, sK16 + offK), kIdescPairQK, k > 0);
                         }
-                        tc_commit_pair(bar(PB_S + (gt & 1)));
+                        tc_commit_pair(bar(PB_S + gt % P_NSBUF));
                     };
                     mbar_wait_cluster(bar(PB_Q), n_seg_done & 1, abort_flag, status);   // Q of this segment is in place in both CTAs
-                    issue_qk(jt);
-                    if (nt == 1) tc_commit_pair(bar(PB_QFREE));      // the segment's last Q K^T is in the pipe
+                    // Q K^T runs two tiles ahead of P V: with three score buffers S(j+2) does not wait for P(j) to be consumed.
+                    // Every barrier is tested one step early, so that a wait that is already satisfied costs no round trip
+                    // between two runs of MMAs.
+                    issue_qk(jt, false);
+                    if (nt > 1) issue_qk(jt + 1, false);
+                    if (nt <= 2) tc_commit_pair(bar(PB_QFREE));      // the segment's last Q K^T is in the pipe
+                    bool k_landed = nt > 2 && mbar_test(bar(PB_FULL + (jt + 2) % P_NSLOT), ((jt + 2) / P_NSLOT) & 1);
                     for (int j = 0; j < nt; ++j) {
                         const int gt = jt + j;
-                        if (j + 1 < nt) {
-                            issue_qk(gt + 1);                                   // runs while the softmax warps work on tile j
-                            if (j + 2 == nt) tc_commit_pair(bar(PB_QFREE));
+                        const bool p_there = mbar_test(bar(PB_P + gt % P_NSBUF), (gt / P_NSBUF) & 1);
+                        if (j + 2 < nt) {
+                            issue_qk(gt + 2, k_landed);
+                            if (j + 3 == nt) tc_commit_pair(bar(PB_QFREE));
                         }
-                        mbar_wait_cluster(bar(PB_P + (gt & 1)), (gt >> 1) & 1, abort_flag, status);
+                        if (!p_there) mbar_wait_cluster(bar(PB_P + gt % P_NSBUF), (gt / P_NSBUF) & 1, abort_flag, status);
+                        k_landed = j + 3 < nt && mbar_test(bar(PB_FULL + (gt + 3) % P_NSLOT), ((gt + 3) / P_NSLOT) & 1);
                         tc_fence_after();
                         const uint32_t sV16 = (sRing + (gt % P_NSLOT) * P_SLOT_BYTES + P_HALF_TILE) >> 4;
 #pragma unroll
                         for (int k = 0; k < BN / 16; ++k)
-                            mma_pair_ts(tmem + 256, tmem + (gt & 1) * 128 + k * 8, smem_desc(kDescVMajor, sV16 + k * (2048 >> 4)), kIdescPairPV,
+                            mma_pair_ts(tmem + P_NSBUF * 128, tmem + (gt % P_NSBUF) * 128 + k * 8, smem_desc(kDescVMajor, sV16 + k * (2048 >> 4)), kIdescPairPV,
                                         (j > 0 || k > 0) ? 1u : 0u);
                         tc_commit_pair(bar(PB_EMPTY + gt % P_NSLOT));         // the tile's K and V are read, O holds tiles 0..j
                     }
@@ -1198,7 +1218,7 @@ attn_tc_pair_kernel(const __grid_constant__ CUtensorMap kmap, const __grid_const
             // =============================== softmax, results (both CTAs) ===============================
             const int rl = ((warp & 3) << 5) + lane;            // row inside this CTA's block = TMEM lane
             const uint32_t lane_bits = (uint32_t)((warp & 3) << 5) << 16;
-            const uint32_t tO = tmem + lane_bits + 256;
+            const uint32_t tO = tmem + lane_bits + P_NSBUF * 128;
             const float sl2 = p.scale * kLog2e;
             for (int si = 0; si < nseg; ++si) {
                 const Seg sg = plan.seg[si];
@@ -1213,11 +1233,11 @@ attn_tc_pair_kernel(const __grid_constant__ CUtensorMap kmap, const __grid_const
 
                 for (int j = 0; j < nt; ++j) {
                     const int gt = jt + j;
-                    const uint32_t tS = tmem + lane_bits + (gt & 1) * 128;
+                    const uint32_t tS = tmem + lane_bits + (gt % P_NSBUF) * 128;
                     int overlap;
                     const int key0 = tile_key0(sg, sg.tile_lo + j, overlap);
                     const bool masked = key0 + BN > sg.L || overlap > 0;
-                    mbar_wait(bar(PB_S + (gt & 1)), (gt >> 1) & 1, abort_flag, status);
+                    mbar_wait(bar(PB_S + gt % P_NSBUF), (gt / P_NSBUF) & 1, abort_flag, status);
                     tc_fence_after();
                     PSTAMP(threadIdx.x == 128 && gt >= 40 && gt < 48, 300 + (gt - 40) * 4);
                     uint32_t x[4][32];
@@ -1295,7 +1315,7 @@ attn_tc_pair_kernel(const __grid_constant__ CUtensorMap kmap, const __grid_const
                     PSTAMP(threadIdx.x == 128 && gt >= 40 && gt < 48, 381 + (gt - 40) * 2);
                     tc_fence_before();
                     __syncwarp();
-                    if (lane == 0) mbar_arrive_remote(leader_bar(PB_P + (gt & 1)));       // one arrival per warp
+                    if (lane == 0) mbar_arrive_remote(leader_bar(PB_P + gt % P_NSBUF));       // one arrival per warp
                     PSTAMP(threadIdx.x == 128 && gt >= 40 && gt < 48, 302 + (gt - 40) * 4);
                 }
 
