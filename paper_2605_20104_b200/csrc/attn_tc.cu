@@ -924,7 +924,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap kmap, const __grid_constant__
 // The last tile of an item is fetched at keys [L+T-128, L+T) instead of a tile-aligned position: it never
 // reaches past the sequence's keys (rows before key 0 are zero-filled by the copy), and the columns that
 // the previous tile already covered are masked like non-ancestors.
-constexpr int P_NTHREADS = 256;
+constexpr int P_NTHREADS = 256;          // producer, Q K^T issuer, Q loader, P V issuer, four softmax warps
 constexpr int P_HALF_TILE = TILE_BYTES / 2;       // this CTA's half of a K tile or of a V tile
 constexpr int P_SLOT_BYTES = 2 * P_HALF_TILE;     // one ring slot: the K half, then the V half of a tile
 constexpr int P_NSLOT = 6;
@@ -1027,6 +1027,184 @@ constexpr uint32_t kIdescPairBase = (1u << 4) | (1u << 7) | (1u << 10) | ((128u 
 constexpr uint32_t kIdescPairQK = kIdescPairBase;
 constexpr uint32_t kIdescPairPV = kIdescPairBase | (1u << 16);
 
+// ---------------------------------------------------------------------------------------------------
+// softmax and results of one 128-row block (four warps, one row per thread), shared by the kernels that
+// keep three score buffers in tensor memory (columns 0..383) and O behind them (384..511)
+// ---------------------------------------------------------------------------------------------------
+struct SoftmaxBars {
+    int S, P, O;             // barrier indices: score buffer ready (x3), P written (x3), all MMAs of the segment complete
+    int pv_done, pv_mod;     // barrier whose phase tile/pv_mod of index pv_done + tile % pv_mod completes with P V of `tile`
+    bool remote;             // P barriers live in CTA 0 of the cluster
+};
+// first key and number of already-covered columns of tile t of an item: the last tile is fetched at keys
+// [L+T-128, L+T), so it never reaches past the sequence's keys (rows before key 0 are zero-filled by the copy)
+__device__ __forceinline__ int tile_key0(const Seg& sg, int t, int& overlap) {
+    const int n_keys = sg.L + sg.T;
+    const int ntiles = (n_keys + BN - 1) / BN;
+    overlap = 0;
+    if (t < ntiles - 1) return t * BN;
+    overlap = ntiles * BN - n_keys;
+    return n_keys - BN;
+}
+
+__device__ __forceinline__ void softmax_rows(const TcArgs& a, const Plan& plan, const SoftmaxBars lay, uint32_t bar0, uint32_t tmem, int rank,
+                                             int& jt, int& n_seg_done, volatile int* abort_flag, unsigned* status) {
+    const graft_attn_params& p = a.p;
+    const int G = a.G;
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int nseg = plan.nseg;
+    auto bar = [&](int i) { return bar0 + 8u * (uint32_t)i; };
+    const int rl = ((warp & 3) << 5) + lane;            // row inside this CTA's block = TMEM lane
+    const uint32_t lane_bits = (uint32_t)((warp & 3) << 5) << 16;
+    const uint32_t tO = tmem + lane_bits + P_NSBUF * 128;
+    const float sl2 = p.scale * kLog2e;
+    for (int si = 0; si < nseg; ++si) {
+        const Seg sg = plan.seg[si];
+        const int nt = sg.tile_hi - sg.tile_lo;
+        const int R = sg.T * G;
+        const int r = sg.rb * BR + (int)rank * 128 + rl;
+        const bool row_valid = r < R;
+        const int t = row_valid ? r / G : 0, g = row_valid ? r % G : 0;
+        const unsigned long long anc = row_valid ? p.tree_anc[(size_t)sg.b * p.T_max + t] : 0ull;
+        const unsigned long long allowed = sg.T >= 64 ? anc : (anc & ((1ull << sg.T) - 1ull));
+        float m_ref = -CUDART_INF_F, l = 0.f;
+
+        for (int j = 0; j < nt; ++j) {
+            const int gt = jt + j;
+            const uint32_t tS = tmem + lane_bits + (gt % P_NSBUF) * 128;
+            int overlap;
+            const int key0 = tile_key0(sg, sg.tile_lo + j, overlap);
+            const bool masked = key0 + BN > sg.L || overlap > 0;
+            mbar_wait(bar(lay.S + gt % P_NSBUF), (gt / P_NSBUF) & 1, abort_flag, status);
+            tc_fence_after();
+            uint32_t x[4][32];
+#pragma unroll
+            for (int c = 0; c < 4; ++c) tmem_ld32(tS + c * 32, x[c]);
+            tmem_wait_ld();
+            if (masked) {
+                // per 32-column chunk one word of allowed columns: cached keys not yet covered, ancestors in the tree
+#pragma unroll
+                for (int c = 0; c < 4; ++c) {
+                    const int u0 = key0 + c * 32 - sg.L;         // tree index of the chunk's first column
+                    uint32_t w;
+                    if (u0 >= 64) w = 0u;
+                    else if (u0 >= 0) w = (uint32_t)(allowed >> u0);
+                    else if (u0 <= -32) w = 0xffffffffu;
+                    else w = (uint32_t)((allowed << (-u0)) | ((1ull << (-u0)) - 1ull));
+                    const int cov = overlap - c * 32;            // columns of this chunk that the previous tile covered
+                    if (cov >= 32) w = 0u;
+                    else if (cov > 0) w &= ~((1u << cov) - 1u);
+#pragma unroll
+                    for (int q = 0; q < 32; ++q)
+                        if (!((w >> q) & 1u)) x[c][q] = 0xff800000u;   // -inf
+                }
+            }
+            float mx0 = -CUDART_INF_F, mx1 = -CUDART_INF_F;
+#pragma unroll
+            for (int c = 0; c < 4; ++c)
+#pragma unroll
+                for (int q = 0; q < 32; q += 4) {
+                    mx0 = fmax3(mx0, __uint_as_float(x[c][q]), __uint_as_float(x[c][q + 1]));
+                    mx1 = fmax3(mx1, __uint_as_float(x[c][q + 2]), __uint_as_float(x[c][q + 3]));
+                }
+            const float mx = fmaxf(mx0, mx1);
+            // reference maximum: move it only when the scores outgrow it by more than the threshold
+            if (mx != -CUDART_INF_F && (m_ref == -CUDART_INF_F || (mx - m_ref) * sl2 > kRescaleThreshold)) {
+                if (m_ref != -CUDART_INF_F) {
+                    // O must hold every earlier tile of the segment before it is rescaled (j > 0 here)
+                    mbar_wait(bar(lay.pv_done + (gt - 1) % lay.pv_mod), ((gt - 1) / lay.pv_mod) & 1, abort_flag, status);
+                    tc_fence_after();
+                    const float alpha = exp2f((m_ref - mx) * sl2);
+                    l *= alpha;
+#pragma unroll 1
+                    for (int c = 0; c < 4; ++c) {
+                        uint32_t o[32];
+                        tmem_ld32(tO + c * 32, o);
+                        tmem_wait_ld();
+#pragma unroll
+                        for (int q = 0; q < 32; ++q) o[q] = __float_as_uint(__uint_as_float(o[q]) * alpha);
+                        tmem_st32(tO + c * 32, o);
+                    }
+                    tmem_wait_st();
+                }
+                m_ref = mx;
+            }
+            const float off = m_ref == -CUDART_INF_F ? 0.f : m_ref * sl2;
+            // P = 2^(s*scale*log2e - off) as bf16 into the first 64 columns of this S buffer
+            float sum0 = 0.f, sum1 = 0.f;
+#pragma unroll
+            for (int c = 0; c < 4; ++c) {
+                uint32_t pk[16];
+#pragma unroll
+                for (int q = 0; q < 32; q += 2) {
+                    const float p0 = ex2(fmaf(__uint_as_float(x[c][q]), sl2, -off));
+                    const float p1 = ex2(fmaf(__uint_as_float(x[c][q + 1]), sl2, -off));
+                    sum0 += p0;
+                    sum1 += p1;
+                    pk[q >> 1] = pack_bf16(p0, p1);
+                }
+                tmem_st16(tS + c * 16, pk);
+            }
+            l += sum0 + sum1;
+            tmem_wait_st();
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) {                               // one arrival per warp
+                if (lay.remote) mbar_arrive_remote(map_to_cta(bar(lay.P + gt % P_NSBUF), 0u));
+                else mbar_arrive(bar(lay.P + gt % P_NSBUF));
+            }
+        }
+
+        // ---- results of the segment: O row from TMEM, final rows or a partial
+        mbar_wait(bar(lay.O), n_seg_done & 1, abort_flag, status);     // every MMA of the segment is complete
+        tc_fence_after();
+        if (sg.slot < 0) {
+            const float inv = l > 0.f ? 1.f / l : 0.f;
+            __nv_bfloat16* orow = reinterpret_cast<__nv_bfloat16*>(p.O) + (size_t)sg.b * p.o_stride_b + (size_t)t * p.o_stride_t +
+                                  (size_t)(sg.h * G + g) * p.o_stride_h;
+#pragma unroll 1
+            for (int c = 0; c < 4; ++c) {
+                uint32_t v[32];
+                tmem_ld32(tO + c * 32, v);
+                tmem_wait_ld();
+                if (row_valid) {
+#pragma unroll
+                    for (int q = 0; q < 4; ++q) {      // 16-byte stores: O strides are only guaranteed 16-byte aligned
+                        uint4 o4;
+                        o4.x = pack_bf16(__uint_as_float(v[q * 8 + 0]) * inv, __uint_as_float(v[q * 8 + 1]) * inv);
+                        o4.y = pack_bf16(__uint_as_float(v[q * 8 + 2]) * inv, __uint_as_float(v[q * 8 + 3]) * inv);
+                        o4.z = pack_bf16(__uint_as_float(v[q * 8 + 4]) * inv, __uint_as_float(v[q * 8 + 5]) * inv);
+                        o4.w = pack_bf16(__uint_as_float(v[q * 8 + 6]) * inv, __uint_as_float(v[q * 8 + 7]) * inv);
+                        *reinterpret_cast<uint4*>(orow + c * 32 + q * 8) = o4;
+                    }
+                }
+            }
+            if (row_valid && p.LSE)
+                p.LSE[((size_t)sg.b * p.Hq + sg.h * G + g) * p.T_max + t] =
+                    l > 0.f ? (m_ref * sl2 + log2f(l)) * kLn2 : -CUDART_INF_F;
+        } else {
+            float* base = a.partial + (size_t)sg.slot * SLOT_FLOATS;
+            const int lr = (int)rank * 128 + rl;
+            float* prow = base + (size_t)lr * D;
+#pragma unroll 1
+            for (int c = 0; c < 4; ++c) {
+                uint32_t v[32];
+                tmem_ld32(tO + c * 32, v);
+                tmem_wait_ld();
+#pragma unroll
+                for (int q = 0; q < 4; ++q)      // 32-byte stores: every store fills a whole sector
+                    st_global_v8(prow + c * 32 + q * 8, v[q * 8], v[q * 8 + 1], v[q * 8 + 2], v[q * 8 + 3], v[q * 8 + 4],
+                                 v[q * 8 + 5], v[q * 8 + 6], v[q * 8 + 7]);
+            }
+            base[BR * D + lr] = m_ref == -CUDART_INF_F ? -CUDART_INF_F : m_ref * sl2;
+            base[BR * D + BR + lr] = l;
+        }
+        tc_fence_before();                 // TMEM reads done before the next segment's MMAs are released
+        jt += nt;
+        ++n_seg_done;
+    }
+}
+
 __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(P_NTHREADS, 1)
 attn_tc_pair_kernel(const __grid_constant__ CUtensorMap kmap, const __grid_constant__ CUtensorMap vmap, const __grid_constant__ CUtensorMap qmap,
                     TcArgs a, unsigned* status) {
@@ -1067,7 +1245,7 @@ attn_tc_pair_kernel(const __grid_constant__ CUtensorMap kmap, const __grid_const
     if (threadIdx.x == 0) {
         for (int i = 0; i < P_NSLOT; ++i) { mbar_init(bar(PB_FULL + i), 1); mbar_init(bar(PB_EMPTY + i), 1); }
         for (int i = 0; i < P_NSBUF; ++i) { mbar_init(bar(PB_S + i), 1); mbar_init(bar(PB_P + i), 8); }      // 4 softmax warps in each CTA
-        mbar_init(bar(PB_Q), a.q_tma ? 2 : 4);      // by TMA: one arrival per CTA; staged by threads: one per stager warp
+        mbar_init(bar(PB_Q), 2);                    // one arrival per CTA (with the byte count when Q goes by TMA)
         mbar_init(bar(PB_O), 1);
         mbar_init(bar(PB_QFREE), 1);
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -1082,15 +1260,6 @@ attn_tc_pair_kernel(const __grid_constant__ CUtensorMap kmap, const __grid_const
     tc_fence_after();
     const uint32_t tmem = ctrl.tmem;
 
-    // first key and number of already-covered columns of tile t of an item
-    auto tile_key0 = [&](const Seg& sg, int t, int& overlap) {
-        const int n_keys = sg.L + sg.T;
-        const int ntiles = (n_keys + BN - 1) / BN;
-        overlap = 0;
-        if (t < ntiles - 1) return t * BN;
-        overlap = ntiles * BN - n_keys;
-        return n_keys - BN;
-    };
 
     // running counters that persist across segments and rounds (each role keeps its own copy)
     int jt = 0;                // tiles issued / processed so far: ring slot and use, S and P barrier phases
@@ -1120,16 +1289,22 @@ attn_tc_pair_kernel(const __grid_constant__ CUtensorMap kmap, const __grid_const
                 }
             }
         } else if (warp == 1) {
-            // =============================== MMA issuer (leader only) ===============================
+            // =============================== Q K^T issuer (leader only) ===============================
+            // Two threads issue the MMAs: one thread cannot issue them as fast as the tensor pipe executes them
+            // (measured: the pipe was active 35 % of the time with a single issuer).  This one runs ahead and
+            // fills the three score buffers; the other one (warp 3) consumes P.  They meet at the slot-free
+            // barrier: buffer g % 3 may be overwritten once P V of tile g - 3 is complete.
             if (lane == 0 && rank == 0) {
                 for (int si = 0; si < nseg; ++si) {
                     const Seg sg = plan.seg[si];
                     const int nt = sg.tile_hi - sg.tile_lo;
-                    // S[buffer gt % 3] = Q K^T with the K half-tiles of ring slot gt % P_NSLOT (V of the same tile lands with it)
-                    // `landed`: the slot's barrier was already seen complete by an earlier test
-                    auto issue_qk = [&](int gt, bool landed) {
-                        if (!landed) mbar_wait(bar(PB_FULL + gt % P_NSLOT), (gt / P_NSLOT) & 1, abort_flag, status);
+                    mbar_wait_cluster(bar(PB_Q), n_seg_done & 1, abort_flag, status);   // Q of this segment is in place in both CTAs
+                    for (int j = 0; j < nt; ++j) {
+                        const int gt = jt + j;
+                        mbar_wait(bar(PB_FULL + gt % P_NSLOT), (gt / P_NSLOT) & 1, abort_flag, status);
+                        if (gt >= P_NSBUF) mbar_wait(bar(PB_EMPTY + (gt - P_NSBUF) % P_NSLOT), ((gt - P_NSBUF) / P_NSLOT) & 1, abort_flag, status);
                         tc_fence_after();
+                        // S[buffer gt % 3] = Q K^T with the K half-tiles of ring slot gt % P_NSLOT (V of the same tile lands with it)
                         const uint32_t sK16 = (sRing + (gt % P_NSLOT) * P_SLOT_BYTES) >> 4;
                         const uint32_t sQ16 = sQ >> 4;
 #pragma unroll
@@ -1139,24 +1314,21 @@ attn_tc_pair_kernel(const __grid_constant__ CUtensorMap kmap, const __grid_const
                             mma_pair_ss(tmem + (gt % P_NSBUF) * 128, smem_desc(kDescKMajor, sQ16 + offQ), smem_desc(kDescKMajor, sK16 + offK), kIdescPairQK, k > 0);
                         }
                         tc_commit_pair(bar(PB_S + gt % P_NSBUF));
-                    };
-                    mbar_wait_cluster(bar(PB_Q), n_seg_done & 1, abort_flag, status);   // Q of this segment is in place in both CTAs
-                    // Q K^T runs two tiles ahead of P V: with three score buffers S(j+2) does not wait for P(j) to be consumed.
-                    // Every barrier is tested one step early, so that a wait that is already satisfied costs no round trip
-                    // between two runs of MMAs.
-                    issue_qk(jt, false);
-                    if (nt > 1) issue_qk(jt + 1, false);
-                    if (nt <= 2) tc_commit_pair(bar(PB_QFREE));      // the segment's last Q K^T is in the pipe
-                    bool k_landed = nt > 2 && mbar_test(bar(PB_FULL + (jt + 2) % P_NSLOT), ((jt + 2) / P_NSLOT) & 1);
+                    }
+                    tc_commit_pair(bar(PB_QFREE));                // the segment's last Q K^T is in the pipe
+                    jt += nt;
+                    ++n_seg_done;
+                }
+            }
+        } else if (warp == 3) {
+            // =============================== P V issuer (leader only) ===============================
+            if (lane == 0 && rank == 0) {
+                for (int si = 0; si < nseg; ++si) {
+                    const Seg sg = plan.seg[si];
+                    const int nt = sg.tile_hi - sg.tile_lo;
                     for (int j = 0; j < nt; ++j) {
                         const int gt = jt + j;
-                        const bool p_there = mbar_test(bar(PB_P + gt % P_NSBUF), (gt / P_NSBUF) & 1);
-                        if (j + 2 < nt) {
-                            issue_qk(gt + 2, k_landed);
-                            if (j + 3 == nt) tc_commit_pair(bar(PB_QFREE));
-                        }
-                        if (!p_there) mbar_wait_cluster(bar(PB_P + gt % P_NSBUF), (gt / P_NSBUF) & 1, abort_flag, status);
-                        k_landed = j + 3 < nt && mbar_test(bar(PB_FULL + (gt + 3) % P_NSLOT), ((gt + 3) / P_NSLOT) & 1);
+                        mbar_wait_cluster(bar(PB_P + gt % P_NSBUF), (gt / P_NSBUF) & 1, abort_flag, status);
                         tc_fence_after();
                         const uint32_t sV16 = (sRing + (gt % P_NSLOT) * P_SLOT_BYTES + P_HALF_TILE) >> 4;
 #pragma unroll
@@ -1167,11 +1339,10 @@ attn_tc_pair_kernel(const __grid_constant__ CUtensorMap kmap, const __grid_const
                     }
                     tc_commit_pair(bar(PB_O));
                     jt += nt;
-                    ++n_seg_done;
                 }
             }
-        } else if (warp == 2 || warp == 3) {
-            // =============================== Q loaders (both CTAs) ===============================
+        } else if (warp == 2) {
+            // =============================== Q loader (both CTAs) ===============================
             for (int si = 0; si < nseg; ++si) {
                 const Seg sg = plan.seg[si];
                 // Q may be overwritten once the previous segment's last Q K^T is complete
@@ -1179,30 +1350,30 @@ attn_tc_pair_kernel(const __grid_constant__ CUtensorMap kmap, const __grid_const
                 const uint32_t qb = leader_bar(PB_Q);
                 const int row0 = sg.rb * BR + (int)rank * 128;
                 if (a.q_tma) {
-                    if (warp == 2 && lane == 0) {
+                    if (lane == 0) {
                         if (rank == 0) mbar_expect_tx(bar(PB_Q), 2 * TILE_BYTES);           // 128 rows in each CTA
                         else mbar_arrive_remote(qb);
                         tma_pair_5d(sQ, &qmap, 0, 0, row0 / G, sg.h, sg.b, qb);
                         tma_pair_5d(sQ + HALF_BYTES, &qmap, 64, 0, row0 / G, sg.h, sg.b, qb);
                     }
                 } else {
-                    // 16-byte asynchronous copies by the 64 threads, K-major with the 128-byte swizzle; rows past the tree read as zero
-                    const int tid = threadIdx.x - 64;
+                    // 16-byte asynchronous copies by the warp, K-major with the 128-byte swizzle; rows past the tree read as zero
+                    const int tid = lane;
                     const int R = sg.T * G;
                     const __nv_bfloat16* Qg = reinterpret_cast<const __nv_bfloat16*>(p.Q) + (size_t)sg.b * p.q_stride_b +
                                               (size_t)sg.h * G * p.q_stride_h;
                     const int ch = tid & 15;
                     int r = row0 + (tid >> 4);
                     int g = r % G;
-                    const int dt = 4 / G, dg = 4 - dt * G;                 // four rows per pass
+                    const int dt = 2 / G, dg = 2 - dt * G;                 // two rows per pass
                     const __nv_bfloat16* src_t = Qg + (size_t)(r / G) * p.q_stride_t + ch * 8;
                     const size_t inc_t = (size_t)dt * p.q_stride_t;
-                    for (int qr = tid >> 4; qr < 128; qr += 4) {
+                    for (int qr = tid >> 4; qr < 128; qr += 2) {
                         const bool valid = r < R;
                         const __nv_bfloat16* src = valid ? src_t + (size_t)g * p.q_stride_h : Qg;
                         const uint32_t dst = sQ + (ch >> 3) * HALF_BYTES + qr * 128 + (((ch & 7) ^ (qr & 7)) << 4);
                         asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"(dst), "l"(src), "r"(valid ? 16 : 0) : "memory");
-                        r += 4;
+                        r += 2;
                         g += dg;
                         src_t += inc_t;
                         if (g >= G) { g -= G; src_t += p.q_stride_t; }
@@ -1216,157 +1387,8 @@ attn_tc_pair_kernel(const __grid_constant__ CUtensorMap kmap, const __grid_const
             }
         } else if (warp >= 4) {
             // =============================== softmax, results (both CTAs) ===============================
-            const int rl = ((warp & 3) << 5) + lane;            // row inside this CTA's block = TMEM lane
-            const uint32_t lane_bits = (uint32_t)((warp & 3) << 5) << 16;
-            const uint32_t tO = tmem + lane_bits + P_NSBUF * 128;
-            const float sl2 = p.scale * kLog2e;
-            for (int si = 0; si < nseg; ++si) {
-                const Seg sg = plan.seg[si];
-                const int nt = sg.tile_hi - sg.tile_lo;
-                const int R = sg.T * G;
-                const int r = sg.rb * BR + (int)rank * 128 + rl;
-                const bool row_valid = r < R;
-                const int t = row_valid ? r / G : 0, g = row_valid ? r % G : 0;
-                const unsigned long long anc = row_valid ? p.tree_anc[(size_t)sg.b * p.T_max + t] : 0ull;
-                const unsigned long long allowed = sg.T >= 64 ? anc : (anc & ((1ull << sg.T) - 1ull));
-                float m_ref = -CUDART_INF_F, l = 0.f;
-
-                for (int j = 0; j < nt; ++j) {
-                    const int gt = jt + j;
-                    const uint32_t tS = tmem + lane_bits + (gt % P_NSBUF) * 128;
-                    int overlap;
-                    const int key0 = tile_key0(sg, sg.tile_lo + j, overlap);
-                    const bool masked = key0 + BN > sg.L || overlap > 0;
-                    mbar_wait(bar(PB_S + gt % P_NSBUF), (gt / P_NSBUF) & 1, abort_flag, status);
-                    tc_fence_after();
-                    PSTAMP(threadIdx.x == 128 && gt >= 40 && gt < 48, 300 + (gt - 40) * 4);
-                    uint32_t x[4][32];
-#pragma unroll
-                    for (int c = 0; c < 4; ++c) tmem_ld32(tS + c * 32, x[c]);
-                    tmem_wait_ld();
-                    if (masked) {
-                        // per 32-column chunk one word of allowed columns: cached keys not yet covered, ancestors in the tree
-#pragma unroll
-                        for (int c = 0; c < 4; ++c) {
-                            const int u0 = key0 + c * 32 - sg.L;         // tree index of the chunk's first column
-                            uint32_t w;
-                            if (u0 >= 64) w = 0u;
-                            else if (u0 >= 0) w = (uint32_t)(allowed >> u0);
-                            else if (u0 <= -32) w = 0xffffffffu;
-                            else w = (uint32_t)((allowed << (-u0)) | ((1ull << (-u0)) - 1ull));
-                            const int cov = overlap - c * 32;            // columns of this chunk that the previous tile covered
-                            if (cov >= 32) w = 0u;
-                            else if (cov > 0) w &= ~((1u << cov) - 1u);
-#pragma unroll
-                            for (int q = 0; q < 32; ++q)
-                                if (!((w >> q) & 1u)) x[c][q] = 0xff800000u;   // -inf
-                        }
-                    }
-                    float mx0 = -CUDART_INF_F, mx1 = -CUDART_INF_F;
-#pragma unroll
-                    for (int c = 0; c < 4; ++c)
-#pragma unroll
-                        for (int q = 0; q < 32; q += 4) {
-                            mx0 = fmax3(mx0, __uint_as_float(x[c][q]), __uint_as_float(x[c][q + 1]));
-                            mx1 = fmax3(mx1, __uint_as_float(x[c][q + 2]), __uint_as_float(x[c][q + 3]));
-                        }
-                    const float mx = fmaxf(mx0, mx1);
-                    PSTAMP(threadIdx.x == 128 && gt >= 40 && gt < 48, 301 + (gt - 40) * 4);
-                    // reference maximum: move it only when the scores outgrow it by more than the threshold
-                    if (mx != -CUDART_INF_F && (m_ref == -CUDART_INF_F || (mx - m_ref) * sl2 > kRescaleThreshold)) {
-                        if (m_ref != -CUDART_INF_F) {
-                            // O must hold every earlier tile of the segment before it is rescaled (j > 0 here)
-                            mbar_wait(bar(PB_EMPTY + (gt - 1) % P_NSLOT), ((gt - 1) / P_NSLOT) & 1, abort_flag, status);
-                            tc_fence_after();
-                            const float alpha = exp2f((m_ref - mx) * sl2);
-                            l *= alpha;
-#pragma unroll 1
-                            for (int c = 0; c < 4; ++c) {
-                                uint32_t o[32];
-                                tmem_ld32(tO + c * 32, o);
-                                tmem_wait_ld();
-#pragma unroll
-                                for (int q = 0; q < 32; ++q) o[q] = __float_as_uint(__uint_as_float(o[q]) * alpha);
-                                tmem_st32(tO + c * 32, o);
-                            }
-                            tmem_wait_st();
-                        }
-                        m_ref = mx;
-                    }
-                    const float off = m_ref == -CUDART_INF_F ? 0.f : m_ref * sl2;
-                    // P = 2^(s*scale*log2e - off) as bf16 into the first 64 columns of this S buffer
-                    float sum0 = 0.f, sum1 = 0.f;
-#pragma unroll
-                    for (int c = 0; c < 4; ++c) {
-                        uint32_t pk[16];
-#pragma unroll
-                        for (int q = 0; q < 32; q += 2) {
-                            const float p0 = ex2(fmaf(__uint_as_float(x[c][q]), sl2, -off));
-                            const float p1 = ex2(fmaf(__uint_as_float(x[c][q + 1]), sl2, -off));
-                            sum0 += p0;
-                            sum1 += p1;
-                            pk[q >> 1] = pack_bf16(p0, p1);
-                        }
-                        tmem_st16(tS + c * 16, pk);
-                    }
-                    l += sum0 + sum1;
-                    PSTAMP(threadIdx.x == 128 && gt >= 40 && gt < 48, 380 + (gt - 40) * 2);
-                    tmem_wait_st();
-                    PSTAMP(threadIdx.x == 128 && gt >= 40 && gt < 48, 381 + (gt - 40) * 2);
-                    tc_fence_before();
-                    __syncwarp();
-                    if (lane == 0) mbar_arrive_remote(leader_bar(PB_P + gt % P_NSBUF));       // one arrival per warp
-                    PSTAMP(threadIdx.x == 128 && gt >= 40 && gt < 48, 302 + (gt - 40) * 4);
-                }
-
-                // ---- results of the segment: O row from TMEM, final rows or a partial
-                mbar_wait(bar(PB_O), n_seg_done & 1, abort_flag, status);     // every MMA of the segment is complete
-                tc_fence_after();
-                if (sg.slot < 0) {
-                    const float inv = l > 0.f ? 1.f / l : 0.f;
-                    __nv_bfloat16* orow = reinterpret_cast<__nv_bfloat16*>(p.O) + (size_t)sg.b * p.o_stride_b + (size_t)t * p.o_stride_t +
-                                          (size_t)(sg.h * G + g) * p.o_stride_h;
-#pragma unroll 1
-                    for (int c = 0; c < 4; ++c) {
-                        uint32_t v[32];
-                        tmem_ld32(tO + c * 32, v);
-                        tmem_wait_ld();
-                        if (row_valid) {
-#pragma unroll
-                            for (int q = 0; q < 4; ++q) {      // 16-byte stores: O strides are only guaranteed 16-byte aligned
-                                uint4 o4;
-                                o4.x = pack_bf16(__uint_as_float(v[q * 8 + 0]) * inv, __uint_as_float(v[q * 8 + 1]) * inv);
-                                o4.y = pack_bf16(__uint_as_float(v[q * 8 + 2]) * inv, __uint_as_float(v[q * 8 + 3]) * inv);
-                                o4.z = pack_bf16(__uint_as_float(v[q * 8 + 4]) * inv, __uint_as_float(v[q * 8 + 5]) * inv);
-                                o4.w = pack_bf16(__uint_as_float(v[q * 8 + 6]) * inv, __uint_as_float(v[q * 8 + 7]) * inv);
-                                *reinterpret_cast<uint4*>(orow + c * 32 + q * 8) = o4;
-                            }
-                        }
-                    }
-                    if (row_valid && p.LSE)
-                        p.LSE[((size_t)sg.b * p.Hq + sg.h * G + g) * p.T_max + t] =
-                            l > 0.f ? (m_ref * sl2 + log2f(l)) * kLn2 : -CUDART_INF_F;
-                } else {
-                    float* base = a.partial + (size_t)sg.slot * SLOT_FLOATS;
-                    const int lr = (int)rank * 128 + rl;
-                    float* prow = base + (size_t)lr * D;
-#pragma unroll 1
-                    for (int c = 0; c < 4; ++c) {
-                        uint32_t v[32];
-                        tmem_ld32(tO + c * 32, v);
-                        tmem_wait_ld();
-#pragma unroll
-                        for (int q = 0; q < 4; ++q)      // 32-byte stores: every store fills a whole sector
-                            st_global_v8(prow + c * 32 + q * 8, v[q * 8], v[q * 8 + 1], v[q * 8 + 2], v[q * 8 + 3], v[q * 8 + 4],
-                                         v[q * 8 + 5], v[q * 8 + 6], v[q * 8 + 7]);
-                    }
-                    base[BR * D + lr] = m_ref == -CUDART_INF_F ? -CUDART_INF_F : m_ref * sl2;
-                    base[BR * D + BR + lr] = l;
-                }
-                tc_fence_before();                 // TMEM reads done before the next segment's MMAs are released
-                jt += nt;
-                ++n_seg_done;
-            }
+            const SoftmaxBars lay = {PB_S, PB_P, PB_O, PB_EMPTY, P_NSLOT, true};
+            softmax_rows(a, plan, lay, bar0, tmem, (int)rank, jt, n_seg_done, abort_flag, status);
         }
 
         // ---- next round (only batches with very many short sequences need more than one)
