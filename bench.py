@@ -318,7 +318,7 @@ def main():
     ap.add_argument("--warmup", type=int, default=10)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default=DEFAULT_WORKLOAD, choices=sorted(WORKLOADS))
-    ap.add_argument("--variant", default="auto", choices=["auto", "mma", "tc", "tc1", "tc2"])
+    ap.add_argument("--variant", default="auto", choices=["auto", "mma", "tc", "tc1", "tc2", "tc3"])
     ap.add_argument("--no-extra", action="store_true", help="skip the other configurations' lines")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     args = ap.parse_args()
@@ -328,7 +328,7 @@ def main():
         return
 
     from paper_2605_20104_b200 import binding as G
-    variant = {"auto": G.ATTN_AUTO, "mma": G.ATTN_MMA_SYNC, "tc": G.ATTN_TCGEN05, "tc1": G.ATTN_TCGEN05_1SM, "tc2": G.ATTN_TCGEN05_2SM}[args.variant]
+    variant = {"auto": G.ATTN_AUTO, "mma": G.ATTN_MMA_SYNC, "tc": G.ATTN_TCGEN05, "tc1": G.ATTN_TCGEN05_1SM, "tc2": G.ATTN_TCGEN05_2SM, "tc3": G.ATTN_TCGEN05_L2PAIR}[args.variant]
     world = int(os.environ.get("WORLD_SIZE", "1"))
     rank = int(os.environ.get("RANK", "0"))
     local = int(os.environ.get("LOCAL_RANK", "0"))

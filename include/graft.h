@@ -81,7 +81,8 @@ enum {
     GRAFT_ATTN_MMA_SYNC = 1,   /* register-tile kernel (any supported shape; the low-row path)    */
     GRAFT_ATTN_TCGEN05 = 2,    /* TMA + tcgen05/TMEM kernels (d = 128): one of the two below        */
     GRAFT_ATTN_TCGEN05_1SM = 3,/* ... one CTA per SM holds both 128-row blocks of an item           */
-    GRAFT_ATTN_TCGEN05_2SM = 4 /* ... a pair of SMs shares every tile                              */
+    GRAFT_ATTN_TCGEN05_2SM = 4,/* ... a pair of SMs shares every tile (two-SM MMAs)                 */
+    GRAFT_ATTN_TCGEN05_L2PAIR = 5 /* ... one 128-row block per SM, partner SMs share tiles through L2 */
 };
 
 /* ---- context --------------------------------------------------------------------------------- */

@@ -25,7 +25,7 @@ OK, ERR_INVALID_ARG, ERR_UNSUPPORTED, ERR_WORKSPACE_TOO_SMALL, ERR_CUDA, ERR_SCR
 FLAG_BAD_SIZE, FLAG_BAD_PARENT, FLAG_BAD_TOKEN, FLAG_ORPHAN = 1, 2, 4, 8
 FLAG_BUDGET, FLAG_BAD_TEMPLATE, FLAG_NAN_SCORE, FLAG_BAD_PATH, FLAG_WAIT_TIMEOUT, FLAG_INTERNAL = 16, 32, 64, 128, 256, 512
 PRUNE_NONE, PRUNE_TOPK, PRUNE_GATED, PRUNE_NODE = 0, 1, 2, 3
-ATTN_AUTO, ATTN_MMA_SYNC, ATTN_TCGEN05, ATTN_TCGEN05_1SM, ATTN_TCGEN05_2SM = 0, 1, 2, 3, 4
+ATTN_AUTO, ATTN_MMA_SYNC, ATTN_TCGEN05, ATTN_TCGEN05_1SM, ATTN_TCGEN05_2SM, ATTN_TCGEN05_L2PAIR = 0, 1, 2, 3, 4, 5
 
 EXPORTS = ("graft_workspace_bytes", "graft_create", "graft_destroy", "graft_status_string", "graft_device_status",
            "graft_build_tree", "graft_tree_verify_attn", "graft_accept", "graft_compact_kv",

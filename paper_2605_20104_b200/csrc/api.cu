@@ -90,6 +90,9 @@ extern "C" int graft_tree_verify_attn(graft_ctx* ctx, const graft_attn_params* p
         case GRAFT_ATTN_TCGEN05_2SM:
             if (!graft_attn_tc_pair_supported(ctx, p)) return GRAFT_ERR_UNSUPPORTED;
             return graft_attn_tc_launch(ctx, p, s, 1);
+        case GRAFT_ATTN_TCGEN05_L2PAIR:
+            if (!graft_attn_tc_supported(ctx, p)) return GRAFT_ERR_UNSUPPORTED;
+            return graft_attn_tc_launch(ctx, p, s, 2);
         case GRAFT_ATTN_AUTO:
             if (graft_attn_tc_supported(ctx, p)) return graft_attn_tc_launch(ctx, p, s);
             return graft_attn_mma_launch(ctx, p, s);

@@ -1048,12 +1048,17 @@ __device__ __forceinline__ int tile_key0(const Seg& sg, int t, int& overlap) {
 }
 
 __device__ __forceinline__ void softmax_rows(const TcArgs& a, const Plan& plan, const SoftmaxBars lay, uint32_t bar0, uint32_t tmem, int rank,
-                                             int& jt, int& n_seg_done, volatile int* abort_flag, unsigned* status) {
+                                             int& jt, int& n_seg_done, volatile int* abort_flag, unsigned* status, volatile int* prof = nullptr) {
     const graft_attn_params& p = a.p;
     const int G = a.G;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int nseg = plan.nseg;
     auto bar = [&](int i) { return bar0 + 8u * (uint32_t)i; };
+#ifdef GRAFT_TC_EXPERIMENTS
+#define SSTAMP(k) do { if (prof && threadIdx.x == 128 && gt >= 40 && gt < 48) prof[(gt - 40) * 4 + (k)] = (int)clock(); } while (0)
+#else
+#define SSTAMP(k) do { (void)prof; } while (0)
+#endif
     const int rl = ((warp & 3) << 5) + lane;            // row inside this CTA's block = TMEM lane
     const uint32_t lane_bits = (uint32_t)((warp & 3) << 5) << 16;
     const uint32_t tO = tmem + lane_bits + P_NSBUF * 128;
@@ -1075,8 +1080,10 @@ __device__ __forceinline__ void softmax_rows(const TcArgs& a, const Plan& plan, 
             int overlap;
             const int key0 = tile_key0(sg, sg.tile_lo + j, overlap);
             const bool masked = key0 + BN > sg.L || overlap > 0;
+            SSTAMP(0);
             mbar_wait(bar(lay.S + gt % P_NSBUF), (gt / P_NSBUF) & 1, abort_flag, status);
             tc_fence_after();
+            SSTAMP(1);
             uint32_t x[4][32];
 #pragma unroll
             for (int c = 0; c < 4; ++c) tmem_ld32(tS + c * 32, x[c]);
@@ -1147,6 +1154,7 @@ __device__ __forceinline__ void softmax_rows(const TcArgs& a, const Plan& plan, 
             }
             l += sum0 + sum1;
             tmem_wait_st();
+            SSTAMP(2);
             tc_fence_before();
             __syncwarp();
             if (lane == 0) {                               // one arrival per warp
@@ -1417,6 +1425,254 @@ attn_tc_pair_kernel(const __grid_constant__ CUtensorMap kmap, const __grid_const
 }
 
 // ---------------------------------------------------------------------------------------------------
+// the row-block kernel: one 128-row block per CTA, partner CTAs share every tile through L2
+// ---------------------------------------------------------------------------------------------------
+// CTAs 2w and 2w+1 form worker w and walk the same tiles of the same items at the same time; CTA 2w owns rows
+// 0..127 of an item, CTA 2w+1 rows 128..255.  Each fetches the whole K and V tile for itself: the second
+// fetch of a line is an L2 hit (two CTAs streaming the same 2 GiB measured 14.2 TB/s into the SMs at
+// 7.1 TB/s from HBM), so HBM still sees every byte once.  Nothing else couples the partners: no cluster, no
+// shared barrier.  With one row block per SM the MMAs are the one-SM ones (Q K^T from shared memory, P V with
+// P in tensor memory at full rate), three score buffers let Q K^T run ahead of P V, and the two kinds are
+// issued by different threads that meet at the V slot's free barrier (P V of tile g-3 complete).
+constexpr int R_NTHREADS = 256;          // producer, Q K^T issuer, Q loader, P V issuer, four softmax warps
+constexpr int R_NK = 3, R_NV = 3;        // ring slots of one K tile / one V tile
+constexpr int R_SMEM_DYN = kCtrlBytes + TILE_BYTES + (R_NK + R_NV) * TILE_BYTES;      // control, Q (128 rows), rings
+enum { RB_FULLK = 0, RB_EMPTYK = RB_FULLK + R_NK, RB_FULLV = RB_EMPTYK + R_NK, RB_EMPTYV = RB_FULLV + R_NV, RB_S = RB_EMPTYV + R_NV,
+       RB_P = RB_S + P_NSBUF, RB_Q = RB_P + P_NSBUF, RB_O = RB_Q + 1, RB_QFREE = RB_O + 1, RB_COUNT = RB_QFREE + 1 };
+struct RbCtrl {
+    uint64_t bar[RB_COUNT];
+    Plan plan;
+    uint32_t tmem;
+    int abort;
+};
+static_assert(sizeof(RbCtrl) <= kCtrlBytes, "control block too large");
+
+__global__ void __launch_bounds__(R_NTHREADS, 1)
+attn_tc_rb_kernel(const __grid_constant__ CUtensorMap kmap, const __grid_constant__ CUtensorMap vmap, const __grid_constant__ CUtensorMap qmap,
+                  TcArgs a, unsigned* status) {
+    extern __shared__ __align__(1024) unsigned char smem_raw[];
+    RbCtrl& ctrl = *reinterpret_cast<RbCtrl*>(smem_raw);
+    Plan& plan = ctrl.plan;
+    const graft_attn_params& p = a.p;
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int G = a.G;
+    const int rank = (int)(blockIdx.x & 1);           // which 128-row block of an item
+#ifdef GRAFT_TC_EXPERIMENTS
+    volatile int* s_prof = (int)blockIdx.x == a.prof_cta ? reinterpret_cast<volatile int*>(smem_raw + R_SMEM_DYN) : nullptr;
+#define RSTAMP(k) do { if (s_prof && gt >= 40 && gt < 48) s_prof[32 + (gt - 40) * 4 + (k)] = (int)clock(); } while (0)
+#else
+    volatile int* s_prof = nullptr;
+#define RSTAMP(k) do { } while (0)
+#endif
+    const int worker = (int)(blockIdx.x >> 1), nworkers = (int)(gridDim.x >> 1);
+
+    if ((smem_u32(smem_raw) & 1023u) != 0) {          // the tiles would miss their alignment: refuse to run
+        if (threadIdx.x == 0) atomicOr(status, (unsigned)GRAFT_FLAG_INTERNAL);
+        return;
+    }
+    const uint32_t sQ = smem_u32(smem_raw) + kCtrlBytes;
+    const uint32_t sK = sQ + TILE_BYTES;
+    const uint32_t sV = sK + R_NK * TILE_BYTES;
+    const uint32_t bar0 = smem_u32(ctrl.bar);
+    auto bar = [&](int i) { return bar0 + 8u * (uint32_t)i; };
+    volatile int* abort_flag = &ctrl.abort;
+
+    // both CTAs of a worker derive the same plan
+    if (warp == 0) plan_first(a, G, worker, nworkers, blockIdx.x == 0, rank == 0, plan);
+    if (threadIdx.x == 0) ctrl.abort = 0;
+    __syncthreads();
+    if (plan.nseg == 0) return;                       // nothing for this worker (short batch)
+
+    if (threadIdx.x == 0) {
+        for (int i = 0; i < R_NK; ++i) { mbar_init(bar(RB_FULLK + i), 1); mbar_init(bar(RB_EMPTYK + i), 1); }
+        for (int i = 0; i < R_NV; ++i) { mbar_init(bar(RB_FULLV + i), 1); mbar_init(bar(RB_EMPTYV + i), 1); }
+        for (int i = 0; i < P_NSBUF; ++i) { mbar_init(bar(RB_S + i), 1); mbar_init(bar(RB_P + i), 4); }      // 4 softmax warps
+        mbar_init(bar(RB_Q), 1);
+        mbar_init(bar(RB_O), 1);
+        mbar_init(bar(RB_QFREE), 1);
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    if (warp == 1) {
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&ctrl.tmem)), "r"(512u) : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem = ctrl.tmem;
+
+    // running counters that persist across segments and rounds (each role keeps its own copy)
+    int jt = 0;                // tiles issued / processed so far: ring slot and use, S and P barrier phases
+    int n_seg_done = 0;        // segments finished (Q, Q-free and O barrier phases)
+
+    for (;;) {                 // rounds of <= MAXSEG segments
+        const int nseg = plan.nseg;
+
+        if (warp == 0) {
+            // =============================== K/V producer ===============================
+            // order of issue: K(0) K(1) V(0) K(2) V(1) ...: a K tile is wanted two tiles before its V tile
+            if (lane == 0) {
+                int total = 0;
+                for (int si = 0; si < nseg; ++si) total += plan.seg[si].tile_hi - plan.seg[si].tile_lo;
+                // tile number `idx` of this round -> its segment and tile
+                auto locate = [&](int idx, Seg& sg, int& t) {
+                    for (int si = 0; si < nseg; ++si) {
+                        const int n = plan.seg[si].tile_hi - plan.seg[si].tile_lo;
+                        if (idx < n) { sg = plan.seg[si]; t = sg.tile_lo + idx; return; }
+                        idx -= n;
+                    }
+                };
+                auto load = [&](int idx, bool is_v) {
+                    Seg sg;
+                    int t = 0, overlap;
+                    locate(idx, sg, t);
+                    const int key0 = tile_key0(sg, t, overlap);
+                    const int g = jt + idx;              // global tile number
+                    const int nslot = is_v ? R_NV : R_NK;
+                    const int slot = g % nslot, use = g / nslot;
+                    const int full = (is_v ? RB_FULLV : RB_FULLK) + slot, empty = (is_v ? RB_EMPTYV : RB_EMPTYK) + slot;
+                    if (use > 0) mbar_wait(bar(empty), (use - 1) & 1, abort_flag, status);
+                    mbar_expect_tx(bar(full), TILE_BYTES);
+                    const uint32_t dst = (is_v ? sV : sK) + slot * TILE_BYTES;
+                    const CUtensorMap* map = is_v ? &vmap : &kmap;
+                    tma_load_4d(dst, map, 0, key0, sg.h, sg.b, bar(full));
+                    tma_load_4d(dst + HALF_BYTES, map, 64, key0, sg.h, sg.b, bar(full));
+                };
+                for (int i = 0; i <= total; ++i) {
+                    if (i < total) load(i, false);
+                    if (i > 0) load(i - 1, true);
+                }
+                jt += total;
+            }
+        } else if (warp == 1) {
+            // =============================== Q K^T issuer ===============================
+            if (lane == 0) {
+                for (int si = 0; si < nseg; ++si) {
+                    const Seg sg = plan.seg[si];
+                    const int nt = sg.tile_hi - sg.tile_lo;
+                    mbar_wait(bar(RB_Q), n_seg_done & 1, abort_flag, status);           // Q of this segment is in place
+                    for (int j = 0; j < nt; ++j) {
+                        const int gt = jt + j;
+                        RSTAMP(2);
+                        mbar_wait(bar(RB_FULLK + gt % R_NK), (gt / R_NK) & 1, abort_flag, status);
+                        RSTAMP(3);
+                        // buffer gt % 3 held P of tile gt - 3: wait until P V of that tile is complete
+                        if (gt >= P_NSBUF) mbar_wait(bar(RB_EMPTYV + (gt - P_NSBUF) % R_NV), ((gt - P_NSBUF) / R_NV) & 1, abort_flag, status);
+                        tc_fence_after();
+                        const uint32_t sK16 = (sK + (gt % R_NK) * TILE_BYTES) >> 4;
+                        const uint32_t sQ16 = sQ >> 4;
+#pragma unroll
+                        for (int k = 0; k < D / 16; ++k) {
+                            const uint32_t off16 = ((k >> 2) * HALF_BYTES + (k & 3) * 32) >> 4;
+                            mma_ss(tmem + (gt % P_NSBUF) * 128, smem_desc(kDescKMajor, sQ16 + off16), smem_desc(kDescKMajor, sK16 + off16), kIdescQK, k > 0);
+                        }
+                        tc_commit(bar(RB_S + gt % P_NSBUF));
+                        tc_commit(bar(RB_EMPTYK + gt % R_NK));           // K tile fully read
+                    }
+                    tc_commit(bar(RB_QFREE));                           // the segment's last Q K^T is in the pipe
+                    jt += nt;
+                    ++n_seg_done;
+                }
+            }
+        } else if (warp == 3) {
+            // =============================== P V issuer ===============================
+            if (lane == 0) {
+                for (int si = 0; si < nseg; ++si) {
+                    const Seg sg = plan.seg[si];
+                    const int nt = sg.tile_hi - sg.tile_lo;
+                    for (int j = 0; j < nt; ++j) {
+                        const int gt = jt + j;
+                        RSTAMP(0);
+                        mbar_wait(bar(RB_FULLV + gt % R_NV), (gt / R_NV) & 1, abort_flag, status);
+                        mbar_wait(bar(RB_P + gt % P_NSBUF), (gt / P_NSBUF) & 1, abort_flag, status);
+                        RSTAMP(1);
+                        tc_fence_after();
+                        const uint32_t sV16 = (sV + (gt % R_NV) * TILE_BYTES) >> 4;
+#pragma unroll
+                        for (int k = 0; k < BN / 16; ++k)
+                            mma_ts(tmem + P_NSBUF * 128, tmem + (gt % P_NSBUF) * 128 + k * 8, smem_desc(kDescVMajor, sV16 + k * (2048 >> 4)), kIdescPV,
+                                   (j > 0 || k > 0) ? 1u : 0u);
+                        tc_commit(bar(RB_EMPTYV + gt % R_NV));           // V tile fully read, O holds tiles 0..j
+                    }
+                    tc_commit(bar(RB_O));
+                    jt += nt;
+                }
+            }
+        } else if (warp == 2) {
+            // =============================== Q loader ===============================
+            for (int si = 0; si < nseg; ++si) {
+                const Seg sg = plan.seg[si];
+                // Q may be overwritten once the previous segment's last Q K^T is complete
+                if (n_seg_done > 0) mbar_wait(bar(RB_QFREE), (n_seg_done - 1) & 1, abort_flag, status);
+                const int row0 = sg.rb * BR + rank * 128;
+                if (a.q_tma) {
+                    if (lane == 0) {
+                        mbar_expect_tx(bar(RB_Q), TILE_BYTES);
+                        tma_load_5d(sQ, &qmap, 0, 0, row0 / G, sg.h, sg.b, bar(RB_Q));
+                        tma_load_5d(sQ + HALF_BYTES, &qmap, 64, 0, row0 / G, sg.h, sg.b, bar(RB_Q));
+                    }
+                } else {
+                    // 16-byte asynchronous copies by the warp, K-major with the 128-byte swizzle; rows past the tree read as zero
+                    const int R = sg.T * G;
+                    const __nv_bfloat16* Qg = reinterpret_cast<const __nv_bfloat16*>(p.Q) + (size_t)sg.b * p.q_stride_b +
+                                              (size_t)sg.h * G * p.q_stride_h;
+                    const int ch = lane & 15;
+                    int r = row0 + (lane >> 4);
+                    int g = r % G;
+                    const int dt = 2 / G, dg = 2 - dt * G;                 // two rows per pass
+                    const __nv_bfloat16* src_t = Qg + (size_t)(r / G) * p.q_stride_t + ch * 8;
+                    const size_t inc_t = (size_t)dt * p.q_stride_t;
+                    for (int qr = lane >> 4; qr < 128; qr += 2) {
+                        const bool valid = r < R;
+                        const __nv_bfloat16* src = valid ? src_t + (size_t)g * p.q_stride_h : Qg;
+                        const uint32_t dst = sQ + (ch >> 3) * HALF_BYTES + qr * 128 + (((ch & 7) ^ (qr & 7)) << 4);
+                        asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"(dst), "l"(src), "r"(valid ? 16 : 0) : "memory");
+                        r += 2;
+                        g += dg;
+                        src_t += inc_t;
+                        if (g >= G) { g -= G; src_t += p.q_stride_t; }
+                    }
+                    asm volatile("cp.async.wait_all;" ::: "memory");
+                    fence_async_smem();
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(bar(RB_Q));
+                }
+                ++n_seg_done;
+            }
+        } else if (warp >= 4) {
+            // =============================== softmax, results ===============================
+            const SoftmaxBars lay = {RB_S, RB_P, RB_O, RB_EMPTYV, R_NV, false};
+            softmax_rows(a, plan, lay, bar0, tmem, rank, jt, n_seg_done, abort_flag, status, s_prof);
+        }
+
+        // ---- next round (only batches with very many short sequences need more than one)
+        const long long g_next = plan.gnext, g_hi = plan.ghi;
+        if (g_next >= g_hi) break;
+        __syncthreads();
+        if (warp == 0) plan_round(a, G, worker, rank == 0, plan, g_next, g_hi);
+        __syncthreads();
+        if (plan.nseg == 0) break;
+    }
+#ifdef GRAFT_TC_EXPERIMENTS
+    __syncthreads();
+    if (s_prof && threadIdx.x < 64) a.desc[300 + threadIdx.x] = s_prof[threadIdx.x];
+#endif
+
+    // ---- teardown: after a timeout some copies may still be in flight: give them time to land before the
+    // shared memory is handed back; the allocating warp frees the tensor memory once everyone is past its last access
+    if (*abort_flag) {
+        const long long t0 = clock64();
+        while (clock64() - t0 < (1ll << 22)) {}
+    }
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 1) {
+        tc_fence_after();
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(512u) : "memory");
+    }
+}
+
+// ---------------------------------------------------------------------------------------------------
 // merge: one warp per output row of the padded [T_max * G] row space of a (b, h_kv)
 // ---------------------------------------------------------------------------------------------------
 // Rows of an item that was cut across CTAs are merged with  M = max m_i, w_i = 2^(m_i - M),
@@ -1591,6 +1847,7 @@ int graft_attn_tc_init() {
     GRAFT_CHECK_CUDA(cudaFuncSetAttribute(attn_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_DYN));
     // pair kernel: how many 2-CTA clusters fit on the device at once (SMs that cannot be paired stay idle)
     GRAFT_CHECK_CUDA(cudaFuncSetAttribute(attn_tc_pair_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, P_SMEM_DYN + kProfBytes));
+    GRAFT_CHECK_CUDA(cudaFuncSetAttribute(attn_tc_rb_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, R_SMEM_DYN + kProfBytes));
     int dev = 0;
     GRAFT_CHECK_CUDA(cudaGetDevice(&dev));
     if (dev >= 0 && dev < kMaxDevices && g_pair_clusters[dev] == 0) {
@@ -1641,11 +1898,12 @@ size_t graft_attn_tc_ws_bytes(int num_sms, int B, int, int, int d, int) {
     return kDescBytes + cut_bytes(B) + (size_t)num_sms * 2 * SLOT_FLOATS * sizeof(float);
 }
 
-int graft_attn_tc_launch(graft_ctx* ctx, const graft_attn_params* p, cudaStream_t stream, int pair) {
+int graft_attn_tc_launch(graft_ctx* ctx, const graft_attn_params* p, cudaStream_t stream, int which) {
     const int G = p->Hq / p->Hkv;
-    // pair < 0: choose.  The pair kernel measured faster on every benchmark configuration (3 % at 64K context
-    // with 240-row items up to 20 % on batches of short sequences), so it runs wherever clusters of two fit.
-    const bool use_pair = pair > 0 || (pair < 0 && graft_attn_tc_pair_supported(ctx, p));
+    // which: 0 two row blocks per CTA, 1 CTA pairs with two-SM MMAs, 2 one row block per CTA with partners sharing
+    // tiles through L2, < 0 choose
+    if (which < 0) which = 2;
+    const bool use_pair = which == 1, use_rb = which == 2;
     if (use_pair && !graft_attn_tc_pair_supported(ctx, p)) return GRAFT_ERR_UNSUPPORTED;
     CUtensorMap kmap, vmap;
     int rc = make_kv_map(&kmap, p->Kc, p, use_pair ? 64 : BN);
@@ -1673,6 +1931,8 @@ int graft_attn_tc_launch(graft_ctx* ctx, const graft_attn_params* p, cudaStream_
         int pairs = pair_clusters();
         if (pairs > ctx->num_sms / 2) pairs = ctx->num_sms / 2;       // the workspace has two slots per SM
         attn_tc_pair_kernel<<<2 * pairs, P_NTHREADS, P_SMEM_DYN + kProfBytes, stream>>>(kmap, vmap, qmap, a, ctx->status);
+    } else if (use_rb) {
+        attn_tc_rb_kernel<<<ctx->num_sms & ~1, R_NTHREADS, R_SMEM_DYN + kProfBytes, stream>>>(kmap, vmap, qmap, a, ctx->status);
     } else
     attn_tc_kernel<<<grid, NTHREADS, SMEM_DYN, stream>>>(kmap, vmap, qmap, a, ctx->status);
     GRAFT_CHECK_CUDA(cudaGetLastError());

@@ -27,8 +27,9 @@ static inline bool graft_aligned16(const void* p) { return (reinterpret_cast<uin
 int graft_attn_mma_init();   // per device, called by graft_create with the device current
 int graft_attn_tc_init();
 int graft_attn_mma_launch(graft_ctx* ctx, const graft_attn_params* p, cudaStream_t stream);
-// pair: 1 = the two-SM (CTA pair) kernel, 0 = the one-SM kernel, -1 = choose
-int graft_attn_tc_launch(graft_ctx* ctx, const graft_attn_params* p, cudaStream_t stream, int pair = -1);
+// which: 0 = two row blocks per CTA, 1 = CTA pairs with two-SM MMAs, 2 = one row block per CTA (partners share tiles
+// through L2), -1 = choose
+int graft_attn_tc_launch(graft_ctx* ctx, const graft_attn_params* p, cudaStream_t stream, int which = -1);
 bool graft_attn_tc_pair_supported(const graft_ctx* ctx, const graft_attn_params* p);
 bool graft_attn_tc_supported(const graft_ctx* ctx, const graft_attn_params* p);
 size_t graft_attn_mma_ws_bytes(int num_sms, int B, int Hq, int Hkv, int d, int T_max);

@@ -27,14 +27,14 @@ def Step():
     return VerifyStep
 
 
-VARIANTS = ["mma", "auto", "one", "pair"]      # "one"/"pair": the one-SM and the two-SM tcgen05 kernel, forced
+VARIANTS = ["mma", "auto", "one", "pair", "l2pair"]      # the last three: one of the tcgen05 kernels, forced
 
 
 def variant_id(G, name, w=None):
-    if name in ("one", "pair") and w is not None and w.d != 128:
+    if name in ("one", "pair", "l2pair") and w is not None and w.d != 128:
         pytest.skip("the tcgen05 kernels take d = 128 only")
     return {"mma": G.ATTN_MMA_SYNC, "auto": G.ATTN_AUTO, "tc": G.ATTN_TCGEN05, "one": G.ATTN_TCGEN05_1SM,
-            "pair": G.ATTN_TCGEN05_2SM}[name]
+            "pair": G.ATTN_TCGEN05_2SM, "l2pair": G.ATTN_TCGEN05_L2PAIR}[name]
 
 
 def check_tree(vs, tree):
