@@ -1047,6 +1047,190 @@ __device__ __forceinline__ int tile_key0(const Seg& sg, int t, int& overlap) {
     return n_keys - BN;
 }
 
+// ---------------------------------------------------------------------------------------------------
+// softmax of a 128-row block by two warpgroups that split the columns of every tile (row-block kernel)
+// ---------------------------------------------------------------------------------------------------
+// Warps w and w + 4 own the same 32 rows (tensor-memory lanes) and take columns 0..63 and 64..127 of the
+// score tile, so two warps per scheduler keep the exponential unit busy and a row's 64 scores stay in
+// registers between the maximum pass and the exponentials.  The half-row maxima are exchanged through
+// shared memory at a 64-thread named barrier (double-buffered by tile parity), so both halves move the
+// reference maximum at the same tiles; each half keeps its own part of the row sum and writes 64 output columns.
+struct SplitShared {
+    float mx[2][2][128];     // [tile parity][half][row]; the idle parity carries the row sums at the end of a segment
+};
+
+__device__ __forceinline__ void softmax_rows_split(const TcArgs& a, const Plan& plan, const SoftmaxBars lay, uint32_t bar0, uint32_t tmem, int rank,
+                                             SplitShared& sh, int& jt, int& n_seg_done, volatile int* abort_flag, unsigned* status) {
+    const graft_attn_params& p = a.p;
+    const int G = a.G;
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int nseg = plan.nseg;
+    auto bar = [&](int i) { return bar0 + 8u * (uint32_t)i; };
+    const int half = (warp - 4) >> 2;                   // columns 0..63 or 64..127 of the score tile, and of O
+    const int rl = ((warp & 3) << 5) + lane;            // row inside this CTA's block = TMEM lane
+    const int pair_bar = 1 + (warp & 3);                // the two warps that own the same 32 rows
+    auto pair_sync = [&]() { asm volatile("bar.sync %0, 64;" ::"r"(pair_bar) : "memory"); };
+    const uint32_t lane_bits = (uint32_t)((warp & 3) << 5) << 16;
+    const uint32_t tO = tmem + lane_bits + P_NSBUF * 128 + half * 64;      // this thread's 64 output columns
+    const float sl2 = p.scale * kLog2e;
+    for (int si = 0; si < nseg; ++si) {
+        const Seg sg = plan.seg[si];
+        const int nt = sg.tile_hi - sg.tile_lo;
+        const int R = sg.T * G;
+        const int r = sg.rb * BR + (int)rank * 128 + rl;
+        const bool row_valid = r < R;
+        const int t = row_valid ? r / G : 0, g = row_valid ? r % G : 0;
+        const unsigned long long anc = row_valid ? p.tree_anc[(size_t)sg.b * p.T_max + t] : 0ull;
+        const unsigned long long allowed = sg.T >= 64 ? anc : (anc & ((1ull << sg.T) - 1ull));
+        float m_ref = -CUDART_INF_F, l = 0.f;
+
+        for (int j = 0; j < nt; ++j) {
+            const int gt = jt + j;
+            const uint32_t tS = tmem + lane_bits + (gt % P_NSBUF) * 128 + half * 64;      // this thread's 64 score columns
+            const uint32_t tP = tmem + lane_bits + (gt % P_NSBUF) * 128 + half * 32;      // its 64 P values (bf16 pairs)
+            int overlap;
+            const int key0 = tile_key0(sg, sg.tile_lo + j, overlap);
+            const bool masked = key0 + BN > sg.L || overlap > 0;
+            mbar_wait(bar(lay.S + gt % P_NSBUF), (gt / P_NSBUF) & 1, abort_flag, status);
+            tc_fence_after();
+            uint32_t x[2][32];
+#pragma unroll
+            for (int c = 0; c < 2; ++c) tmem_ld32(tS + c * 32, x[c]);
+            tmem_wait_ld();
+            if (masked) {
+                // per 32-column chunk one word of allowed columns: cached keys not yet covered, ancestors in the tree
+#pragma unroll
+                for (int c = 0; c < 2; ++c) {
+                    const int u0 = key0 + (half * 2 + c) * 32 - sg.L;         // tree index of the chunk's first column
+                    uint32_t w;
+                    if (u0 >= 64) w = 0u;
+                    else if (u0 >= 0) w = (uint32_t)(allowed >> u0);
+                    else if (u0 <= -32) w = 0xffffffffu;
+                    else w = (uint32_t)((allowed << (-u0)) | ((1ull << (-u0)) - 1ull));
+                    const int cov = overlap - (half * 2 + c) * 32;            // columns of this chunk that the previous tile covered
+                    if (cov >= 32) w = 0u;
+                    else if (cov > 0) w &= ~((1u << cov) - 1u);
+#pragma unroll
+                    for (int q = 0; q < 32; ++q)
+                        if (!((w >> q) & 1u)) x[c][q] = 0xff800000u;   // -inf
+                }
+            }
+            float mx0 = -CUDART_INF_F, mx1 = -CUDART_INF_F;
+#pragma unroll
+            for (int c = 0; c < 2; ++c)
+#pragma unroll
+                for (int q = 0; q < 32; q += 4) {
+                    mx0 = fmax3(mx0, __uint_as_float(x[c][q]), __uint_as_float(x[c][q + 1]));
+                    mx1 = fmax3(mx1, __uint_as_float(x[c][q + 2]), __uint_as_float(x[c][q + 3]));
+                }
+            float mx = fmaxf(mx0, mx1);
+            sh.mx[gt & 1][half][rl] = mx;
+            pair_sync();                 // also: the partner's scores are in its registers, P may overwrite them
+            mx = fmaxf(mx, sh.mx[gt & 1][half ^ 1][rl]);
+            // reference maximum: move it only when the scores outgrow it by more than the threshold
+            if (mx != -CUDART_INF_F && (m_ref == -CUDART_INF_F || (mx - m_ref) * sl2 > kRescaleThreshold)) {
+                if (m_ref != -CUDART_INF_F) {
+                    // O must hold every earlier tile of the segment before it is rescaled (j > 0 here)
+                    mbar_wait(bar(lay.pv_done + (gt - 1) % lay.pv_mod), ((gt - 1) / lay.pv_mod) & 1, abort_flag, status);
+                    tc_fence_after();
+                    const float alpha = exp2f((m_ref - mx) * sl2);
+                    l *= alpha;
+#pragma unroll 1
+                    for (int c = 0; c < 2; ++c) {
+                        uint32_t o[32];
+                        tmem_ld32(tO + c * 32, o);
+                        tmem_wait_ld();
+#pragma unroll
+                        for (int q = 0; q < 32; ++q) o[q] = __float_as_uint(__uint_as_float(o[q]) * alpha);
+                        tmem_st32(tO + c * 32, o);
+                    }
+                    tmem_wait_st();
+                }
+                m_ref = mx;
+            }
+            const float off = m_ref == -CUDART_INF_F ? 0.f : m_ref * sl2;
+            // P = 2^(s*scale*log2e - off) as bf16 into the first 64 columns of this S buffer
+            float sum0 = 0.f, sum1 = 0.f;
+#pragma unroll
+            for (int c = 0; c < 2; ++c) {
+                uint32_t pk[16];
+#pragma unroll
+                for (int q = 0; q < 32; q += 2) {
+                    const float p0 = ex2(fmaf(__uint_as_float(x[c][q]), sl2, -off));
+                    const float p1 = ex2(fmaf(__uint_as_float(x[c][q + 1]), sl2, -off));
+                    sum0 += p0;
+                    sum1 += p1;
+                    pk[q >> 1] = pack_bf16(p0, p1);
+                }
+                tmem_st16(tP + c * 16, pk);
+            }
+            l += sum0 + sum1;
+            tmem_wait_st();
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) {                               // one arrival per warp
+                if (lay.remote) mbar_arrive_remote(map_to_cta(bar(lay.P + gt % P_NSBUF), 0u));
+                else mbar_arrive(bar(lay.P + gt % P_NSBUF));
+            }
+        }
+
+        // ---- results of the segment: the two halves of the row sum, then 64 O columns each: final rows or a partial
+        const int last = (jt + nt - 1) & 1;          // the exchange buffer of the other parity is idle
+        sh.mx[last ^ 1][half][rl] = l;
+        mbar_wait(bar(lay.O), n_seg_done & 1, abort_flag, status);     // every MMA of the segment is complete
+        tc_fence_after();
+        pair_sync();
+        l += sh.mx[last ^ 1][half ^ 1][rl];
+        if (sg.slot < 0) {
+            const float inv = l > 0.f ? 1.f / l : 0.f;
+            __nv_bfloat16* orow = reinterpret_cast<__nv_bfloat16*>(p.O) + (size_t)sg.b * p.o_stride_b + (size_t)t * p.o_stride_t +
+                                  (size_t)(sg.h * G + g) * p.o_stride_h + half * 64;
+#pragma unroll 1
+            for (int c = 0; c < 2; ++c) {
+                uint32_t v[32];
+                tmem_ld32(tO + c * 32, v);
+                tmem_wait_ld();
+                if (row_valid) {
+#pragma unroll
+                    for (int q = 0; q < 4; ++q) {      // 16-byte stores: O strides are only guaranteed 16-byte aligned
+                        uint4 o4;
+                        o4.x = pack_bf16(__uint_as_float(v[q * 8 + 0]) * inv, __uint_as_float(v[q * 8 + 1]) * inv);
+                        o4.y = pack_bf16(__uint_as_float(v[q * 8 + 2]) * inv, __uint_as_float(v[q * 8 + 3]) * inv);
+                        o4.z = pack_bf16(__uint_as_float(v[q * 8 + 4]) * inv, __uint_as_float(v[q * 8 + 5]) * inv);
+                        o4.w = pack_bf16(__uint_as_float(v[q * 8 + 6]) * inv, __uint_as_float(v[q * 8 + 7]) * inv);
+                        *reinterpret_cast<uint4*>(orow + c * 32 + q * 8) = o4;
+                    }
+                }
+            }
+            if (half == 0 && row_valid && p.LSE)
+                p.LSE[((size_t)sg.b * p.Hq + sg.h * G + g) * p.T_max + t] =
+                    l > 0.f ? (m_ref * sl2 + log2f(l)) * kLn2 : -CUDART_INF_F;
+        } else {
+            float* base = a.partial + (size_t)sg.slot * SLOT_FLOATS;
+            const int lr = (int)rank * 128 + rl;
+            float* prow = base + (size_t)lr * D + half * 64;
+#pragma unroll 1
+            for (int c = 0; c < 2; ++c) {
+                uint32_t v[32];
+                tmem_ld32(tO + c * 32, v);
+                tmem_wait_ld();
+#pragma unroll
+                for (int q = 0; q < 4; ++q)      // 32-byte stores: every store fills a whole sector
+                    st_global_v8(prow + c * 32 + q * 8, v[q * 8], v[q * 8 + 1], v[q * 8 + 2], v[q * 8 + 3], v[q * 8 + 4],
+                                 v[q * 8 + 5], v[q * 8 + 6], v[q * 8 + 7]);
+            }
+            if (half == 0) {
+                base[BR * D + lr] = m_ref == -CUDART_INF_F ? -CUDART_INF_F : m_ref * sl2;
+                base[BR * D + BR + lr] = l;
+            }
+        }
+        tc_fence_before();                 // TMEM reads done before the next segment's MMAs are released
+        pair_sync();                       // the partner has read this segment's sum before the next segment's tiles reuse the buffer
+        jt += nt;
+        ++n_seg_done;
+    }
+}
+
 __device__ __forceinline__ void softmax_rows(const TcArgs& a, const Plan& plan, const SoftmaxBars lay, uint32_t bar0, uint32_t tmem, int rank,
                                              int& jt, int& n_seg_done, volatile int* abort_flag, unsigned* status, volatile int* prof = nullptr) {
     const graft_attn_params& p = a.p;
@@ -1434,9 +1618,9 @@ attn_tc_pair_kernel(const __grid_constant__ CUtensorMap kmap, const __grid_const
 // shared barrier.  With one row block per SM the MMAs are the one-SM ones (Q K^T from shared memory, P V with
 // P in tensor memory at full rate), three score buffers let Q K^T run ahead of P V, and the two kinds are
 // issued by different threads that meet at the V slot's free barrier (P V of tile g-3 complete).
-constexpr int R_NTHREADS = 256;          // producer, Q K^T issuer, Q loader, P V issuer, four softmax warps
+constexpr int R_NTHREADS = 384;          // producer, MMA issuer, Q loader, one idle warp, eight softmax warps
 constexpr int R_NK = 3, R_NV = 3;        // ring slots of one K tile / one V tile
-constexpr int R_SMEM_DYN = kCtrlBytes + TILE_BYTES + (R_NK + R_NV) * TILE_BYTES;      // control, Q (128 rows), rings
+constexpr int R_SMEM_DYN = kCtrlBytes + TILE_BYTES + (R_NK + R_NV) * TILE_BYTES + 2048;   // control, Q (128 rows), rings, softmax exchange: 227 KB
 enum { RB_FULLK = 0, RB_EMPTYK = RB_FULLK + R_NK, RB_FULLV = RB_EMPTYK + R_NK, RB_EMPTYV = RB_FULLV + R_NV, RB_S = RB_EMPTYV + R_NV,
        RB_P = RB_S + P_NSBUF, RB_Q = RB_P + P_NSBUF, RB_O = RB_Q + 1, RB_QFREE = RB_O + 1, RB_COUNT = RB_QFREE + 1 };
 struct RbCtrl {
@@ -1457,13 +1641,6 @@ attn_tc_rb_kernel(const __grid_constant__ CUtensorMap kmap, const __grid_constan
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int G = a.G;
     const int rank = (int)(blockIdx.x & 1);           // which 128-row block of an item
-#ifdef GRAFT_TC_EXPERIMENTS
-    volatile int* s_prof = (int)blockIdx.x == a.prof_cta ? reinterpret_cast<volatile int*>(smem_raw + R_SMEM_DYN) : nullptr;
-#define RSTAMP(k) do { if (s_prof && gt >= 40 && gt < 48) s_prof[32 + (gt - 40) * 4 + (k)] = (int)clock(); } while (0)
-#else
-    volatile int* s_prof = nullptr;
-#define RSTAMP(k) do { } while (0)
-#endif
     const int worker = (int)(blockIdx.x >> 1), nworkers = (int)(gridDim.x >> 1);
 
     if ((smem_u32(smem_raw) & 1023u) != 0) {          // the tiles would miss their alignment: refuse to run
@@ -1486,7 +1663,7 @@ attn_tc_rb_kernel(const __grid_constant__ CUtensorMap kmap, const __grid_constan
     if (threadIdx.x == 0) {
         for (int i = 0; i < R_NK; ++i) { mbar_init(bar(RB_FULLK + i), 1); mbar_init(bar(RB_EMPTYK + i), 1); }
         for (int i = 0; i < R_NV; ++i) { mbar_init(bar(RB_FULLV + i), 1); mbar_init(bar(RB_EMPTYV + i), 1); }
-        for (int i = 0; i < P_NSBUF; ++i) { mbar_init(bar(RB_S + i), 1); mbar_init(bar(RB_P + i), 4); }      // 4 softmax warps
+        for (int i = 0; i < P_NSBUF; ++i) { mbar_init(bar(RB_S + i), 1); mbar_init(bar(RB_P + i), 8); }      // 8 softmax warps
         mbar_init(bar(RB_Q), 1);
         mbar_init(bar(RB_O), 1);
         mbar_init(bar(RB_QFREE), 1);
@@ -1500,6 +1677,7 @@ attn_tc_rb_kernel(const __grid_constant__ CUtensorMap kmap, const __grid_constan
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem = ctrl.tmem;
+    SplitShared& split = *reinterpret_cast<SplitShared*>(smem_raw + kCtrlBytes + TILE_BYTES + (R_NK + R_NV) * TILE_BYTES);
 
     // running counters that persist across segments and rounds (each role keeps its own copy)
     int jt = 0;                // tiles issued / processed so far: ring slot and use, S and P barrier phases
@@ -1545,19 +1723,17 @@ attn_tc_rb_kernel(const __grid_constant__ CUtensorMap kmap, const __grid_constan
                 jt += total;
             }
         } else if (warp == 1) {
-            // =============================== Q K^T issuer ===============================
+            // =============================== MMA issuer ===============================
+            // One thread issues everything, so the tensor pipe keeps its order: Q K^T of tile j+3 goes in right
+            // behind P V of tile j, whose P it overwrites, without a barrier round trip in between.  Up to three
+            // score tiles are ahead of the softmax.
             if (lane == 0) {
                 for (int si = 0; si < nseg; ++si) {
                     const Seg sg = plan.seg[si];
                     const int nt = sg.tile_hi - sg.tile_lo;
-                    mbar_wait(bar(RB_Q), n_seg_done & 1, abort_flag, status);           // Q of this segment is in place
-                    for (int j = 0; j < nt; ++j) {
-                        const int gt = jt + j;
-                        RSTAMP(2);
-                        mbar_wait(bar(RB_FULLK + gt % R_NK), (gt / R_NK) & 1, abort_flag, status);
-                        RSTAMP(3);
-                        // buffer gt % 3 held P of tile gt - 3: wait until P V of that tile is complete
-                        if (gt >= P_NSBUF) mbar_wait(bar(RB_EMPTYV + (gt - P_NSBUF) % R_NV), ((gt - P_NSBUF) / R_NV) & 1, abort_flag, status);
+                    // `landed`: the K slot's barrier was already seen complete by an earlier test
+                    auto issue_qk = [&](int gt, bool landed) {
+                        if (!landed) mbar_wait(bar(RB_FULLK + gt % R_NK), (gt / R_NK) & 1, abort_flag, status);
                         tc_fence_after();
                         const uint32_t sK16 = (sK + (gt % R_NK) * TILE_BYTES) >> 4;
                         const uint32_t sQ16 = sQ >> 4;
@@ -1568,24 +1744,18 @@ attn_tc_rb_kernel(const __grid_constant__ CUtensorMap kmap, const __grid_constan
                         }
                         tc_commit(bar(RB_S + gt % P_NSBUF));
                         tc_commit(bar(RB_EMPTYK + gt % R_NK));           // K tile fully read
-                    }
-                    tc_commit(bar(RB_QFREE));                           // the segment's last Q K^T is in the pipe
-                    jt += nt;
-                    ++n_seg_done;
-                }
-            }
-        } else if (warp == 3) {
-            // =============================== P V issuer ===============================
-            if (lane == 0) {
-                for (int si = 0; si < nseg; ++si) {
-                    const Seg sg = plan.seg[si];
-                    const int nt = sg.tile_hi - sg.tile_lo;
+                    };
+                    mbar_wait(bar(RB_Q), n_seg_done & 1, abort_flag, status);           // Q of this segment is in place
+                    for (int j = 0; j < P_NSBUF && j < nt; ++j) issue_qk(jt + j, false);
+                    if (nt <= P_NSBUF) tc_commit(bar(RB_QFREE));       // the segment's last Q K^T is in the pipe
+                    // Issuing an MMA blocks until the pipe takes it and a barrier test costs a round trip of about a
+                    // hundred cycles, so every barrier is tested ahead of the run of MMAs before the one that needs it.
+                    bool v_ok = false, p_ok = false;
                     for (int j = 0; j < nt; ++j) {
                         const int gt = jt + j;
-                        RSTAMP(0);
-                        mbar_wait(bar(RB_FULLV + gt % R_NV), (gt / R_NV) & 1, abort_flag, status);
-                        mbar_wait(bar(RB_P + gt % P_NSBUF), (gt / P_NSBUF) & 1, abort_flag, status);
-                        RSTAMP(1);
+                        if (!v_ok) mbar_wait(bar(RB_FULLV + gt % R_NV), (gt / R_NV) & 1, abort_flag, status);
+                        if (!p_ok) mbar_wait(bar(RB_P + gt % P_NSBUF), (gt / P_NSBUF) & 1, abort_flag, status);
+                        const bool k_ok = j + P_NSBUF < nt && mbar_test(bar(RB_FULLK + (gt + P_NSBUF) % R_NK), ((gt + P_NSBUF) / R_NK) & 1);
                         tc_fence_after();
                         const uint32_t sV16 = (sV + (gt % R_NV) * TILE_BYTES) >> 4;
 #pragma unroll
@@ -1593,9 +1763,16 @@ attn_tc_rb_kernel(const __grid_constant__ CUtensorMap kmap, const __grid_constan
                             mma_ts(tmem + P_NSBUF * 128, tmem + (gt % P_NSBUF) * 128 + k * 8, smem_desc(kDescVMajor, sV16 + k * (2048 >> 4)), kIdescPV,
                                    (j > 0 || k > 0) ? 1u : 0u);
                         tc_commit(bar(RB_EMPTYV + gt % R_NV));           // V tile fully read, O holds tiles 0..j
+                        v_ok = j + 1 < nt && mbar_test(bar(RB_FULLV + (gt + 1) % R_NV), ((gt + 1) / R_NV) & 1);
+                        p_ok = j + 1 < nt && mbar_test(bar(RB_P + (gt + 1) % P_NSBUF), ((gt + 1) / P_NSBUF) & 1);
+                        if (j + P_NSBUF < nt) {
+                            issue_qk(gt + P_NSBUF, k_ok);
+                            if (j + P_NSBUF + 1 == nt) tc_commit(bar(RB_QFREE));
+                        }
                     }
                     tc_commit(bar(RB_O));
                     jt += nt;
+                    ++n_seg_done;
                 }
             }
         } else if (warp == 2) {
@@ -1642,7 +1819,7 @@ attn_tc_rb_kernel(const __grid_constant__ CUtensorMap kmap, const __grid_constan
         } else if (warp >= 4) {
             // =============================== softmax, results ===============================
             const SoftmaxBars lay = {RB_S, RB_P, RB_O, RB_EMPTYV, R_NV, false};
-            softmax_rows(a, plan, lay, bar0, tmem, rank, jt, n_seg_done, abort_flag, status, s_prof);
+            softmax_rows_split(a, plan, lay, bar0, tmem, rank, split, jt, n_seg_done, abort_flag, status);
         }
 
         // ---- next round (only batches with very many short sequences need more than one)
@@ -1653,10 +1830,6 @@ attn_tc_rb_kernel(const __grid_constant__ CUtensorMap kmap, const __grid_constan
         __syncthreads();
         if (plan.nseg == 0) break;
     }
-#ifdef GRAFT_TC_EXPERIMENTS
-    __syncthreads();
-    if (s_prof && threadIdx.x < 64) a.desc[300 + threadIdx.x] = s_prof[threadIdx.x];
-#endif
 
     // ---- teardown: after a timeout some copies may still be in flight: give them time to land before the
     // shared memory is handed back; the allocating warp frees the tensor memory once everyone is past its last access
@@ -1847,7 +2020,7 @@ int graft_attn_tc_init() {
     GRAFT_CHECK_CUDA(cudaFuncSetAttribute(attn_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_DYN));
     // pair kernel: how many 2-CTA clusters fit on the device at once (SMs that cannot be paired stay idle)
     GRAFT_CHECK_CUDA(cudaFuncSetAttribute(attn_tc_pair_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, P_SMEM_DYN + kProfBytes));
-    GRAFT_CHECK_CUDA(cudaFuncSetAttribute(attn_tc_rb_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, R_SMEM_DYN + kProfBytes));
+    GRAFT_CHECK_CUDA(cudaFuncSetAttribute(attn_tc_rb_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, R_SMEM_DYN));
     int dev = 0;
     GRAFT_CHECK_CUDA(cudaGetDevice(&dev));
     if (dev >= 0 && dev < kMaxDevices && g_pair_clusters[dev] == 0) {
@@ -1901,8 +2074,10 @@ size_t graft_attn_tc_ws_bytes(int num_sms, int B, int, int, int d, int) {
 int graft_attn_tc_launch(graft_ctx* ctx, const graft_attn_params* p, cudaStream_t stream, int which) {
     const int G = p->Hq / p->Hkv;
     // which: 0 two row blocks per CTA, 1 CTA pairs with two-SM MMAs, 2 one row block per CTA with partners sharing
-    // tiles through L2, < 0 choose
-    if (which < 0) which = 2;
+    // tiles through L2, < 0 choose.  Measured: kernels 1 and 2 are within a few per cent of each other and both
+    // beat kernel 0 everywhere; the pair kernel wins when a KV head carries more than 256 rows, the row-block
+    // kernel otherwise.
+    if (which < 0) which = (p->T_max * G > 256 && graft_attn_tc_pair_supported(ctx, p)) ? 1 : 2;
     const bool use_pair = which == 1, use_rb = which == 2;
     if (use_pair && !graft_attn_tc_pair_supported(ctx, p)) return GRAFT_ERR_UNSUPPORTED;
     CUtensorMap kmap, vmap;
@@ -1932,7 +2107,7 @@ int graft_attn_tc_launch(graft_ctx* ctx, const graft_attn_params* p, cudaStream_
         if (pairs > ctx->num_sms / 2) pairs = ctx->num_sms / 2;       // the workspace has two slots per SM
         attn_tc_pair_kernel<<<2 * pairs, P_NTHREADS, P_SMEM_DYN + kProfBytes, stream>>>(kmap, vmap, qmap, a, ctx->status);
     } else if (use_rb) {
-        attn_tc_rb_kernel<<<ctx->num_sms & ~1, R_NTHREADS, R_SMEM_DYN + kProfBytes, stream>>>(kmap, vmap, qmap, a, ctx->status);
+        attn_tc_rb_kernel<<<ctx->num_sms & ~1, R_NTHREADS, R_SMEM_DYN, stream>>>(kmap, vmap, qmap, a, ctx->status);
     } else
     attn_tc_kernel<<<grid, NTHREADS, SMEM_DYN, stream>>>(kmap, vmap, qmap, a, ctx->status);
     GRAFT_CHECK_CUDA(cudaGetLastError());
