@@ -426,9 +426,10 @@ def main():
 # dram__bytes_read.sum + dram__bytes_write.sum of the attention kernel per launch, from the ncu
 # captures summarised under profiles/ (None until a capture of that workload exists)
 TRAFFIC = {
-    # 1.03 x algorithmic bytes, measured on cfg4-B1-32k (profiles/attn_tc_kernel_cfg4-B1-32k.md) and scaled
-    # by the keys processed where the workload is too large for a full capture
-    "cfg4-B1-32k": 138.9e6, "cfg4-B1": 1.03 * 269.6e6, "cfg4-B4": 1.03 * 1078.5e6,
+    # cfg4-B1-32k and cfg3: measured (profiles/attn_tc_pair_kernel_cfg4-B1-32k.md, profiles/attn_tc_rb_kernel_cfg3.md);
+    # the 64K workloads are too large for a full capture under the size rule: 1.026 x algorithmic bytes as measured
+    # at 32K, scaled by the keys processed (same kernel, traffic grows in proportion)
+    "cfg4-B1-32k": 138.85e6, "cfg3": 144.5e6, "cfg4-B1": 1.026 * 269.6e6, "cfg4-B4": 1.026 * 1078.5e6,
 }
 
 if __name__ == "__main__":
