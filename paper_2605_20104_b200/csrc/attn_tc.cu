@@ -537,6 +537,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap kmap, const __grid_constant__
     if (threadIdx.x == 0) s_abort = 0;
     __syncthreads();
     if (s_nseg == 0) return;                      // nothing for this CTA (short batch)
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");      // the merge kernel may be set up from now on (it waits for this grid to end)
 
     // ring load n of a segment's tile t: K (which = 0) or V (which = 1)
     auto issue_load = [&](const Seg& sg, int t, int which, int n) {
@@ -1433,6 +1434,7 @@ attn_tc_pair_kernel(const __grid_constant__ CUtensorMap kmap, const __grid_const
     if (threadIdx.x == 0) ctrl.abort = 0;
     __syncthreads();
     if (plan.nseg == 0) return;                       // nothing for this pair (short batch); no cluster operation was started
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");      // the merge kernel may be set up from now on (it waits for this grid to end)
 
     if (threadIdx.x == 0) {
         for (int i = 0; i < P_NSLOT; ++i) { mbar_init(bar(PB_FULL + i), 1); mbar_init(bar(PB_EMPTY + i), 1); }
@@ -1659,6 +1661,7 @@ attn_tc_rb_kernel(const __grid_constant__ CUtensorMap kmap, const __grid_constan
     if (threadIdx.x == 0) ctrl.abort = 0;
     __syncthreads();
     if (plan.nseg == 0) return;                       // nothing for this worker (short batch)
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");      // the merge kernel may be set up from now on (it waits for this grid to end)
 
     if (threadIdx.x == 0) {
         for (int i = 0; i < R_NK; ++i) { mbar_init(bar(RB_FULLK + i), 1); mbar_init(bar(RB_EMPTYK + i), 1); }
@@ -1855,6 +1858,7 @@ attn_tc_rb_kernel(const __grid_constant__ CUtensorMap kmap, const __grid_constan
 constexpr int kMergeWarps = 8;       // warps per CTA; rows per CTA is a launch parameter (8: one per warp, or 32)
 
 __global__ void __launch_bounds__(kMergeWarps * 32, 2) merge_streamk_kernel(TcArgs a, int rows_per_cta, unsigned* status) {
+    asm volatile("griddepcontrol.wait;" ::: "memory");      // launched early: nothing is read before the attention kernel is complete
     const graft_attn_params& p = a.p;
     const int G = a.G;
     const int rows_pad = p.T_max * G;
@@ -2115,7 +2119,18 @@ int graft_attn_tc_launch(graft_ctx* ctx, const graft_attn_params* p, cudaStream_
     const int rows_pad = p->T_max * a.G;
     const int rows_per_cta = (long long)p->B * p->Hkv * rows_pad >= 32768 ? 32 : 8;
     const int groups = (rows_pad + rows_per_cta - 1) / rows_per_cta;
-    merge_streamk_kernel<<<p->B * p->Hkv * groups, kMergeWarps * 32, 0, stream>>>(a, rows_per_cta, ctx->status);
-    GRAFT_CHECK_CUDA(cudaGetLastError());
+    // programmatic dependent launch: the merge CTAs are set up while the attention kernel still runs and wait
+    // (griddepcontrol.wait) until it has completed and its writes are visible
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((unsigned)(p->B * p->Hkv * groups));
+    cfg.blockDim = dim3(kMergeWarps * 32);
+    cfg.dynamicSmemBytes = 0;
+    cfg.stream = stream;
+    cudaLaunchAttribute attr;
+    attr.id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr.val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = &attr;
+    cfg.numAttrs = 1;
+    GRAFT_CHECK_CUDA(cudaLaunchKernelEx(&cfg, merge_streamk_kernel, a, rows_per_cta, ctx->status));
     return GRAFT_OK;
 }
