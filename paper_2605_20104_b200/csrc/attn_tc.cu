@@ -925,12 +925,12 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap kmap, const __grid_constant__
 // The last tile of an item is fetched at keys [L+T-128, L+T) instead of a tile-aligned position: it never
 // reaches past the sequence's keys (rows before key 0 are zero-filled by the copy), and the columns that
 // the previous tile already covered are masked like non-ancestors.
-constexpr int P_NTHREADS = 256;          // producer, Q K^T issuer, Q loader, P V issuer, four softmax warps
+constexpr int P_NTHREADS = 384;          // producer, Q K^T issuer, Q loader, P V issuer, eight softmax warps
 constexpr int P_HALF_TILE = TILE_BYTES / 2;       // this CTA's half of a K tile or of a V tile
 constexpr int P_SLOT_BYTES = 2 * P_HALF_TILE;     // one ring slot: the K half, then the V half of a tile
 constexpr int P_NSLOT = 6;
 constexpr int kCtrlBytes = 1024;
-constexpr int P_SMEM_DYN = kCtrlBytes + TILE_BYTES + P_NSLOT * P_SLOT_BYTES;      // control, Q (128 rows), ring
+constexpr int P_SMEM_DYN = kCtrlBytes + TILE_BYTES + P_NSLOT * P_SLOT_BYTES + 2048;      // control, Q (128 rows), ring, softmax exchange: 227 KB
 constexpr int P_NSBUF = 3;                        // score buffers in tensor memory (128 columns each), O behind them
 enum { PB_FULL = 0, PB_EMPTY = P_NSLOT, PB_S = 2 * P_NSLOT, PB_P = PB_S + P_NSBUF, PB_Q = PB_P + P_NSBUF, PB_O = PB_Q + 1,
        PB_QFREE = PB_O + 1, PB_COUNT = PB_QFREE + 1 };
@@ -941,11 +941,6 @@ struct PairCtrl {
     int abort;
 };
 static_assert(sizeof(PairCtrl) <= kCtrlBytes, "control block too large");
-#ifdef GRAFT_TC_EXPERIMENTS
-constexpr int kProfBytes = 1024;      // time stamps of one CTA
-#else
-constexpr int kProfBytes = 0;
-#endif
 
 __device__ __forceinline__ uint32_t cluster_ctarank() {
     uint32_t r;
@@ -1029,8 +1024,8 @@ constexpr uint32_t kIdescPairQK = kIdescPairBase;
 constexpr uint32_t kIdescPairPV = kIdescPairBase | (1u << 16);
 
 // ---------------------------------------------------------------------------------------------------
-// softmax and results of one 128-row block (four warps, one row per thread), shared by the kernels that
-// keep three score buffers in tensor memory (columns 0..383) and O behind them (384..511)
+// pieces shared by the kernels that keep three score buffers in tensor memory (columns 0..383) and O behind
+// them (384..511)
 // ---------------------------------------------------------------------------------------------------
 struct SoftmaxBars {
     int S, P, O;             // barrier indices: score buffer ready (x3), P written (x3), all MMAs of the segment complete
@@ -1049,7 +1044,7 @@ __device__ __forceinline__ int tile_key0(const Seg& sg, int t, int& overlap) {
 }
 
 // ---------------------------------------------------------------------------------------------------
-// softmax of a 128-row block by two warpgroups that split the columns of every tile (row-block kernel)
+// softmax and results of a 128-row block by two warpgroups that split the columns of every tile
 // ---------------------------------------------------------------------------------------------------
 // Warps w and w + 4 own the same 32 rows (tensor-memory lanes) and take columns 0..63 and 64..127 of the
 // score tile, so two warps per scheduler keep the exponential unit busy and a row's 64 scores stay in
@@ -1232,171 +1227,6 @@ __device__ __forceinline__ void softmax_rows_split(const TcArgs& a, const Plan& 
     }
 }
 
-__device__ __forceinline__ void softmax_rows(const TcArgs& a, const Plan& plan, const SoftmaxBars lay, uint32_t bar0, uint32_t tmem, int rank,
-                                             int& jt, int& n_seg_done, volatile int* abort_flag, unsigned* status, volatile int* prof = nullptr) {
-    const graft_attn_params& p = a.p;
-    const int G = a.G;
-    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const int nseg = plan.nseg;
-    auto bar = [&](int i) { return bar0 + 8u * (uint32_t)i; };
-#ifdef GRAFT_TC_EXPERIMENTS
-#define SSTAMP(k) do { if (prof && threadIdx.x == 128 && gt >= 40 && gt < 48) prof[(gt - 40) * 4 + (k)] = (int)clock(); } while (0)
-#else
-#define SSTAMP(k) do { (void)prof; } while (0)
-#endif
-    const int rl = ((warp & 3) << 5) + lane;            // row inside this CTA's block = TMEM lane
-    const uint32_t lane_bits = (uint32_t)((warp & 3) << 5) << 16;
-    const uint32_t tO = tmem + lane_bits + P_NSBUF * 128;
-    const float sl2 = p.scale * kLog2e;
-    for (int si = 0; si < nseg; ++si) {
-        const Seg sg = plan.seg[si];
-        const int nt = sg.tile_hi - sg.tile_lo;
-        const int R = sg.T * G;
-        const int r = sg.rb * BR + (int)rank * 128 + rl;
-        const bool row_valid = r < R;
-        const int t = row_valid ? r / G : 0, g = row_valid ? r % G : 0;
-        const unsigned long long anc = row_valid ? p.tree_anc[(size_t)sg.b * p.T_max + t] : 0ull;
-        const unsigned long long allowed = sg.T >= 64 ? anc : (anc & ((1ull << sg.T) - 1ull));
-        float m_ref = -CUDART_INF_F, l = 0.f;
-
-        for (int j = 0; j < nt; ++j) {
-            const int gt = jt + j;
-            const uint32_t tS = tmem + lane_bits + (gt % P_NSBUF) * 128;
-            int overlap;
-            const int key0 = tile_key0(sg, sg.tile_lo + j, overlap);
-            const bool masked = key0 + BN > sg.L || overlap > 0;
-            SSTAMP(0);
-            mbar_wait(bar(lay.S + gt % P_NSBUF), (gt / P_NSBUF) & 1, abort_flag, status);
-            tc_fence_after();
-            SSTAMP(1);
-            uint32_t x[4][32];
-#pragma unroll
-            for (int c = 0; c < 4; ++c) tmem_ld32(tS + c * 32, x[c]);
-            tmem_wait_ld();
-            if (masked) {
-                // per 32-column chunk one word of allowed columns: cached keys not yet covered, ancestors in the tree
-#pragma unroll
-                for (int c = 0; c < 4; ++c) {
-                    const int u0 = key0 + c * 32 - sg.L;         // tree index of the chunk's first column
-                    uint32_t w;
-                    if (u0 >= 64) w = 0u;
-                    else if (u0 >= 0) w = (uint32_t)(allowed >> u0);
-                    else if (u0 <= -32) w = 0xffffffffu;
-                    else w = (uint32_t)((allowed << (-u0)) | ((1ull << (-u0)) - 1ull));
-                    const int cov = overlap - c * 32;            // columns of this chunk that the previous tile covered
-                    if (cov >= 32) w = 0u;
-                    else if (cov > 0) w &= ~((1u << cov) - 1u);
-#pragma unroll
-                    for (int q = 0; q < 32; ++q)
-                        if (!((w >> q) & 1u)) x[c][q] = 0xff800000u;   // -inf
-                }
-            }
-            float mx0 = -CUDART_INF_F, mx1 = -CUDART_INF_F;
-#pragma unroll
-            for (int c = 0; c < 4; ++c)
-#pragma unroll
-                for (int q = 0; q < 32; q += 4) {
-                    mx0 = fmax3(mx0, __uint_as_float(x[c][q]), __uint_as_float(x[c][q + 1]));
-                    mx1 = fmax3(mx1, __uint_as_float(x[c][q + 2]), __uint_as_float(x[c][q + 3]));
-                }
-            const float mx = fmaxf(mx0, mx1);
-            // reference maximum: move it only when the scores outgrow it by more than the threshold
-            if (mx != -CUDART_INF_F && (m_ref == -CUDART_INF_F || (mx - m_ref) * sl2 > kRescaleThreshold)) {
-                if (m_ref != -CUDART_INF_F) {
-                    // O must hold every earlier tile of the segment before it is rescaled (j > 0 here)
-                    mbar_wait(bar(lay.pv_done + (gt - 1) % lay.pv_mod), ((gt - 1) / lay.pv_mod) & 1, abort_flag, status);
-                    tc_fence_after();
-                    const float alpha = exp2f((m_ref - mx) * sl2);
-                    l *= alpha;
-#pragma unroll 1
-                    for (int c = 0; c < 4; ++c) {
-                        uint32_t o[32];
-                        tmem_ld32(tO + c * 32, o);
-                        tmem_wait_ld();
-#pragma unroll
-                        for (int q = 0; q < 32; ++q) o[q] = __float_as_uint(__uint_as_float(o[q]) * alpha);
-                        tmem_st32(tO + c * 32, o);
-                    }
-                    tmem_wait_st();
-                }
-                m_ref = mx;
-            }
-            const float off = m_ref == -CUDART_INF_F ? 0.f : m_ref * sl2;
-            // P = 2^(s*scale*log2e - off) as bf16 into the first 64 columns of this S buffer
-            float sum0 = 0.f, sum1 = 0.f;
-#pragma unroll
-            for (int c = 0; c < 4; ++c) {
-                uint32_t pk[16];
-#pragma unroll
-                for (int q = 0; q < 32; q += 2) {
-                    const float p0 = ex2(fmaf(__uint_as_float(x[c][q]), sl2, -off));
-                    const float p1 = ex2(fmaf(__uint_as_float(x[c][q + 1]), sl2, -off));
-                    sum0 += p0;
-                    sum1 += p1;
-                    pk[q >> 1] = pack_bf16(p0, p1);
-                }
-                tmem_st16(tS + c * 16, pk);
-            }
-            l += sum0 + sum1;
-            tmem_wait_st();
-            SSTAMP(2);
-            tc_fence_before();
-            __syncwarp();
-            if (lane == 0) {                               // one arrival per warp
-                if (lay.remote) mbar_arrive_remote(map_to_cta(bar(lay.P + gt % P_NSBUF), 0u));
-                else mbar_arrive(bar(lay.P + gt % P_NSBUF));
-            }
-        }
-
-        // ---- results of the segment: O row from TMEM, final rows or a partial
-        mbar_wait(bar(lay.O), n_seg_done & 1, abort_flag, status);     // every MMA of the segment is complete
-        tc_fence_after();
-        if (sg.slot < 0) {
-            const float inv = l > 0.f ? 1.f / l : 0.f;
-            __nv_bfloat16* orow = reinterpret_cast<__nv_bfloat16*>(p.O) + (size_t)sg.b * p.o_stride_b + (size_t)t * p.o_stride_t +
-                                  (size_t)(sg.h * G + g) * p.o_stride_h;
-#pragma unroll 1
-            for (int c = 0; c < 4; ++c) {
-                uint32_t v[32];
-                tmem_ld32(tO + c * 32, v);
-                tmem_wait_ld();
-                if (row_valid) {
-#pragma unroll
-                    for (int q = 0; q < 4; ++q) {      // 16-byte stores: O strides are only guaranteed 16-byte aligned
-                        uint4 o4;
-                        o4.x = pack_bf16(__uint_as_float(v[q * 8 + 0]) * inv, __uint_as_float(v[q * 8 + 1]) * inv);
-                        o4.y = pack_bf16(__uint_as_float(v[q * 8 + 2]) * inv, __uint_as_float(v[q * 8 + 3]) * inv);
-                        o4.z = pack_bf16(__uint_as_float(v[q * 8 + 4]) * inv, __uint_as_float(v[q * 8 + 5]) * inv);
-                        o4.w = pack_bf16(__uint_as_float(v[q * 8 + 6]) * inv, __uint_as_float(v[q * 8 + 7]) * inv);
-                        *reinterpret_cast<uint4*>(orow + c * 32 + q * 8) = o4;
-                    }
-                }
-            }
-            if (row_valid && p.LSE)
-                p.LSE[((size_t)sg.b * p.Hq + sg.h * G + g) * p.T_max + t] =
-                    l > 0.f ? (m_ref * sl2 + log2f(l)) * kLn2 : -CUDART_INF_F;
-        } else {
-            float* base = a.partial + (size_t)sg.slot * SLOT_FLOATS;
-            const int lr = (int)rank * 128 + rl;
-            float* prow = base + (size_t)lr * D;
-#pragma unroll 1
-            for (int c = 0; c < 4; ++c) {
-                uint32_t v[32];
-                tmem_ld32(tO + c * 32, v);
-                tmem_wait_ld();
-#pragma unroll
-                for (int q = 0; q < 4; ++q)      // 32-byte stores: every store fills a whole sector
-                    st_global_v8(prow + c * 32 + q * 8, v[q * 8], v[q * 8 + 1], v[q * 8 + 2], v[q * 8 + 3], v[q * 8 + 4],
-                                 v[q * 8 + 5], v[q * 8 + 6], v[q * 8 + 7]);
-            }
-            base[BR * D + lr] = m_ref == -CUDART_INF_F ? -CUDART_INF_F : m_ref * sl2;
-            base[BR * D + BR + lr] = l;
-        }
-        tc_fence_before();                 // TMEM reads done before the next segment's MMAs are released
-        jt += nt;
-        ++n_seg_done;
-    }
-}
 
 __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(P_NTHREADS, 1)
 attn_tc_pair_kernel(const __grid_constant__ CUtensorMap kmap, const __grid_constant__ CUtensorMap vmap, const __grid_constant__ CUtensorMap qmap,
@@ -1408,14 +1238,6 @@ attn_tc_pair_kernel(const __grid_constant__ CUtensorMap kmap, const __grid_const
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int G = a.G;
     const uint32_t rank = cluster_ctarank();          // 0: leader (issues the MMAs), 1: peer
-#ifdef GRAFT_TC_EXPERIMENTS
-    const long long t_entry = clock64();
-    const bool prof = (int)blockIdx.x == a.prof_cta;
-    volatile int* s_prof = reinterpret_cast<volatile int*>(smem_raw + P_SMEM_DYN);       // experiments: 1 KB more is requested
-#define PSTAMP(cond, idx) do { if (prof && (cond)) s_prof[(idx) - 256] = (int)(clock() - (int)t_entry); } while (0)
-#else
-#define PSTAMP(cond, idx) do { } while (0)
-#endif
     const int worker = (int)(blockIdx.x >> 1), nworkers = (int)(gridDim.x >> 1);
 
     if ((smem_u32(smem_raw) & 1023u) != 0) {          // the tiles would miss their alignment: refuse to run (both CTAs alike)
@@ -1438,7 +1260,7 @@ attn_tc_pair_kernel(const __grid_constant__ CUtensorMap kmap, const __grid_const
 
     if (threadIdx.x == 0) {
         for (int i = 0; i < P_NSLOT; ++i) { mbar_init(bar(PB_FULL + i), 1); mbar_init(bar(PB_EMPTY + i), 1); }
-        for (int i = 0; i < P_NSBUF; ++i) { mbar_init(bar(PB_S + i), 1); mbar_init(bar(PB_P + i), 8); }      // 4 softmax warps in each CTA
+        for (int i = 0; i < P_NSBUF; ++i) { mbar_init(bar(PB_S + i), 1); mbar_init(bar(PB_P + i), 16); }      // 8 softmax warps in each CTA
         mbar_init(bar(PB_Q), 2);                    // one arrival per CTA (with the byte count when Q goes by TMA)
         mbar_init(bar(PB_O), 1);
         mbar_init(bar(PB_QFREE), 1);
@@ -1453,6 +1275,7 @@ attn_tc_pair_kernel(const __grid_constant__ CUtensorMap kmap, const __grid_const
     cluster_sync_all();                               // the partner's barriers exist before anything signals them
     tc_fence_after();
     const uint32_t tmem = ctrl.tmem;
+    SplitShared& split = *reinterpret_cast<SplitShared*>(smem_raw + kCtrlBytes + TILE_BYTES + P_NSLOT * P_SLOT_BYTES);
 
 
     // running counters that persist across segments and rounds (each role keeps its own copy)
@@ -1582,7 +1405,7 @@ attn_tc_pair_kernel(const __grid_constant__ CUtensorMap kmap, const __grid_const
         } else if (warp >= 4) {
             // =============================== softmax, results (both CTAs) ===============================
             const SoftmaxBars lay = {PB_S, PB_P, PB_O, PB_EMPTY, P_NSLOT, true};
-            softmax_rows(a, plan, lay, bar0, tmem, (int)rank, jt, n_seg_done, abort_flag, status);
+            softmax_rows_split(a, plan, lay, bar0, tmem, (int)rank, split, jt, n_seg_done, abort_flag, status);
         }
 
         // ---- next round (only batches with very many short sequences need more than one)
@@ -1594,11 +1417,6 @@ attn_tc_pair_kernel(const __grid_constant__ CUtensorMap kmap, const __grid_const
         if (plan.nseg == 0) break;
     }
 
-    PSTAMP(threadIdx.x == 128, 299);
-#ifdef GRAFT_TC_EXPERIMENTS
-    __syncthreads();
-    if (prof && threadIdx.x < 256) a.desc[256 + threadIdx.x] = s_prof[threadIdx.x];
-#endif
     // ---- teardown: nobody leaves while its partner may still read its shared memory or signal its barriers;
     // both CTAs free the tensor memory of the pair
     tc_fence_before();
@@ -2023,7 +1841,7 @@ int graft_attn_tc_init() {
     }
     GRAFT_CHECK_CUDA(cudaFuncSetAttribute(attn_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_DYN));
     // pair kernel: how many 2-CTA clusters fit on the device at once (SMs that cannot be paired stay idle)
-    GRAFT_CHECK_CUDA(cudaFuncSetAttribute(attn_tc_pair_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, P_SMEM_DYN + kProfBytes));
+    GRAFT_CHECK_CUDA(cudaFuncSetAttribute(attn_tc_pair_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, P_SMEM_DYN));
     GRAFT_CHECK_CUDA(cudaFuncSetAttribute(attn_tc_rb_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, R_SMEM_DYN));
     int dev = 0;
     GRAFT_CHECK_CUDA(cudaGetDevice(&dev));
@@ -2033,7 +1851,7 @@ int graft_attn_tc_init() {
         cudaLaunchConfig_t cfg = {};
         cfg.gridDim = dim3((unsigned)(sms & ~1));
         cfg.blockDim = dim3(P_NTHREADS);
-        cfg.dynamicSmemBytes = P_SMEM_DYN + kProfBytes;
+        cfg.dynamicSmemBytes = P_SMEM_DYN;
         cudaLaunchAttribute attr;
         attr.id = cudaLaunchAttributeClusterDimension;
         attr.val.clusterDim.x = 2;
@@ -2109,7 +1927,7 @@ int graft_attn_tc_launch(graft_ctx* ctx, const graft_attn_params* p, cudaStream_
     if (use_pair) {
         int pairs = pair_clusters();
         if (pairs > ctx->num_sms / 2) pairs = ctx->num_sms / 2;       // the workspace has two slots per SM
-        attn_tc_pair_kernel<<<2 * pairs, P_NTHREADS, P_SMEM_DYN + kProfBytes, stream>>>(kmap, vmap, qmap, a, ctx->status);
+        attn_tc_pair_kernel<<<2 * pairs, P_NTHREADS, P_SMEM_DYN, stream>>>(kmap, vmap, qmap, a, ctx->status);
     } else if (use_rb) {
         attn_tc_rb_kernel<<<ctx->num_sms & ~1, R_NTHREADS, R_SMEM_DYN, stream>>>(kmap, vmap, qmap, a, ctx->status);
     } else
