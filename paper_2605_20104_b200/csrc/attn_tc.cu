@@ -1013,6 +1013,64 @@ __device__ __forceinline__ void mma_pair_ts(uint32_t d_tmem, uint32_t a_tmem, ui
                  "tcgen05.mma.cta_group::2.kind::f16 [%0], [%1], %2, %3, p;\n\t}"
                  ::"r"(d_tmem), "r"(a_tmem), "l"(b_desc), "r"(idesc), "r"(accumulate) : "memory");
 }
+// The eight MMAs of one tile as one run of instructions (the issuing warp shares its scheduler with two busy
+// softmax warps, so every instruction it does not need is time the tensor pipe waits): descriptors advance by
+// constants, 2 per 16 elements of K inside a 64-element box, `a_box` / `b_box` between the boxes (16-byte units).
+__device__ __forceinline__ void mma_pair_ss8(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc, uint32_t a_box, uint32_t b_box) {
+    asm volatile(
+        "{\n\t"
+        ".reg .pred pT, pF;\n\t"
+        ".reg .b64 da, db, ia, ib;\n\t"
+        "setp.eq.b32 pT, %3, %3;\n\t"
+        "setp.ne.b32 pF, %3, %3;\n\t"
+        "cvt.u64.u32 ia, %4;\n\t"
+        "cvt.u64.u32 ib, %5;\n\t"
+        "tcgen05.mma.cta_group::2.kind::f16 [%0], %1, %2, %3, pF;\n\t"
+        "add.s64 da, %1, 2;\n\t add.s64 db, %2, 2;\n\t"
+        "tcgen05.mma.cta_group::2.kind::f16 [%0], da, db, %3, pT;\n\t"
+        "add.s64 da, %1, 4;\n\t add.s64 db, %2, 4;\n\t"
+        "tcgen05.mma.cta_group::2.kind::f16 [%0], da, db, %3, pT;\n\t"
+        "add.s64 da, %1, 6;\n\t add.s64 db, %2, 6;\n\t"
+        "tcgen05.mma.cta_group::2.kind::f16 [%0], da, db, %3, pT;\n\t"
+        "add.s64 da, %1, ia;\n\t add.s64 db, %2, ib;\n\t"
+        "tcgen05.mma.cta_group::2.kind::f16 [%0], da, db, %3, pT;\n\t"
+        "add.s64 da, da, 2;\n\t add.s64 db, db, 2;\n\t"
+        "tcgen05.mma.cta_group::2.kind::f16 [%0], da, db, %3, pT;\n\t"
+        "add.s64 da, da, 2;\n\t add.s64 db, db, 2;\n\t"
+        "tcgen05.mma.cta_group::2.kind::f16 [%0], da, db, %3, pT;\n\t"
+        "add.s64 da, da, 2;\n\t add.s64 db, db, 2;\n\t"
+        "tcgen05.mma.cta_group::2.kind::f16 [%0], da, db, %3, pT;\n\t"
+        "}"
+        ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(a_box), "r"(b_box) : "memory");
+}
+// P V: A advances by 8 tensor-memory columns, B by `b_step` (16-byte units) per 16 keys; `accumulate`: O already holds tiles
+__device__ __forceinline__ void mma_pair_ts8(uint32_t d_tmem, uint32_t a_tmem, uint64_t b_desc, uint32_t idesc, uint32_t b_step, uint32_t accumulate) {
+    asm volatile(
+        "{\n\t"
+        ".reg .pred pT, p0;\n\t"
+        ".reg .b64 db, ib;\n\t"
+        ".reg .b32 ta;\n\t"
+        "setp.eq.b32 pT, %3, %3;\n\t"
+        "setp.ne.b32 p0, %5, 0;\n\t"
+        "cvt.u64.u32 ib, %4;\n\t"
+        "tcgen05.mma.cta_group::2.kind::f16 [%0], [%1], %2, %3, p0;\n\t"
+        "add.u32 ta, %1, 8;\n\t add.s64 db, %2, ib;\n\t"
+        "tcgen05.mma.cta_group::2.kind::f16 [%0], [ta], db, %3, pT;\n\t"
+        "add.u32 ta, ta, 8;\n\t add.s64 db, db, ib;\n\t"
+        "tcgen05.mma.cta_group::2.kind::f16 [%0], [ta], db, %3, pT;\n\t"
+        "add.u32 ta, ta, 8;\n\t add.s64 db, db, ib;\n\t"
+        "tcgen05.mma.cta_group::2.kind::f16 [%0], [ta], db, %3, pT;\n\t"
+        "add.u32 ta, ta, 8;\n\t add.s64 db, db, ib;\n\t"
+        "tcgen05.mma.cta_group::2.kind::f16 [%0], [ta], db, %3, pT;\n\t"
+        "add.u32 ta, ta, 8;\n\t add.s64 db, db, ib;\n\t"
+        "tcgen05.mma.cta_group::2.kind::f16 [%0], [ta], db, %3, pT;\n\t"
+        "add.u32 ta, ta, 8;\n\t add.s64 db, db, ib;\n\t"
+        "tcgen05.mma.cta_group::2.kind::f16 [%0], [ta], db, %3, pT;\n\t"
+        "add.u32 ta, ta, 8;\n\t add.s64 db, db, ib;\n\t"
+        "tcgen05.mma.cta_group::2.kind::f16 [%0], [ta], db, %3, pT;\n\t"
+        "}"
+        ::"r"(d_tmem), "r"(a_tmem), "l"(b_desc), "r"(idesc), "r"(b_step), "r"(accumulate) : "memory");
+}
 // arrive on the barrier at this offset in both CTAs once every MMA issued so far is complete
 __device__ __forceinline__ void tc_commit_pair(uint32_t bar) {
     asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], %1;"
@@ -1324,12 +1382,8 @@ attn_tc_pair_kernel(const __grid_constant__ CUtensorMap kmap, const __grid_const
                         // S[buffer gt % 3] = Q K^T with the K half-tiles of ring slot gt % P_NSLOT (V of the same tile lands with it)
                         const uint32_t sK16 = (sRing + (gt % P_NSLOT) * P_SLOT_BYTES) >> 4;
                         const uint32_t sQ16 = sQ >> 4;
-#pragma unroll
-                        for (int k = 0; k < D / 16; ++k) {
-                            const uint32_t offQ = ((k >> 2) * HALF_BYTES + (k & 3) * 32) >> 4;
-                            const uint32_t offK = ((k >> 2) * (P_HALF_TILE / 2) + (k & 3) * 32) >> 4;
-                            mma_pair_ss(tmem + (gt % P_NSBUF) * 128, smem_desc(kDescKMajor, sQ16 + offQ), smem_desc(kDescKMajor, sK16 + offK), kIdescPairQK, k > 0);
-                        }
+                        mma_pair_ss8(tmem + (gt % P_NSBUF) * 128, smem_desc(kDescKMajor, sQ16), smem_desc(kDescKMajor, sK16), kIdescPairQK,
+                                     HALF_BYTES >> 4, (P_HALF_TILE / 2) >> 4);
                         tc_commit_pair(bar(PB_S + gt % P_NSBUF));
                     }
                     tc_commit_pair(bar(PB_QFREE));                // the segment's last Q K^T is in the pipe
@@ -1348,10 +1402,7 @@ attn_tc_pair_kernel(const __grid_constant__ CUtensorMap kmap, const __grid_const
                         mbar_wait_cluster(bar(PB_P + gt % P_NSBUF), (gt / P_NSBUF) & 1, abort_flag, status);
                         tc_fence_after();
                         const uint32_t sV16 = (sRing + (gt % P_NSLOT) * P_SLOT_BYTES + P_HALF_TILE) >> 4;
-#pragma unroll
-                        for (int k = 0; k < BN / 16; ++k)
-                            mma_pair_ts(tmem + P_NSBUF * 128, tmem + (gt % P_NSBUF) * 128 + k * 8, smem_desc(kDescVMajor, sV16 + k * (2048 >> 4)), kIdescPairPV,
-                                        (j > 0 || k > 0) ? 1u : 0u);
+                        mma_pair_ts8(tmem + P_NSBUF * 128, tmem + (gt % P_NSBUF) * 128, smem_desc(kDescVMajor, sV16), kIdescPairPV, 2048 >> 4, j > 0 ? 1u : 0u);
                         tc_commit_pair(bar(PB_EMPTY + gt % P_NSLOT));         // the tile's K and V are read, O holds tiles 0..j
                     }
                     tc_commit_pair(bar(PB_O));
