@@ -81,6 +81,7 @@ def lib():
         _lib.orc_tree_attn_rows.restype = C.c_int
         _lib.orc_accept.restype = None
         _lib.orc_compact_kv.restype = None
+        _lib.orc_update_adjacency.restype = C.c_uint
     return _lib
 
 
@@ -189,3 +190,19 @@ def compact_kv(Kc, Vc, seq_len, n_acc, path) -> dict:
                      new_seq_len=_p(nsl, _i32p, np.int32))
     lib().orc_compact_kv(C.byref(a))
     return dict(K=Kn.reshape(shp), V=Vn.reshape(shp), new_seq_len=nsl)
+
+
+def update_adjacency(logits_bits, tree_token, tree_size, M, k: int) -> dict:
+    """logits_bits: uint16 (bf16 bit patterns) [B*T_max, V]; M: int32 [V, k].  Returns the updated copy of M,
+    target_next [B, T_max] and the flag word."""
+    lg = np.ascontiguousarray(logits_bits, np.uint16)
+    tt, ts = _arr(tree_token, np.int32), _arr(tree_size, np.int32)
+    B, T = tt.shape
+    V = lg.shape[1]
+    assert lg.shape[0] == B * T and M.shape == (V, k)
+    Mn = np.array(M, dtype=np.int32, order="C", copy=True)
+    tn = np.empty((B, T), np.int32)
+    flags = lib().orc_update_adjacency(C.c_int(B), C.c_int(T), C.c_int(V), C.c_int(k), _p(lg, _u16p, np.uint16),
+                                       _p(tt, _i32p, np.int32), _p(ts, _i32p, np.int32), _p(Mn, _i32p, np.int32),
+                                       _p(tn, _i32p, np.int32))
+    return dict(M=Mn, target_next=tn, flags=int(flags))

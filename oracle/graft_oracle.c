@@ -12,7 +12,9 @@
  * enumeration on tiny trees; chain tree == causal attention (library SDPA); T = 1 == plain
  * decode attention; row sums == 1; locality of the ancestor mask; split invariance;
  * the paper's stage budgets 8+52 / 24+36 / 40+20 and template depth histograms; the
- * closed form x_u = M[x_parent(u), r_u]; Propositions 1 and 2 (monotone accepted length).
+ * closed form x_u = M[x_parent(u), r_u]; Propositions 1 and 2 (monotone accepted length);
+ * the adjacency update against a library stable sort, against softmax probabilities, a hand-worked
+ * row with ties / NaN / -inf, and the sequential definition of the duplicate-token winner.
  * Parity unpinned: nothing beyond the printed per-depth counts fixes the retrieval
  * templates' exact rank paths; they are inputs here, not computed.
  */
@@ -414,4 +416,49 @@ void orc_compact_kv(const orc_compact_args *a) {
                     memcpy(a->V_new + dst, a->V_old + src, (size_t)a->d * 2);
                 }
     }
+}
+
+/* ------------------------------------------------------------------------------------------------
+ * Online update of the adjacency matrix (the appendix equation "M[x_i] <- argtopk(p_{i+1})" and the
+ * same rule in the retrieval section): for every verified tree node i of every request, in the
+ * order of the flattened node index r = b * T_max + i, the row of M that belongs to the node's token
+ * is replaced by the ids of the k largest entries of the target's next-token scores at that node.
+ * The scores are given as logits; softmax is monotone, so the ids are the same as for probabilities.
+ * Ids are listed by decreasing score, equal scores by increasing id; NaN scores are never chosen (if
+ * fewer than k scores are not NaN the list is filled with -1 and the NaN flag is set).  Walking r
+ * upwards makes the node with the highest r win when several nodes of the step carry one token.
+ * target_next[r] is the first id of the list (the greedy target id after node i), -1 for padding.
+ * Tokens outside [0, V) update nothing (ids other than -1 also set the bad-token flag).
+ * ------------------------------------------------------------------------------------------------ */
+unsigned orc_update_adjacency(int B, int T_max, int V, int k, const uint16_t *logits /* bf16 bits [B*T_max, V] */,
+                              const int32_t *tree_token, const int32_t *tree_size, int32_t *M /* [V, k] in place */,
+                              int32_t *target_next /* [B*T_max] */) {
+    unsigned flags = 0;
+    double *s = (double *)malloc((size_t)V * sizeof(double));
+    char *taken = (char *)malloc((size_t)V);
+    int32_t *top = (int32_t *)malloc((size_t)k * sizeof(int32_t));
+    for (int b = 0; b < B; ++b) {
+        int T = tree_size[b];
+        if (T < 0 || T > T_max) { T = 0; flags |= ORC_FLAG_BAD_SIZE; }
+        for (int i = 0; i < T_max; ++i) {
+            const size_t r = (size_t)b * T_max + i;
+            if (i >= T) { target_next[r] = -1; continue; }
+            for (int v = 0; v < V; ++v) { s[v] = bf16_to_double(logits[r * V + v]); taken[v] = 0; }
+            for (int j = 0; j < k; ++j) {
+                int best = -1;
+                for (int v = 0; v < V; ++v) {
+                    if (taken[v] || s[v] != s[v]) continue;
+                    if (best < 0 || s[v] > s[best]) best = v;       /* strict: the lowest id wins a tie */
+                }
+                top[j] = best;
+                if (best >= 0) taken[best] = 1; else flags |= ORC_FLAG_NAN_SCORE;
+            }
+            target_next[r] = top[0];
+            const int x = tree_token[r];
+            if (x >= 0 && x < V) memcpy(M + (size_t)x * k, top, (size_t)k * sizeof(int32_t));
+            else if (x != -1) flags |= ORC_FLAG_BAD_TOKEN;
+        }
+    }
+    free(s); free(taken); free(top);
+    return flags;
 }

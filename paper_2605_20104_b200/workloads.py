@@ -424,3 +424,16 @@ def custom(parents: List[np.ndarray], *, Hq: int, Hkv: int, d: int, L: Sequence[
                     K_max=T_max, V=V, k=k, scale=float(np.float32(1.0 / math.sqrt(d))),
                     seq_len=seq_len, draft_token=tok, draft_parent=par, draft_score=sc, n_draft=nd,
                     M=_random_M(rng, V, k), mode=MODE_NONE, p_draft=p, p_graft=p, seed=seed, std=std)
+
+
+def make_logits(B: int, T_max: int, V: int, seed: int, peaks: int = 12) -> np.ndarray:
+    """Target logits of all tree nodes, bf16 bit patterns [B*T_max, V]: a broad body (normal, sigma 2.5) with a
+    few high entries per row, as the output of an LM head looks after the final norm; rounding to bf16 makes
+    equal values common, also among the largest entries.  Rows of padding nodes are filled like the others."""
+    rng = np.random.default_rng(np.random.PCG64(seed))
+    N = B * T_max
+    x = rng.standard_normal((N, V), dtype=np.float32) * np.float32(2.5)
+    cols = rng.integers(0, V, size=(N, peaks))
+    vals = (rng.integers(32, 60, size=(N, peaks)) * np.float32(0.25)).astype(np.float32)     # 8.0 .. 14.75 in steps of 1/4
+    np.put_along_axis(x, cols, vals, axis=1)
+    return bf16_bits(torch.from_numpy(x).to(torch.bfloat16))
