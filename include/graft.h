@@ -9,7 +9,8 @@
  *     graft_build_tree        Algorithm 2 from "Resolve (K_draft, K_ret)" on: prune, graft, rebuild
  *     [caller: QKV projection writes the tree tokens' K/V to cache slots L_b .. L_b + T_b - 1]
  *     graft_tree_verify_attn  Sec. 3.3: tree attention of the T tree tokens over cache + ancestors
- *     [caller: lm_head / argmax gives target_next]
+ *     [caller: lm_head gives the target logits of the tree nodes]
+ *     graft_update_adjacency  retrieval section / appendix: M[x_i] <- argtopk(p_{i+1}); also target_next
  *     graft_accept            Algorithm 1 "select the accepted path" (greedy, lossless)
  *     graft_compact_kv        Algorithm 1 "append accepted tokens and update target KV cache"
  *
@@ -204,6 +205,31 @@ int graft_tree_verify_attn(graft_ctx* ctx, const graft_attn_params* p, void* str
  */
 size_t graft_noalloc_scratch_bytes(void);
 int graft_tree_verify_attn_noalloc(const graft_attn_params* p, void* stream, unsigned* device_flags_out);
+
+/* ---- graft_update_adjacency ------------------------------------------------------------------- */
+/*
+ * Online refresh of the retrieval matrix (retrieval section and appendix, "M[x_i] <- argtopk(p_{i+1})",
+ * over the whole verified tree, accepted and rejected nodes, all requests in one flattened batch), and
+ * the target's greedy ids for graft_accept.  Row r = b * T_max + i of `logits` holds the target's
+ * next-token logits at tree node i of sequence b (softmax is monotone: the ids of the k largest logits
+ * are those of the k largest probabilities).  For every node i < tree_size[b] with a token x in [0, V):
+ * M[x, 0..k) <- the ids of the k largest logits of row r, by decreasing logit, equal logits by increasing
+ * id; NaN is never chosen (GRAFT_FLAG_NAN_SCORE and -1 entries if fewer than k logits are not NaN).
+ * When several nodes of the step carry the same token, the node with the highest r wins.  Rows of M of
+ * other tokens do not change.  target_next[r] (optional) <- the first id of the list, -1 for padding
+ * nodes.  Token -1 updates nothing; any other id outside [0, V) sets GRAFT_FLAG_BAD_TOKEN.
+ * k <= 16; logits: 16-byte aligned base, row stride a multiple of 8 elements.
+ */
+typedef struct {
+    int B, T_max, V, k;
+    const void* logits; int64_t logits_stride_row;   /* bf16 [B * T_max, V] */
+    const int32_t* tree_token;   /* [B, T_max] */
+    const int32_t* tree_size;    /* [B] */
+    int32_t* M;                  /* [V, k], updated in place */
+    int32_t* target_next;        /* out [B, T_max], may be NULL */
+} graft_update_params;
+
+int graft_update_adjacency(graft_ctx* ctx, const graft_update_params* p, void* stream);
 
 /* ---- graft_accept ---------------------------------------------------------------------------- */
 /*

@@ -29,7 +29,7 @@ ATTN_AUTO, ATTN_MMA_SYNC, ATTN_TCGEN05, ATTN_TCGEN05_1SM, ATTN_TCGEN05_2SM, ATTN
 
 EXPORTS = ("graft_workspace_bytes", "graft_create", "graft_destroy", "graft_status_string", "graft_device_status",
            "graft_build_tree", "graft_tree_verify_attn", "graft_accept", "graft_compact_kv",
-           "graft_noalloc_scratch_bytes", "graft_tree_verify_attn_noalloc")
+           "graft_noalloc_scratch_bytes", "graft_tree_verify_attn_noalloc", "graft_update_adjacency")
 
 _vp = C.c_void_p
 
@@ -59,6 +59,11 @@ class AcceptParams(C.Structure):
                                     "best_node", "bonus")])
 
 
+class UpdateParams(C.Structure):
+    _fields_ = ([(n, C.c_int) for n in ("B", "T_max", "V", "k")] + [("logits", _vp), ("logits_stride_row", C.c_int64)] +
+                [(n, _vp) for n in ("tree_token", "tree_size", "M", "target_next")])
+
+
 class CompactParams(C.Structure):
     _fields_ = ([(n, C.c_int) for n in ("B", "Hkv", "d", "S_cap", "T_max", "n_layers")] +
                 [(n, C.c_int64) for n in ("layer_stride", "kv_stride_b", "kv_stride_h", "kv_stride_s")] +
@@ -76,7 +81,8 @@ _lib.graft_status_string.argtypes = [C.c_int]
 _lib.graft_device_status.restype = C.c_int
 _lib.graft_device_status.argtypes = [_vp, _vp, C.POINTER(C.c_uint), C.c_int]
 for _name, _typ in (("graft_build_tree", BuildParams), ("graft_tree_verify_attn", AttnParams),
-                    ("graft_accept", AcceptParams), ("graft_compact_kv", CompactParams)):
+                    ("graft_accept", AcceptParams), ("graft_compact_kv", CompactParams),
+                    ("graft_update_adjacency", UpdateParams)):
     getattr(_lib, _name).restype = C.c_int
     getattr(_lib, _name).argtypes = [_vp, C.POINTER(_typ), _vp]
 
@@ -226,6 +232,22 @@ def accept_params(*, tree_token, tree_parent, tree_anc, tree_size, target_next, 
                      target_next=_ptr(target_next, i32), n_acc=_ptr(n_acc, i32), path=_ptr(path, i32),
                      best_node=_ptr(best_node, i32), bonus=_ptr(bonus, i32))
     return p
+
+
+def update_adjacency_params(*, logits, tree_token, tree_size, M, target_next=None) -> UpdateParams:
+    """logits: bf16 [B*T_max, V] (rows may be strided); M: int32 [V, k], updated in place."""
+    i32 = torch.int32
+    B, T_max = tree_token.shape
+    assert logits.dim() == 2 and logits.shape[0] == B * T_max and logits.stride(1) == 1
+    V, k = M.shape
+    assert logits.shape[1] == V and M.is_contiguous()
+    return UpdateParams(B=B, T_max=T_max, V=V, k=k, logits=_ptr(logits, torch.bfloat16),
+                        logits_stride_row=logits.stride(0), tree_token=_ptr(tree_token, i32), tree_size=_ptr(tree_size, i32),
+                        M=_ptr(M, i32), target_next=_ptr(target_next, i32) if target_next is not None else None)
+
+
+def graft_update_adjacency(ctx: Context, **kw) -> None:
+    launch("graft_update_adjacency", ctx, update_adjacency_params(**kw))
 
 
 def graft_accept(ctx: Context, **kw) -> None:

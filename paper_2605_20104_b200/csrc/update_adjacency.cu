@@ -1,0 +1,243 @@
+// graft_update_adjacency: M[token of node] <- ids of the k largest target logits at that node, one CTA per node.
+//
+// The row of V logits is streamed twice (the second time out of L2), never sorted:
+//   pass 1  every thread keeps the maximum of the entries it sees (packed bf16 max); the k-th largest of the
+//           512 thread maxima is a lower bound tau of the row's k-th largest entry, because the k largest
+//           thread maxima are k different entries;
+//   pass 2  entries above tau go to a candidate list in shared memory: they all sit with the at most k-1
+//           threads whose maximum is above tau, so the list is bounded by (k-1) x entries per thread;
+//           entries equal to tau are unbounded in number (ties are common in bf16), but only the k with the
+//           lowest ids can matter and each thread meets its own in increasing order, so a thread keeps its
+//           first k in registers;
+//   select  one warp takes the k best of the list (by value, equal values by id), then the CTA fills up
+//           with the lowest ids among the entries equal to tau.
+// NaN is never chosen (the packed max and the comparisons ignore it); -0 and +0 are equal.
+// The node with the highest flattened index wins a token that several nodes of the step carry: a CTA
+// writes its row of M only if no later valid node has the same token.
+#include <cuda_bf16.h>
+#include <math_constants.h>
+#include "graft_internal.cuh"
+
+namespace {
+
+constexpr int UT = 512;             // threads per CTA
+constexpr int UK = 16;              // largest k
+constexpr int UCAP = 4608;          // candidate list entries
+
+__device__ __forceinline__ uint32_t hmax2_bits(uint32_t a, uint32_t b) {
+    __nv_bfloat162 x = *reinterpret_cast<__nv_bfloat162*>(&a), y = *reinterpret_cast<__nv_bfloat162*>(&b);
+    __nv_bfloat162 m = __hmax2(x, y);
+    return *reinterpret_cast<uint32_t*>(&m);
+}
+__device__ __forceinline__ uint32_t heq2_bits(uint32_t a, uint32_t b) {
+    __nv_bfloat162 x = *reinterpret_cast<__nv_bfloat162*>(&a), y = *reinterpret_cast<__nv_bfloat162*>(&b);
+    __nv_bfloat162 m = __heq2(x, y);
+    return *reinterpret_cast<uint32_t*>(&m);
+}
+__device__ __forceinline__ float lo_f(uint32_t w) { return __uint_as_float(w << 16); }
+__device__ __forceinline__ float hi_f(uint32_t w) { return __uint_as_float(w & 0xffff0000u); }
+
+// (value, id) order of the result: larger value first, equal values by lower id
+__device__ __forceinline__ bool before(float va, int ia, float vb, int ib) { return va > vb || (va == vb && ia < ib); }
+
+__global__ void __launch_bounds__(UT, 2) update_kernel(graft_update_params p, unsigned* status) {
+    __shared__ float s_cv[UCAP];
+    __shared__ int s_ci[UCAP];
+    __shared__ float s_wtop[UT / 32][UK];
+    __shared__ int s_red[UT / 32];
+    __shared__ int s_cnt, s_min, s_dup;
+    __shared__ float s_tau;
+    __shared__ int s_top[UK];
+
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int r = blockIdx.x, b = r / p.T_max, i = r % p.T_max;
+    int T = p.tree_size[b];
+    if (T < 0 || T > p.T_max) {
+        if (i == 0 && tid == 0) atomicOr(status, (unsigned)GRAFT_FLAG_BAD_SIZE);
+        T = 0;
+    }
+    if (i >= T) {                       // padding node
+        if (tid == 0 && p.target_next) p.target_next[r] = -1;
+        return;
+    }
+    const int k = p.k, V = p.V;
+    const uint16_t* row = reinterpret_cast<const uint16_t*>(p.logits) + (size_t)r * p.logits_stride_row;
+    const uint4* row4 = reinterpret_cast<const uint4*>(row);
+    const int nvec = V >> 3, ntail = V & 7;
+    if (tid == 0) s_cnt = 0;
+
+    // ---- pass 1: thread maxima
+    uint32_t m0 = 0xff80ff80u, m1 = m0, m2 = m0, m3 = m0;          // -inf pairs
+    for (int v = tid; v < nvec; v += UT) {
+        const uint4 q = row4[v];
+        m0 = hmax2_bits(m0, q.x); m1 = hmax2_bits(m1, q.y); m2 = hmax2_bits(m2, q.z); m3 = hmax2_bits(m3, q.w);
+    }
+    m0 = hmax2_bits(hmax2_bits(m0, m1), hmax2_bits(m2, m3));
+    float tm = fmaxf(lo_f(m0), hi_f(m0));
+    if (tid < ntail) {
+        const float f = lo_f(row[(size_t)nvec * 8 + tid]);
+        if (f == f) tm = fmaxf(tm, f);
+    }
+    // ---- tau = k-th largest of the thread maxima: each warp sorts its 32 (bitonic, descending), warp 0 picks among the tops
+    float x = tm;
+#pragma unroll
+    for (int size = 2; size <= 32; size <<= 1)
+#pragma unroll
+        for (int stride = size >> 1; stride > 0; stride >>= 1) {
+            const float y = __shfl_xor_sync(0xffffffffu, x, stride);
+            const bool up = ((lane & size) == 0) == ((lane & stride) == 0);      // keeps the larger one
+            x = up ? fmaxf(x, y) : fminf(x, y);
+        }
+    if (lane < UK) s_wtop[warp][lane] = x;
+    __syncthreads();
+    if (warp == 0) {
+        float c[(UT / 32) * UK / 32];               // 8 values per lane
+#pragma unroll
+        for (int q = 0; q < (UT / 32) * UK / 32; ++q) c[q] = (&s_wtop[0][0])[q * 32 + lane];
+        float tau = -CUDART_INF_F;
+        for (int j = 0; j < k; ++j) {
+            float best = -CUDART_INF_F;
+            int at = 0;
+#pragma unroll
+            for (int q = 0; q < (UT / 32) * UK / 32; ++q)
+                if (c[q] > best) { best = c[q]; at = q; }
+            float wbest = best;
+#pragma unroll
+            for (int o = 16; o; o >>= 1) wbest = fmaxf(wbest, __shfl_xor_sync(0xffffffffu, wbest, o));
+            tau = wbest;
+            const unsigned who = __ballot_sync(0xffffffffu, best == wbest);
+            if (lane == __ffs(who) - 1) {            // remove one occurrence
+#pragma unroll
+                for (int q = 0; q < (UT / 32) * UK / 32; ++q)
+                    if (q == at) c[q] = -CUDART_INF_F;
+            }
+        }
+        if (lane == 0) s_tau = tau;
+    }
+    __syncthreads();
+    const float tau = s_tau;
+    const __nv_bfloat16 tb = __float2bfloat16_rn(tau);       // exact: tau is a bf16 value
+    const uint32_t t16 = *reinterpret_cast<const uint16_t*>(&tb);
+    const uint32_t tau2 = t16 | (t16 << 16);
+
+    // ---- pass 2: candidates above tau, the thread's first k ids equal to tau
+    int eq[UK];
+    int n_eq = 0;
+    auto visit = [&](float f, int id) {
+        if (f > tau) {
+            const int at = atomicAdd(&s_cnt, 1);
+            if (at < UCAP) { s_cv[at] = f; s_ci[at] = id; }
+        } else if (f == tau && n_eq < k) {
+#pragma unroll
+            for (int q = 0; q < UK; ++q)
+                if (q == n_eq) eq[q] = id;
+            ++n_eq;
+        }
+    };
+    auto visit_word = [&](uint32_t w, int id) {
+        if (hmax2_bits(w, tau2) != tau2 || heq2_bits(w, tau2) != 0u) {
+            visit(lo_f(w), id);
+            visit(hi_f(w), id + 1);
+        }
+    };
+    for (int v = tid; v < nvec; v += UT) {
+        const uint4 q = row4[v];
+        visit_word(q.x, v * 8);
+        visit_word(q.y, v * 8 + 2);
+        visit_word(q.z, v * 8 + 4);
+        visit_word(q.w, v * 8 + 6);
+    }
+    if (tid < ntail) visit(lo_f(row[(size_t)nvec * 8 + tid]), nvec * 8 + tid);
+    __syncthreads();
+    int n_gt = s_cnt;
+    if (n_gt > UCAP) {                  // cannot happen for shapes the host accepts
+        if (tid == 0) atomicOr(status, (unsigned)GRAFT_FLAG_INTERNAL);
+        n_gt = UCAP;
+    }
+
+    // ---- the k best of the list (warp 0)
+    int n_sel = 0;
+    if (warp == 0) {
+        for (int j = 0; j < k && j < n_gt; ++j) {
+            float bv = -CUDART_INF_F;
+            int bi = 0x7fffffff, be = -1;
+            for (int e = lane; e < n_gt; e += 32) {
+                const int id = s_ci[e];
+                if (id >= 0 && before(s_cv[e], id, bv, bi)) { bv = s_cv[e]; bi = id; be = e; }
+            }
+#pragma unroll
+            for (int o = 16; o; o >>= 1) {
+                const float ov = __shfl_xor_sync(0xffffffffu, bv, o);
+                const int oi = __shfl_xor_sync(0xffffffffu, bi, o), oe = __shfl_xor_sync(0xffffffffu, be, o);
+                if (before(ov, oi, bv, bi)) { bv = ov; bi = oi; be = oe; }
+            }
+            if (lane == 0) { s_top[j] = bi; s_ci[be] = -1; }
+            __syncwarp();
+        }
+    }
+    n_sel = n_gt < k ? n_gt : k;
+    __syncthreads();
+
+    // ---- fill up with the lowest ids among the entries equal to tau
+    int ptr = 0;
+    for (int j = n_sel; j < k; ++j) {
+        int cur = 0x7fffffff;
+#pragma unroll
+        for (int q = 0; q < UK; ++q)
+            if (q == ptr && q < n_eq) cur = eq[q];
+        int w = cur;
+#pragma unroll
+        for (int o = 16; o; o >>= 1) w = min(w, __shfl_xor_sync(0xffffffffu, w, o));
+        if (lane == 0) s_red[warp] = w;
+        __syncthreads();
+        if (warp == 0) {
+            int z = lane < UT / 32 ? s_red[lane] : 0x7fffffff;
+#pragma unroll
+            for (int o = 16; o; o >>= 1) z = min(z, __shfl_xor_sync(0xffffffffu, z, o));
+            if (lane == 0) {
+                s_min = z;
+                s_top[j] = z == 0x7fffffff ? -1 : z;
+                if (z == 0x7fffffff) atomicOr(status, (unsigned)GRAFT_FLAG_NAN_SCORE);     // fewer than k entries that are not NaN
+            }
+        }
+        __syncthreads();
+        if (cur == s_min && cur != 0x7fffffff) ++ptr;
+        __syncthreads();
+    }
+
+    // ---- results: the greedy id; the row of M unless a later node of the step carries the same token
+    const int tok = p.tree_token[r];
+    if (tid == 0) {
+        s_dup = 0;
+        if (p.target_next) p.target_next[r] = s_top[0];
+        if (tok != -1 && (tok < 0 || tok >= V)) atomicOr(status, (unsigned)GRAFT_FLAG_BAD_TOKEN);
+    }
+    __syncthreads();
+    if (tok < 0 || tok >= V) return;
+    const int N = p.B * p.T_max;
+    bool dup = false;
+    for (int r2 = r + 1 + tid; r2 < N; r2 += UT) {
+        const int b2 = r2 / p.T_max, i2 = r2 % p.T_max;
+        const int T2 = p.tree_size[b2];
+        if (T2 >= 0 && T2 <= p.T_max && i2 < T2 && p.tree_token[r2] == tok) dup = true;
+    }
+    if (dup) s_dup = 1;
+    __syncthreads();
+    if (!s_dup && tid < k) p.M[(size_t)tok * k + tid] = s_top[tid];
+}
+
+}  // namespace
+
+extern "C" int graft_update_adjacency(graft_ctx* ctx, const graft_update_params* p, void* stream) {
+    if (!ctx || !p) return GRAFT_ERR_INVALID_ARG;
+    if (p->B <= 0 || p->T_max <= 0 || p->V <= 0 || p->k <= 0) return GRAFT_ERR_INVALID_ARG;
+    if (!p->logits || !p->tree_token || !p->tree_size || !p->M) return GRAFT_ERR_INVALID_ARG;
+    if (!graft_aligned16(p->logits) || p->logits_stride_row < p->V || p->logits_stride_row % 8 != 0) return GRAFT_ERR_INVALID_ARG;
+    if (p->k > UK || p->V < p->k) return GRAFT_ERR_UNSUPPORTED;
+    // the candidate list holds what k-1 threads can contribute
+    const long long per_thread = (((long long)(p->V >> 3) + UT - 1) / UT) * 8 + 1;
+    if ((p->k - 1) * per_thread > UCAP) return GRAFT_ERR_UNSUPPORTED;
+    update_kernel<<<p->B * p->T_max, UT, 0, static_cast<cudaStream_t>(stream)>>>(*p, ctx->status);
+    GRAFT_CHECK_CUDA(cudaGetLastError());
+    return GRAFT_OK;
+}
