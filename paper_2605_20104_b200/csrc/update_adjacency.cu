@@ -1,14 +1,15 @@
 // graft_update_adjacency: M[token of node] <- ids of the k largest target logits at that node, one CTA per node.
 //
-// The row of V logits is streamed twice (the second time out of L2), never sorted:
+// The row of V logits is streamed once, a small part of it twice (out of L2), never sorted:
 //   pass 1  every thread keeps the maximum of the entries it sees (packed bf16 max); the k-th largest of the
 //           512 thread maxima is a lower bound tau of the row's k-th largest entry, because the k largest
 //           thread maxima are k different entries;
 //   pass 2  entries above tau go to a candidate list in shared memory: they all sit with the at most k-1
-//           threads whose maximum is above tau, so the list is bounded by (k-1) x entries per thread;
-//           entries equal to tau are unbounded in number (ties are common in bf16), but only the k with the
-//           lowest ids can matter and each thread meets its own in increasing order, so a thread keeps its
-//           first k in registers;
+//           threads whose maximum is above tau, so the list is bounded by (k-1) x entries per thread; entries
+//           equal to tau are unbounded in number (ties are common in bf16), but only the k with the lowest
+//           ids can matter.  Normally only a dozen threads reached tau: the CTA reads just their strides
+//           again (one vector per thread, 2 % of the row).  With many ties every thread reads its own stride
+//           again and keeps the first k ids it meets (it meets them in increasing order);
 //   select  one warp takes the k best of the list (by value, equal values by id), then the CTA fills up
 //           with the lowest ids among the entries equal to tau.
 // NaN is never chosen (the packed max and the comparisons ignore it); -0 and +0 are equal.
@@ -44,8 +45,8 @@ __global__ void __launch_bounds__(UT, 2) update_kernel(graft_update_params p, un
     __shared__ float s_cv[UCAP];
     __shared__ int s_ci[UCAP];
     __shared__ float s_wtop[UT / 32][UK];
-    __shared__ int s_red[UT / 32];
-    __shared__ int s_cnt, s_min, s_dup;
+    __shared__ int s_hot[UT];
+    __shared__ int s_cnt, s_nhot, s_min, s_dup;
     __shared__ float s_tau;
     __shared__ int s_top[UK];
 
@@ -64,13 +65,20 @@ __global__ void __launch_bounds__(UT, 2) update_kernel(graft_update_params p, un
     const uint16_t* row = reinterpret_cast<const uint16_t*>(p.logits) + (size_t)r * p.logits_stride_row;
     const uint4* row4 = reinterpret_cast<const uint4*>(row);
     const int nvec = V >> 3, ntail = V & 7;
-    if (tid == 0) s_cnt = 0;
+    if (tid == 0) { s_cnt = 0; s_nhot = 0; }
 
     // ---- pass 1: thread maxima
     uint32_t m0 = 0xff80ff80u, m1 = m0, m2 = m0, m3 = m0;          // -inf pairs
-    for (int v = tid; v < nvec; v += UT) {
-        const uint4 q = row4[v];
-        m0 = hmax2_bits(m0, q.x); m1 = hmax2_bits(m1, q.y); m2 = hmax2_bits(m2, q.z); m3 = hmax2_bits(m3, q.w);
+    // four independent 16-byte loads per thread in flight: the scan is bound by memory latency otherwise
+    constexpr int UNR = 4;
+    for (int v = tid; v < nvec; v += UNR * UT) {
+        uint4 q[UNR];
+#pragma unroll
+        for (int u = 0; u < UNR; ++u) q[u] = v + u * UT < nvec ? __ldg(row4 + v + u * UT) : make_uint4(0xff80ff80u, 0xff80ff80u, 0xff80ff80u, 0xff80ff80u);
+#pragma unroll
+        for (int u = 0; u < UNR; ++u) {
+            m0 = hmax2_bits(m0, q[u].x); m1 = hmax2_bits(m1, q[u].y); m2 = hmax2_bits(m2, q[u].z); m3 = hmax2_bits(m3, q[u].w);
+        }
     }
     m0 = hmax2_bits(hmax2_bits(m0, m1), hmax2_bits(m2, m3));
     float tm = fmaxf(lo_f(m0), hi_f(m0));
@@ -120,34 +128,78 @@ __global__ void __launch_bounds__(UT, 2) update_kernel(graft_update_params p, un
     const uint32_t t16 = *reinterpret_cast<const uint16_t*>(&tb);
     const uint32_t tau2 = t16 | (t16 << 16);
 
-    // ---- pass 2: candidates above tau, the thread's first k ids equal to tau
-    int eq[UK];
-    int n_eq = 0;
-    auto visit = [&](float f, int id) {
-        if (f > tau) {
-            const int at = atomicAdd(&s_cnt, 1);
-            if (at < UCAP) { s_cv[at] = f; s_ci[at] = id; }
-        } else if (f == tau && n_eq < k) {
-#pragma unroll
-            for (int q = 0; q < UK; ++q)
-                if (q == n_eq) eq[q] = id;
-            ++n_eq;
-        }
-    };
-    auto visit_word = [&](uint32_t w, int id) {
-        if (hmax2_bits(w, tau2) != tau2 || heq2_bits(w, tau2) != 0u) {
-            visit(lo_f(w), id);
-            visit(hi_f(w), id + 1);
-        }
-    };
-    for (int v = tid; v < nvec; v += UT) {
-        const uint4 q = row4[v];
-        visit_word(q.x, v * 8);
-        visit_word(q.y, v * 8 + 2);
-        visit_word(q.z, v * 8 + 4);
-        visit_word(q.w, v * 8 + 6);
+    // ---- pass 2: candidates above tau and the ids of the entries equal to tau.  Only threads whose maximum
+    // reached tau can hold either, and they are few (k-1 above tau, plus ties): their strides are read again by
+    // the whole CTA, one 16-byte vector per thread, out of L2.  Rows with so many ties at tau that this does not fit
+    // (a constant row, say) take the general path: every thread reads its stride again and keeps its first k ids.
+    const int iters = (nvec + UT - 1) / UT;               // vectors per stride
+    if (tm >= tau) {
+        const int at = atomicAdd(&s_nhot, 1);
+        s_hot[at] = tid;
     }
-    if (tid < ntail) visit(lo_f(row[(size_t)nvec * 8 + tid]), nvec * 8 + tid);
+    __syncthreads();
+    const int nhot = s_nhot;
+    const bool few = (long long)nhot * iters <= UT;
+    uint32_t eqmask = 0;                // few: elements of this thread's vector that equal tau
+    int vbase = 0;
+    int eq[UK];                         // general path: the thread's first k ids equal to tau, increasing
+    int n_eq = 0, ptr = 0;
+    int tail_eq = 0x7fffffff;
+    auto gt = [&](float f, int id) {
+        const int at = atomicAdd(&s_cnt, 1);
+        if (at < UCAP) { s_cv[at] = f; s_ci[at] = id; }
+    };
+    if (few) {
+        if (tid < nhot * iters) {
+            const int v = s_hot[tid / iters] + UT * (tid % iters);
+            if (v < nvec) {
+                const uint4 q = __ldg(row4 + v);
+                const uint32_t w[4] = {q.x, q.y, q.z, q.w};
+                vbase = v * 8;
+#pragma unroll
+                for (int e = 0; e < 8; ++e) {
+                    const float f = (e & 1) ? hi_f(w[e >> 1]) : lo_f(w[e >> 1]);
+                    if (f > tau) gt(f, vbase + e);
+                    else if (f == tau) eqmask |= 1u << e;
+                }
+            }
+        }
+    } else {
+        auto visit = [&](float f, int id) {
+            if (f > tau) gt(f, id);
+            else if (f == tau && n_eq < k) {
+#pragma unroll
+                for (int q = 0; q < UK; ++q)
+                    if (q == n_eq) eq[q] = id;
+                ++n_eq;
+            }
+        };
+        auto visit_word = [&](uint32_t w, int id) {
+            if (hmax2_bits(w, tau2) != tau2 || heq2_bits(w, tau2) != 0u) {
+                visit(lo_f(w), id);
+                visit(hi_f(w), id + 1);
+            }
+        };
+        for (int v = tid; v < nvec; v += 4 * UT) {
+            uint4 q[4];
+#pragma unroll
+            for (int u = 0; u < 4; ++u)      // NaN pairs past the end: never candidates
+                q[u] = v + u * UT < nvec ? __ldg(row4 + v + u * UT) : make_uint4(0x7fc07fc0u, 0x7fc07fc0u, 0x7fc07fc0u, 0x7fc07fc0u);
+#pragma unroll
+            for (int u = 0; u < 4; ++u) {
+                const int id = (v + u * UT) * 8;
+                visit_word(q[u].x, id);
+                visit_word(q[u].y, id + 2);
+                visit_word(q[u].z, id + 4);
+                visit_word(q[u].w, id + 6);
+            }
+        }
+    }
+    if (tid < ntail) {                  // the last V % 8 entries, one per thread (their ids are the row's largest)
+        const float f = lo_f(row[(size_t)nvec * 8 + tid]);
+        if (f > tau) gt(f, nvec * 8 + tid);
+        else if (f == tau) tail_eq = nvec * 8 + tid;
+    }
     __syncthreads();
     int n_gt = s_cnt;
     if (n_gt > UCAP) {                  // cannot happen for shapes the host accepts
@@ -178,32 +230,33 @@ __global__ void __launch_bounds__(UT, 2) update_kernel(graft_update_params p, un
     n_sel = n_gt < k ? n_gt : k;
     __syncthreads();
 
-    // ---- fill up with the lowest ids among the entries equal to tau
-    int ptr = 0;
+    // ---- fill up with the lowest ids among the entries equal to tau: every round each thread offers the lowest
+    // id it still holds and the CTA takes the minimum
     for (int j = n_sel; j < k; ++j) {
-        int cur = 0x7fffffff;
-#pragma unroll
-        for (int q = 0; q < UK; ++q)
-            if (q == ptr && q < n_eq) cur = eq[q];
-        int w = cur;
-#pragma unroll
-        for (int o = 16; o; o >>= 1) w = min(w, __shfl_xor_sync(0xffffffffu, w, o));
-        if (lane == 0) s_red[warp] = w;
+        if (tid == 0) s_min = 0x7fffffff;
         __syncthreads();
-        if (warp == 0) {
-            int z = lane < UT / 32 ? s_red[lane] : 0x7fffffff;
+        int cur = tail_eq;
+        if (few) {
+            if (eqmask) cur = vbase + __ffs(eqmask) - 1;
+        } else {
 #pragma unroll
-            for (int o = 16; o; o >>= 1) z = min(z, __shfl_xor_sync(0xffffffffu, z, o));
-            if (lane == 0) {
-                s_min = z;
-                s_top[j] = z == 0x7fffffff ? -1 : z;
-                if (z == 0x7fffffff) atomicOr(status, (unsigned)GRAFT_FLAG_NAN_SCORE);     // fewer than k entries that are not NaN
-            }
+            for (int q = 0; q < UK; ++q)
+                if (q == ptr && q < n_eq) cur = eq[q];
         }
+        if (cur != 0x7fffffff) atomicMin(&s_min, cur);
         __syncthreads();
-        if (cur == s_min && cur != 0x7fffffff) ++ptr;
-        __syncthreads();
+        const int won = s_min;
+        if (cur == won && cur != 0x7fffffff) {          // ids are unique: exactly one thread advances
+            if (few && eqmask) eqmask &= eqmask - 1;
+            else if (!few && ptr < n_eq) ++ptr;
+            else tail_eq = 0x7fffffff;
+        }
+        if (tid == 0) {
+            s_top[j] = won == 0x7fffffff ? -1 : won;
+            if (won == 0x7fffffff) atomicOr(status, (unsigned)GRAFT_FLAG_NAN_SCORE);     // fewer than k entries that are not NaN
+        }
     }
+    __syncthreads();
 
     // ---- results: the greedy id; the row of M unless a later node of the step carries the same token
     const int tok = p.tree_token[r];
