@@ -113,6 +113,12 @@ class VerifyStep:
         key = ("attn", self.Q.data_ptr(), self.Kc.data_ptr(), self.Vc.data_ptr(), variant, lse)
         G.launch("graft_tree_verify_attn", self.ctx, self._cached(key, make))
 
+    def update_adjacency(self, logits: torch.Tensor) -> None:
+        """logits: bf16 [B*T_max, V] on the device; refreshes M in place and writes target_next for accept()."""
+        key = ("update", logits.data_ptr())
+        G.launch("graft_update_adjacency", self.ctx, self._cached(key, lambda: G.update_adjacency_params(
+            logits=logits, tree_token=self.tree_token, tree_size=self.tree_size, M=self.M, target_next=self.target_next)))
+
     def accept(self) -> None:
         G.launch("graft_accept", self.ctx, self._cached("accept", lambda: G.accept_params(
             tree_token=self.tree_token, tree_parent=self.tree_parent, tree_anc=self.tree_anc, tree_size=self.tree_size,
