@@ -61,6 +61,8 @@ constexpr int NTHREADS = 384;
 constexpr int SMEM_DYN = 2 * TILE_BYTES + NSLOT * TILE_BYTES + 1024;   // Q (2 blocks) + ring + alignment slack
 constexpr int MAXSEG = 16;       // segments planned per round
 constexpr int kW2 = 5, kW1 = 4;        // cost units of a tile that carries two / one 128-row blocks (measured ratio ~1.25)
+constexpr int kOvh = 6 * kW2;          // units charged to the start of every item: new Q, pipeline refill, results of the last one
+                                       // cost a worker about as much as six tiles (measured: workers with an item boundary finished 5-8 us late)
 constexpr int kStreamMinTiles = 64;   // shorter per-CTA ranges use one piece per CTA instead of stream-K
 constexpr size_t SLOT_FLOATS = (size_t)BR * (D + 2);   // O[BR][D], then m2[BR], then l[BR]
 constexpr float kLog2e = 1.4426950408889634f;
@@ -109,7 +111,7 @@ __device__ __forceinline__ void seq_shape(const graft_attn_params& p, int G, int
 }
 // units of one KV head of a sequence
 __device__ __forceinline__ long long head_units(int ntiles, int nrb, int wlast) {
-    return nrb > 0 ? (long long)ntiles * (kW2 * (nrb - 1) + wlast) : 0;
+    return nrb > 0 ? (long long)ntiles * (kW2 * (nrb - 1) + wlast) + (long long)nrb * kOvh : 0;
 }
 
 // An item of ntiles tiles in pieces of about `per` tiles: nsplit equal, non-empty pieces of plen tiles.
@@ -204,8 +206,16 @@ __device__ __forceinline__ void choose_cut(const graft_attn_params& p, int G, in
 
 // position and weight of item (h, rb) of a sequence on the unit axis
 __device__ __forceinline__ void item_span(const SeqInfo& si, int h, int rb, long long& U, int& w) {
-    U = si.base + (long long)h * head_units(si.ntiles, si.nrb, si.wlast) + (long long)rb * si.ntiles * kW2;
+    U = si.base + (long long)h * head_units(si.ntiles, si.nrb, si.wlast) + (long long)rb * ((long long)si.ntiles * kW2 + kOvh);
     w = rb < si.nrb - 1 ? kW2 : si.wlast;
+}
+// An item that starts at unit U: tile 0 owns the kOvh start-up units and its own w, tile t >= 1 starts at U + kOvh + t * w.
+// Number of tiles whose first unit lies below g.
+__device__ __forceinline__ long long tiles_below(long long g, long long U, int w) {
+    if (g <= U) return 0;
+    const long long a = g - U - kOvh;
+    const long long c = a > 0 ? (a + w - 1) / w : 0;
+    return c < 1 ? 1 : c;
 }
 __device__ __forceinline__ int item_id(const graft_attn_params& p, int b, int h, int rb) { return ((b * p.Hkv + h) << 3) | rb; }
 
@@ -241,15 +251,14 @@ __device__ __forceinline__ void plan_round(const TcArgs& a, int G, int worker, b
         // walk the items of this sequence from the one that holds unit g
         int h = (int)((g - si.base) / hu);
         const long long rem = (g - si.base) % hu;
-        int rb = (int)(rem / ((long long)si.ntiles * kW2));
+        int rb = (int)(rem / ((long long)si.ntiles * kW2 + kOvh));
         if (rb > si.nrb - 1) rb = si.nrb - 1;
         while (g < g_hi && g < seq_end && n < MAXSEG) {
             long long U;
             int w;
             item_span(si, h, rb, U, w);
-            const long long item_end = U + (long long)si.ntiles * w;
-            long long t_lo = (g - U + w - 1) / w, t_hi = (g_hi - U + w - 1) / w;
-            if (t_lo < 0) t_lo = 0;
+            const long long item_end = U + kOvh + (long long)si.ntiles * w;
+            long long t_lo = tiles_below(g, U, w), t_hi = tiles_below(g_hi, U, w);
             if (t_hi > si.ntiles) t_hi = si.ntiles;
             if (t_lo < t_hi) {
                 const bool whole = t_lo == 0 && t_hi == si.ntiles;
@@ -1780,7 +1789,8 @@ __global__ void __launch_bounds__(kMergeWarps * 32, 2) merge_streamk_kernel(TcAr
         int w;
         item_span(si, h, rb, U, w);
         c_first = (int)(U / per);
-        nparts = (int)((U + (long long)(si.ntiles - 1) * w) / per) - c_first + 1;
+        const long long last = si.ntiles > 1 ? U + kOvh + (long long)(si.ntiles - 1) * w : U;      // first unit of the last tile
+        nparts = (int)(last / per) - c_first + 1;
     }
     if (nparts <= 1) continue;             // one CTA had the whole item and wrote the final rows
     // stream-K: part i lives in CTA c_first + i, in the slot whose descriptor names this item (none if
