@@ -17,30 +17,25 @@
 // by every CTA and by the merge kernel: no communication, no atomics on floats, no waiting between
 // CTAs, bit-reproducible results for a given GPU model.
 //
-// Warp roles inside a CTA:
+// Three kernels share this schedule, the TMA / tcgen05 / TMEM mechanics and the merge kernel:
+//   attn_tc_kernel       one CTA per SM holds both 128-row halves of an item (below);
+//   attn_tc_pair_kernel  a cluster of two CTAs, tcgen05.mma.cta_group::2 over the 256 rows, the K/V tile split
+//                        between the two shared memories (the default when a KV head carries more than 256 rows);
+//   attn_tc_rb_kernel    one 128-row block per CTA, partner CTAs fetch the same tiles and share them through L2
+//                        (the default otherwise).
+// A worker of the cut is a CTA in the first kernel and the CTA pair (2w, 2w+1) in the other two.
+//
+// Warp roles inside a CTA of attn_tc_kernel:
 //   warp 0      TMA producer: K and V tiles (two 64-column boxes each, 128-byte swizzle) into a
 //               5-slot ring of 32 KB buffers, one mbarrier pair (full / empty) per slot; the ring runs
 //               ahead across segment boundaries
 //   warp 1      MMA issuer: S = Q K^T (8 x m128 n128 k16, both operands from shared memory) and
 //               O += P V (8 x m128 n128 k16, P from TMEM, V as an MN-major operand); owns TMEM
-//   warps 2-3   Q stagers: copy the item's Q rows into shared memory (swizzled, K-major); for the next
-//               segment they do so as soon as the current segment's last Q K^T has completed (the MMA issuer
-//               commits a barrier right behind it), i.e. while the last softmax, P V and result write-out run
+//   warps 2-3   Q stagers: fetch the item's Q rows into shared memory (by TMA when H_q / H_kv divides 128, else
+//               16-byte asynchronous copies, swizzled, K-major); for the next segment they do so as soon as the
+//               current segment's last Q K^T has completed (the MMA issuer commits a barrier right behind it)
 //   warps 4-7   softmax of row block 0: thread i <-> TMEM lane i <-> row i; write results
 //   warps 8-11  softmax of row block 1
-// The two row blocks ping-pong: while one block's softmax runs on the SIMT pipes, the tensor pipe
-// works on the other block (its P V of this tile, then its Q K^T of the next).  TMEM columns:
-// S0 [0,128) S1 [128,256) O0 [256,384) O1 [384,512); P (bf16) overwrites the first 64 columns of
-// its S.  tcgen05.mma instructions of one thread execute in issue order, so the Q K^T that refills S
-// may be issued right behind the P V that reads P from it, and "S of tile j+1 is ready" implies
-// "P V of tile j is complete" (O is quiescent whenever a softmax thread rescales it).
-//
-// Softmax keeps a reference maximum per row and rescales O only when the maximum grows by more
-// than 2^8 (P then stays below 256, harmless in bf16/fp32); the row sum absorbs the same factor.
-// The ancestor bitmask of a row lives in one 64-bit register and is applied only in tiles that
-// reach past the cached prefix.  Cache slots at or past L_b + T_b inside the last tile are masked in S
-// and their V rows are zeroed in shared memory (0 x NaN would otherwise poison the accumulator).
-//
 // Every mbarrier wait is bounded: on a timeout the kernel sets GRAFT_FLAG_WAIT_TIMEOUT, stops
 // waiting anywhere in the CTA, drains its outstanding copies, frees TMEM and returns.
 #include <cuda.h>
