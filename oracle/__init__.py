@@ -153,7 +153,8 @@ def tree_attn(Q, Kc, Vc, seq_len, tree_size, tree_anc, scale, rows: Optional[np.
     if rows is None:
         nt = lib().orc_tree_attn(C.byref(a))
     else:
-        rows = np.ascontiguousarray(rows, np.int32).reshape(-1, 3)
+        # every row once: the C loop hands rows to threads, and a row listed twice would be written by two of them at once
+        rows = np.unique(np.ascontiguousarray(rows, np.int32).reshape(-1, 3), axis=0)
         nt = lib().orc_tree_attn_rows(C.byref(a), C.c_int(len(rows)), _p(rows, _i32p, np.int32))
     return dict(O=O, LSE=LSE, rowsum=rowsum, threads=int(nt))
 

@@ -23,7 +23,8 @@ extern "C" int graft_create(graft_ctx** out, int device, void* workspace, size_t
     if (major != 10) { cudaSetDevice(prev); return GRAFT_ERR_UNSUPPORTED; }   // sm_100a code only
     int rc = graft_attn_mma_init();
     if (rc == GRAFT_OK) rc = graft_attn_tc_init();
-    if (rc == GRAFT_OK && cudaMemset(workspace, 0, GRAFT_WS_HEADER) != cudaSuccess) rc = GRAFT_ERR_CUDA;
+    // the whole workspace starts at zero: status word, and the arrival counters of the attention kernels' merge
+    if (rc == GRAFT_OK && cudaMemset(workspace, 0, workspace_bytes) != cudaSuccess) rc = GRAFT_ERR_CUDA;
     if (rc == GRAFT_OK && cudaDeviceSynchronize() != cudaSuccess) rc = GRAFT_ERR_CUDA;
     cudaSetDevice(prev);
     if (rc != GRAFT_OK) return rc;
@@ -34,6 +35,7 @@ extern "C" int graft_create(graft_ctx** out, int device, void* workspace, size_t
     c->ws = workspace;
     c->ws_bytes = workspace_bytes;
     c->status = static_cast<unsigned*>(workspace);
+    c->epoch = 0;
     *out = c;
     return GRAFT_OK;
 }
