@@ -218,6 +218,9 @@ __device__ __forceinline__ long long tiles_below(long long g, long long U, int w
     return c < 1 ? 1 : c;
 }
 __device__ __forceinline__ int item_id(const graft_attn_params& p, int b, int h, int rb) { return ((b * p.Hkv + h) << 3) | rb; }
+// what a slot descriptor holds: the item, stamped with the call's number, so that a descriptor left by an earlier call
+// (a worker that has not yet reset its own in this call) never matches
+__device__ __forceinline__ int item_tag(const TcArgs& a, int id) { return id | (int)((a.epoch & 0x7fu) << 24); }
 
 struct Seg {
     int b, h, rb;            // item
@@ -287,7 +290,7 @@ __device__ __forceinline__ void plan_round(const TcArgs& a, int G, int worker, b
                         if (lo < hi) ++sg.nparts;
                     }
                     pl.seg[n] = sg;
-                    if (!whole && write_desc) a.desc[sg.slot] = item_id(p, si.b, h, rb);
+                    if (!whole && write_desc) a.desc[sg.slot] = item_tag(a, item_id(p, si.b, h, rb));
                 }
                 if (!whole) ++n_partial;
                 ++n;
@@ -339,7 +342,7 @@ __device__ __forceinline__ void plan_first(const TcArgs& a, int G, int worker, i
                 sg.slot = nsplit == 1 ? -1 : 2 * worker;
                 sg.c_first = worker - sp;
                 sg.c_span = sg.nparts = nsplit;
-                if (nsplit > 1 && write_desc) a.desc[sg.slot] = item_id(p, sg.b, sg.h, sg.rb);
+                if (nsplit > 1 && write_desc) a.desc[sg.slot] = item_tag(a, item_id(p, sg.b, sg.h, sg.rb));
                 pl.seg[0] = sg;
                 pl.nseg = 1;
             }
@@ -1349,7 +1352,7 @@ __device__ __forceinline__ void softmax_rows_split(const TcArgs& a, const Plan& 
             if (*merge_flag) {
                 __threadfence();                          // the other parts' stores are visible now
                 // every thread merges its own 64 columns of its own row, part after part (few parts: see the launch code)
-                const int id = item_id(p, sg.b, sg.h, sg.rb);
+                const int id = item_tag(a, item_id(p, sg.b, sg.h, sg.rb));
                 float M = -CUDART_INF_F;
                 for (int c = sg.c_first; c < sg.c_first + sg.c_span; ++c) {
                     const int sl = __ldcg(a.desc + 2 * c) == id ? 2 * c : (__ldcg(a.desc + 2 * c + 1) == id ? 2 * c + 1 : -1);      // from L2: an earlier merge of this CTA may have cached the line
@@ -1886,7 +1889,7 @@ __global__ void __launch_bounds__(kMergeWarps * 32, 2) merge_streamk_kernel(TcAr
     const int rb = r / BR, rl = r % BR;
     // the partial slots that hold pieces of this item, from the same cut as in the attention kernel
     int nparts, c_first = 0, piece_cta0 = 0;
-    const int id = item_id(p, b, h, rb);
+    const int id = item_tag(a, item_id(p, b, h, rb));
     if (pieces) {
         int nsplit, plen;
         piece_shape(si.ntiles, per, nsplit, plen);
@@ -2050,6 +2053,7 @@ bool graft_attn_tc_pair_supported(const graft_ctx* ctx, const graft_attn_params*
 
 bool graft_attn_tc_supported(const graft_ctx* ctx, const graft_attn_params* p) {
     if (p->d != D) return false;
+    if ((long long)p->B * p->Hkv * 8 >= (1ll << 24)) return false;      // item ids share a word with the call stamp
     // TMA: 16-byte aligned base and strides (checked by the caller), strides below 2^40 bytes
     if (p->kv_stride_s * 2 >= (1ll << 40) || p->kv_stride_h * 2 >= (1ll << 40) || p->kv_stride_b * 2 >= (1ll << 40)) return false;
     if (p->kv_stride_s == 0 || p->kv_stride_h == 0 || p->kv_stride_b == 0) return false;

@@ -340,6 +340,34 @@ def test_one_long_sequence_among_short_ones(orc, G, Step, variant):
     full_case(orc, G, Step, w, variant, rows=rows)
 
 
+@pytest.mark.parametrize("variant", ["auto", "pair", "l2pair"])
+def test_repeated_calls_on_one_context(orc, G, Step, variant):
+    """The kernels that merge in place keep arrival counters and slot descriptors in the workspace across calls: the
+    same call three times, then a different batch on the same context, all exact and the repeats bit-identical."""
+    rng = np.random.default_rng(29)
+    parents = [W.random_tree_parents(rng, 24) for _ in range(8)]
+    w = W.custom(parents, Hq=32, Hkv=8, d=128, L=[700, 650, 900, 300, 1200, 800, 750, 1000], T_max=32, seed=29)
+    tree = orc.build_tree(w)
+    W.make_qkv(w, tree["tree_size"], poison=True)
+    vs = Step(w)
+    vs.build()
+    outs = []
+    for _ in range(3):
+        vs.O.fill_(float("nan"))
+        vs.attn(variant_id(G, variant, w))
+        torch.cuda.synchronize()
+        check_attn(orc, w, vs, tree)
+        outs.append(vs.O.cpu().view(torch.int16).numpy().copy())
+    assert (outs[0] == outs[1]).all() and (outs[0] == outs[2]).all()
+    # other (shorter: the cache is poisoned past the old ends) lengths, same buffers
+    vs.seq_len[:] = torch.tensor([5, 600, 64, 300, 127, 128, 129, 1], dtype=torch.int32)
+    w.seq_len = vs.seq_len.cpu().numpy().copy()
+    vs.attn(variant_id(G, variant, w))
+    torch.cuda.synchronize()
+    check_attn(orc, w, vs, tree)
+    assert vs.ctx.device_status() == 0
+
+
 def test_one_and_two_block_items_mixed(orc, G, Step):
     """G = 16 with tree sizes whose last row block has at most / more than 128 rows, ragged lengths:
     items of different cost per tile on the cut axis, several row blocks per KV head."""
