@@ -1052,6 +1052,11 @@ __device__ __forceinline__ void tma_pair_4d(uint32_t dst, const CUtensorMap* map
     asm volatile("cp.async.bulk.tensor.4d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4, %5}], [%6];"
                  ::"r"(dst), "l"(map), "r"(x), "r"(y), "r"(z), "r"(w), "r"(cluster_bar) : "memory");
 }
+// the same with an L2 eviction policy: K/V bytes are read once, so they should leave L2 before the partials do
+__device__ __forceinline__ void tma_pair_4d_hint(uint32_t dst, const CUtensorMap* map, int x, int y, int z, int w, uint32_t cluster_bar, uint64_t policy) {
+    asm volatile("cp.async.bulk.tensor.4d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint [%0], [%1, {%2, %3, %4, %5}], [%6], %7;"
+                 ::"r"(dst), "l"(map), "r"(x), "r"(y), "r"(z), "r"(w), "r"(cluster_bar), "l"(policy) : "memory");
+}
 __device__ __forceinline__ void tma_pair_5d(uint32_t dst, const CUtensorMap* map, int x, int y, int z, int w, int v, uint32_t cluster_bar) {
     asm volatile("cp.async.bulk.tensor.5d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4, %5, %6}], [%7];"
                  ::"r"(dst), "l"(map), "r"(x), "r"(y), "r"(z), "r"(w), "r"(v), "r"(cluster_bar) : "memory");
@@ -1464,6 +1469,8 @@ attn_tc_pair_kernel(const __grid_constant__ CUtensorMap kmap, const __grid_const
         if (warp == 0) {
             // =============================== K/V producer (both CTAs) ===============================
             if (lane == 0) {
+                uint64_t stream_once;
+                asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(stream_once));
                 for (int si = 0; si < nseg; ++si) {
                     const Seg sg = plan.seg[si];
                     for (int t = sg.tile_lo; t < sg.tile_hi; ++t, ++jt) {
@@ -1475,9 +1482,9 @@ attn_tc_pair_kernel(const __grid_constant__ CUtensorMap kmap, const __grid_const
                         const uint32_t dst = sRing + slot * P_SLOT_BYTES;
                         const uint32_t fb = leader_bar(PB_FULL + slot);
                         // 64 keys of the K tile, all of d (two 64-column boxes); all keys of the V tile, 64 columns of d
-                        tma_pair_4d(dst, &kmap, 0, key0 + 64 * (int)rank, sg.h, sg.b, fb);
-                        tma_pair_4d(dst + P_HALF_TILE / 2, &kmap, 64, key0 + 64 * (int)rank, sg.h, sg.b, fb);
-                        tma_pair_4d(dst + P_HALF_TILE, &vmap, 64 * (int)rank, key0, sg.h, sg.b, fb);
+                        tma_pair_4d_hint(dst, &kmap, 0, key0 + 64 * (int)rank, sg.h, sg.b, fb, stream_once);
+                        tma_pair_4d_hint(dst + P_HALF_TILE / 2, &kmap, 64, key0 + 64 * (int)rank, sg.h, sg.b, fb, stream_once);
+                        tma_pair_4d_hint(dst + P_HALF_TILE, &vmap, 64 * (int)rank, key0, sg.h, sg.b, fb, stream_once);
                     }
                 }
             }
