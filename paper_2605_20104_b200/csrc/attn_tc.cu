@@ -1853,7 +1853,7 @@ attn_tc_rb_kernel(const __grid_constant__ CUtensorMap kmap, const __grid_constan
 // same cut as in the attention kernel.
 constexpr int kMergeWarps = 8;       // warps per CTA; rows per CTA is a launch parameter (8: one per warp, or 32)
 
-__global__ void __launch_bounds__(kMergeWarps * 32, 2) merge_streamk_kernel(TcArgs a, int rows_per_cta, unsigned* status) {
+__global__ void __launch_bounds__(kMergeWarps * 32, 4) merge_streamk_kernel(TcArgs a, int rows_per_cta, unsigned* status) {
     asm volatile("griddepcontrol.wait;" ::: "memory");      // launched early: nothing is read before the attention kernel is complete
     const graft_attn_params& p = a.p;
     const int G = a.G;
@@ -1941,10 +1941,10 @@ __global__ void __launch_bounds__(kMergeWarps * 32, 2) merge_streamk_kernel(TcAr
         }
         den += wgt * l;
         const int cnt = min(32, nparts - i0);
-        for (int j0 = 0; j0 < cnt; j0 += 16) {      // 16 partial rows in flight per round
-            float4 x[16];
+        for (int j0 = 0; j0 < cnt; j0 += 8) {       // 8 partial rows in flight per round and four CTAs per SM: the kernel is bound by
+            float4 x[8];                              // the memory round trips in flight (two CTAs of 123 registers: +4 us on four 64K sequences)
 #pragma unroll
-            for (int j = 0; j < 16; ++j)
+            for (int j = 0; j < 8; ++j)
                 if (j0 + j < cnt) {
                     // the owner lane of part j0 + j knows whether it exists; a missing part has weight 0
                     const unsigned long long pbj = __shfl_sync(0xffffffffu, (unsigned long long)my_pb, j0 + j);
@@ -1952,7 +1952,7 @@ __global__ void __launch_bounds__(kMergeWarps * 32, 2) merge_streamk_kernel(TcAr
                                : make_float4(0.f, 0.f, 0.f, 0.f);
                 }
 #pragma unroll
-            for (int j = 0; j < 16; ++j)
+            for (int j = 0; j < 8; ++j)
                 if (j0 + j < cnt) {
                     const float wj = __shfl_sync(0xffffffffu, wgt, j0 + j);
                     acc[0] += wj * x[j].x; acc[1] += wj * x[j].y; acc[2] += wj * x[j].z; acc[3] += wj * x[j].w;
