@@ -1047,12 +1047,8 @@ __device__ __forceinline__ void mbar_wait_cluster(uint32_t bar, uint32_t parity,
         }
     }
 }
-// copies whose completion is counted on a barrier of the pair's leader
-__device__ __forceinline__ void tma_pair_4d(uint32_t dst, const CUtensorMap* map, int x, int y, int z, int w, uint32_t cluster_bar) {
-    asm volatile("cp.async.bulk.tensor.4d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4, %5}], [%6];"
-                 ::"r"(dst), "l"(map), "r"(x), "r"(y), "r"(z), "r"(w), "r"(cluster_bar) : "memory");
-}
-// the same with an L2 eviction policy: K/V bytes are read once, so they should leave L2 before the partials do
+// copies whose completion is counted on a barrier of the pair's leader; K/V tiles carry an L2 eviction policy: they are
+// read once, so they should leave L2 before the partials do
 __device__ __forceinline__ void tma_pair_4d_hint(uint32_t dst, const CUtensorMap* map, int x, int y, int z, int w, uint32_t cluster_bar, uint64_t policy) {
     asm volatile("cp.async.bulk.tensor.4d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint [%0], [%1, {%2, %3, %4, %5}], [%6], %7;"
                  ::"r"(dst), "l"(map), "r"(x), "r"(y), "r"(z), "r"(w), "r"(cluster_bar), "l"(policy) : "memory");
@@ -1060,17 +1056,6 @@ __device__ __forceinline__ void tma_pair_4d_hint(uint32_t dst, const CUtensorMap
 __device__ __forceinline__ void tma_pair_5d(uint32_t dst, const CUtensorMap* map, int x, int y, int z, int w, int v, uint32_t cluster_bar) {
     asm volatile("cp.async.bulk.tensor.5d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4, %5, %6}], [%7];"
                  ::"r"(dst), "l"(map), "r"(x), "r"(y), "r"(z), "r"(w), "r"(v), "r"(cluster_bar) : "memory");
-}
-// D[tmem of both CTAs] (+)= A * B over the pair; issued by one thread of the leader
-__device__ __forceinline__ void mma_pair_ss(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc, uint32_t accumulate) {
-    asm volatile("{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
-                 "tcgen05.mma.cta_group::2.kind::f16 [%0], %1, %2, %3, p;\n\t}"
-                 ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate) : "memory");
-}
-__device__ __forceinline__ void mma_pair_ts(uint32_t d_tmem, uint32_t a_tmem, uint64_t b_desc, uint32_t idesc, uint32_t accumulate) {
-    asm volatile("{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
-                 "tcgen05.mma.cta_group::2.kind::f16 [%0], [%1], %2, %3, p;\n\t}"
-                 ::"r"(d_tmem), "r"(a_tmem), "l"(b_desc), "r"(idesc), "r"(accumulate) : "memory");
 }
 // The eight MMAs of one tile as one run of instructions (the issuing warp shares its scheduler with two busy
 // softmax warps, so every instruction it does not need is time the tensor pipe waits): descriptors advance by
