@@ -207,3 +207,32 @@ def update_adjacency(logits_bits, tree_token, tree_size, M, k: int) -> dict:
                                        _p(tt, _i32p, np.int32), _p(ts, _i32p, np.int32), _p(Mn, _i32p, np.int32),
                                        _p(tn, _i32p, np.int32))
     return dict(M=Mn, target_next=tn, flags=int(flags))
+
+
+def retrieve_envelope(root_token, M, env_parent, env_rank, root_stride: int = 1) -> dict:
+    """root_token: int32, request b's root at [b * root_stride]; M: int32 [V, k]; the template as parent / rank
+    lists.  Returns env_token [B, N_env] and the flag word."""
+    rt = np.ascontiguousarray(root_token, np.int32).reshape(-1)
+    Mc = np.ascontiguousarray(M, np.int32)
+    ep, er = _arr(env_parent, np.int32), _arr(env_rank, np.int32)
+    V, k = Mc.shape
+    B = (len(rt) + root_stride - 1) // root_stride
+    out = np.empty((B, len(ep)), np.int32)
+    fn = lib().orc_retrieve_envelope
+    fn.restype = C.c_uint
+    flags = fn(C.c_int(B), C.c_int(V), C.c_int(k), C.c_int(len(ep)), _p(rt, _i32p, np.int32), C.c_long(root_stride),
+               _p(Mc, _i32p, np.int32), _p(ep, _i32p, np.int32), _p(er, _i32p, np.int32), _p(out, _i32p, np.int32))
+    return dict(env_token=out, flags=int(flags))
+
+
+def path_indices(tree_parent, tree_size, D_max: int) -> dict:
+    """tree_parent: int32 [B, T_max]; returns path_index [B, T_max, D_max], n_paths [B] and the flag word."""
+    tp, ts = _arr(tree_parent, np.int32), _arr(tree_size, np.int32)
+    B, T = tp.shape
+    out = np.empty((B, T, D_max), np.int32)
+    n = np.empty(B, np.int32)
+    fn = lib().orc_path_indices
+    fn.restype = C.c_uint
+    flags = fn(C.c_int(B), C.c_int(T), C.c_int(D_max), _p(tp, _i32p, np.int32), _p(ts, _i32p, np.int32),
+               _p(out, _i32p, np.int32), _p(n, _i32p, np.int32))
+    return dict(path_index=out, n_paths=n, flags=int(flags))

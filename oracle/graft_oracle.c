@@ -14,7 +14,11 @@
  * the paper's stage budgets 8+52 / 24+36 / 40+20 and template depth histograms; the
  * closed form x_u = M[x_parent(u), r_u]; Propositions 1 and 2 (monotone accepted length);
  * the adjacency update against a library stable sort, against softmax probabilities, a hand-worked
- * row with ties / NaN / -inf, and the sequential definition of the duplicate-token winner.
+ * row with ties / NaN / -inf, and the sequential definition of the duplicate-token winner;
+ * the retrieval envelope against the lookup equation folded along explicit rank paths, a shift matrix
+ * with a closed form, the tree assembly's own lookups and the printed shape of the full template
+ * (80 nodes, 8+16+14+11+8+7+6+5+5 over depths 1..9); the candidate-path table against a top-down
+ * enumeration, chain and star trees, and acceptance written over paths.
  * Parity unpinned: nothing beyond the printed per-depth counts fixes the retrieval
  * templates' exact rank paths; they are inputs here, not computed.
  */
@@ -460,5 +464,69 @@ unsigned orc_update_adjacency(int B, int T_max, int V, int k, const uint16_t *lo
         }
     }
     free(s); free(taken); free(top);
+    return flags;
+}
+
+/* ------------------------------------------------------------------------------------------------
+ * Root-centred retrieval envelope (retrieval section, "Lightweight parallel retrieval"; template
+ * appendix, lookup equation x_u = M[x_F(u), r_u]): the tokens of every node of a static template,
+ * filled from the request's root token in template order.  The template is a list of nodes with a
+ * parent index inside the list (-1: child of the root) and a successor rank; a parent precedes its
+ * children, so one pass in list order has every parent token ready.  An empty row of M (-1) and a
+ * missing root make the whole subtree -1.  Root ids outside [-1, V) count as -1 (bad-token flag), and
+ * so do matrix entries outside [-1, V); a node whose parent index or rank is out of range gets -1
+ * (bad-template flag).  root_token[b * root_stride] is request b's root.
+ * ------------------------------------------------------------------------------------------------ */
+unsigned orc_retrieve_envelope(int B, int V, int k, int N_env, const int32_t *root_token, long root_stride, const int32_t *M,
+                               const int32_t *env_parent, const int32_t *env_rank, int32_t *env_token /* [B, N_env] */) {
+    unsigned flags = 0;
+    for (int b = 0; b < B; ++b) {
+        int32_t x_root = root_token[(size_t)b * root_stride];
+        if (x_root < -1 || x_root >= V) { x_root = -1; flags |= ORC_FLAG_BAD_TOKEN; }
+        int32_t *x = env_token + (size_t)b * N_env;
+        for (int u = 0; u < N_env; ++u) {
+            const int f = env_parent[u], r = env_rank[u];
+            if (f < -1 || f >= u || r < 0 || r >= k) { x[u] = -1; flags |= ORC_FLAG_BAD_TEMPLATE; continue; }
+            const int32_t x_f = f < 0 ? x_root : x[f];
+            int32_t v = x_f >= 0 ? M[(size_t)x_f * k + r] : -1;
+            if (v < -1 || v >= V) { v = -1; flags |= ORC_FLAG_BAD_TOKEN; }
+            x[u] = v;
+        }
+    }
+    return flags;
+}
+
+/* ------------------------------------------------------------------------------------------------
+ * Candidate-path indices (verification section: after flattening, "position IDs, ancestor mask, and
+ * candidate-path indices" are rebuilt): one row per leaf of the flattened tree, leaves in increasing
+ * node index, holding the node indices from the root (index 0) down to the leaf and then -1 up to
+ * D_max columns; rows past the last leaf hold -1.  n_paths[b] is the number of leaves.  A tree of size
+ * 0 has no paths.  A leaf deeper than D_max - 1 keeps the first D_max nodes of its path (bad-size flag).
+ * ------------------------------------------------------------------------------------------------ */
+unsigned orc_path_indices(int B, int T_max, int D_max, const int32_t *tree_parent, const int32_t *tree_size,
+                          int32_t *path_index /* [B, T_max, D_max] */, int32_t *n_paths /* [B] */) {
+    unsigned flags = 0;
+    int32_t *up = (int32_t *)malloc((size_t)(T_max + 1) * sizeof(int32_t));
+    for (int b = 0; b < B; ++b) {
+        const int32_t *par = tree_parent + (size_t)b * T_max;
+        int32_t *rows = path_index + (size_t)b * T_max * D_max;
+        for (int i = 0; i < T_max * D_max; ++i) rows[i] = -1;
+        int T = tree_size[b];
+        if (T < 0 || T > T_max) { T = 0; flags |= ORC_FLAG_BAD_SIZE; }
+        int n = 0;
+        for (int i = 0; i < T; ++i) {
+            int is_leaf = 1;
+            for (int j = i + 1; j < T; ++j)
+                if (par[j] == i) { is_leaf = 0; break; }
+            if (!is_leaf) continue;
+            int len = 0;
+            for (int j = i; j >= 0 && len <= T_max; j = par[j]) up[len++] = j;    /* leaf, ..., root */
+            if (len > D_max) flags |= ORC_FLAG_BAD_SIZE;
+            for (int c = 0; c < len && c < D_max; ++c) rows[(size_t)n * D_max + c] = up[len - 1 - c];
+            ++n;
+        }
+        n_paths[b] = n;
+    }
+    free(up);
     return flags;
 }

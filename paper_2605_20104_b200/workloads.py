@@ -95,6 +95,37 @@ def chains_template(lengths: Sequence[int]) -> Tuple[np.ndarray, np.ndarray]:
     return np.asarray(parent, np.int32), np.asarray(rank, np.int32)
 
 
+def template_rank_paths(parent: np.ndarray, rank: np.ndarray) -> List[Tuple[int, ...]]:
+    """(parent, rank) lists of a template -> the rank path of every node."""
+    paths: List[Tuple[int, ...]] = []
+    for f, r in zip(parent.tolist(), rank.tolist()):
+        paths.append((() if f < 0 else paths[f]) + (r,))
+    return paths
+
+
+def retrieval_envelope(templates: Sequence[Tuple[np.ndarray, np.ndarray]]) -> Tuple[np.ndarray, np.ndarray, List[np.ndarray]]:
+    """The smallest template that contains every node (rank path) of the given templates, and for each
+    of them the index of its nodes inside that envelope.  Envelope nodes are ordered by depth, then
+    lexicographically, so a parent always precedes its children."""
+    all_paths = [template_rank_paths(tp, tr) for tp, tr in templates]
+    union = sorted({q[:n] for ps in all_paths for q in ps for n in range(1, len(q) + 1)}, key=lambda q: (len(q), q))
+    index = {q: i for i, q in enumerate(union)}
+    env_parent, env_rank = paths_to_parent_rank(union) if union else (np.zeros(0, np.int32), np.zeros(0, np.int32))
+    return env_parent, env_rank, [np.asarray([index[q] for q in ps], np.int32) for ps in all_paths]
+
+
+def workload_envelope(w: "Workload") -> Tuple[np.ndarray, np.ndarray, np.ndarray]:
+    """Envelope of a workload's stage templates and the envelope index of every template node
+    (tmpl_env, laid out like tmpl_parent / tmpl_rank)."""
+    if w.tmpl_offset is None:
+        stages = [(w.tmpl_parent, w.tmpl_rank)]
+    else:
+        off = w.tmpl_offset.tolist()
+        stages = [(w.tmpl_parent[a:b], w.tmpl_rank[a:b]) for a, b in zip(off[:-1], off[1:])]
+    ep, er, maps = retrieval_envelope(stages)
+    return ep, er, (np.concatenate(maps).astype(np.int32) if maps else np.zeros(0, np.int32))
+
+
 DENSE60_WIDTHS = (8, 16, 14, 10, 7, 4)
 DENSE60_CAPS = (8, 4, 2, 1, 1, 1)
 
