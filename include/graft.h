@@ -6,7 +6,10 @@
  * target model's KV cache.  Per layer-step the caller runs, on one CUDA stream and without any host
  * synchronisation in between:
  *
+ *     graft_retrieve_envelope retrieval section: the root-centred template filled from M, on a side stream
+ *                             while the draft model runs (optional: graft_build_tree can do its own lookups)
  *     graft_build_tree        Algorithm 2 from "Resolve (K_draft, K_ret)" on: prune, graft, rebuild
+ *     graft_path_indices      Sec. 3.3: the candidate-path table of the flattened tree (optional output)
  *     [caller: QKV projection writes the tree tokens' K/V to cache slots L_b .. L_b + T_b - 1]
  *     graft_tree_verify_attn  Sec. 3.3: tree attention of the T tree tokens over cache + ancestors
  *     [caller: lm_head gives the target logits of the tree nodes]
@@ -148,9 +151,64 @@ typedef struct {
     int32_t* tree_src;           /* out [B, T_max] */
     uint64_t* tree_anc;          /* out [B, T_max], bit u of anc[t]: node u visible to node t */
     int32_t* tree_size;          /* out [B] */
+    /* optional: tokens of a precomputed retrieval envelope (graft_retrieve_envelope).  With env_token
+       set, template node u of the chosen stage takes env_token[b, tmpl_env[tmpl_offset[c] + u]]
+       instead of its own chain of lookups in M; tmpl_parent still gives the tree structure.  The
+       caller guarantees that the envelope node has the template node's rank path and that the
+       envelope was filled from this call's root tokens and M; an index outside [0, N_env) sets
+       GRAFT_FLAG_BAD_TEMPLATE and gives token -1. */
+    int N_env;
+    const int32_t* env_token;    /* [B, N_env] or NULL */
+    const int32_t* tmpl_env;     /* [N_tmpl] */
 } graft_build_params;
 
 int graft_build_tree(graft_ctx* ctx, const graft_build_params* p, void* stream);
+
+/* ---- graft_retrieve_envelope ----------------------------------------------------------------- */
+/*
+ * Root-centred retrieval envelope (retrieval section, "Lightweight parallel retrieval": the envelope is
+ * materialised in parallel with drafting and a stage-matched part of it is selected afterwards; template
+ * appendix: x_u = M[x_F(u), r_u], filled level by level from the root token).  The template is a list of
+ * N_env nodes, node u with env_parent[u] in [-1, u) (-1: child of the root) and env_rank[u] in [0, k).
+ * env_token[b, u] is the token of node u for request b; an empty row of M (-1) or a root of -1 makes
+ * the whole subtree -1.  Root ids and matrix entries outside [-1, V) count as -1 (GRAFT_FLAG_BAD_TOKEN);
+ * a node with a parent index or rank out of range gets -1 (GRAFT_FLAG_BAD_TEMPLATE).
+ * Request b's root is root_token[b * root_stride] (pass draft_token and N_max to read node 0 of the
+ * draft trees in place).  N_env <= 1024, k <= 16.  The call reads only the root tokens, M and the
+ * template, so it may run on another stream than the rest of the step; the caller orders it before
+ * graft_build_tree (an event) and after the previous step's graft_update_adjacency.
+ */
+typedef struct {
+    int B, V, k, N_env;
+    const int32_t* root_token;   /* request b's root at [b * root_stride] */
+    int64_t root_stride;
+    const int32_t* M;            /* [V, k] */
+    const int32_t* env_parent;   /* [N_env] */
+    const int32_t* env_rank;     /* [N_env] */
+    int32_t* env_token;          /* out [B, N_env] */
+} graft_envelope_params;
+
+int graft_retrieve_envelope(graft_ctx* ctx, const graft_envelope_params* p, void* stream);
+
+/* ---- graft_path_indices ---------------------------------------------------------------------- */
+/*
+ * Candidate-path indices of the flattened tree (Sec. 3.3: "rebuilds the standard tree position IDs,
+ * ancestor mask, and candidate-path indices"): one row per leaf, leaves in increasing node index; a row
+ * lists the node indices from the root (0) to the leaf and then -1 up to D_max columns; rows past the
+ * last leaf hold -1.  n_paths[b] = number of leaves (0 for an empty tree).  A leaf deeper than
+ * D_max - 1 keeps the first D_max nodes of its path and sets GRAFT_FLAG_BAD_SIZE, as does a
+ * tree_size outside [0, T_max] (no paths).  tree_parent must satisfy parent[i] < i (as
+ * graft_build_tree writes it).  T_max <= 64, 1 <= D_max <= 64.
+ */
+typedef struct {
+    int B, T_max, D_max;
+    const int32_t* tree_parent;  /* [B, T_max] */
+    const int32_t* tree_size;    /* [B] */
+    int32_t* path_index;         /* out [B, T_max, D_max] */
+    int32_t* n_paths;            /* out [B] */
+} graft_paths_params;
+
+int graft_path_indices(graft_ctx* ctx, const graft_paths_params* p, void* stream);
 
 /* ---- graft_tree_verify_attn ------------------------------------------------------------------ */
 /*

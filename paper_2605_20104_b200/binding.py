@@ -29,7 +29,8 @@ ATTN_AUTO, ATTN_MMA_SYNC, ATTN_TCGEN05, ATTN_TCGEN05_1SM, ATTN_TCGEN05_2SM, ATTN
 
 EXPORTS = ("graft_workspace_bytes", "graft_create", "graft_destroy", "graft_status_string", "graft_device_status",
            "graft_build_tree", "graft_tree_verify_attn", "graft_accept", "graft_compact_kv",
-           "graft_noalloc_scratch_bytes", "graft_tree_verify_attn_noalloc", "graft_update_adjacency")
+           "graft_noalloc_scratch_bytes", "graft_tree_verify_attn_noalloc", "graft_update_adjacency",
+           "graft_retrieve_envelope", "graft_path_indices")
 
 _vp = C.c_void_p
 
@@ -40,7 +41,18 @@ class BuildParams(C.Structure):
                 [(n, _vp) for n in ("draft_token", "draft_parent", "draft_score", "n_draft", "seq_len", "M", "keep_count",
                                     "k_max", "ckpt_depth", "ckpt_keep", "ckpt_log_tau", "tmpl_offset", "tmpl_parent",
                                     "tmpl_rank", "tree_token", "tree_parent", "tree_pos", "tree_src", "tree_anc",
-                                    "tree_size")])
+                                    "tree_size")] +
+                [("N_env", C.c_int), ("env_token", _vp), ("tmpl_env", _vp)])
+
+
+class EnvelopeParams(C.Structure):
+    _fields_ = ([(n, C.c_int) for n in ("B", "V", "k", "N_env")] + [("root_token", _vp), ("root_stride", C.c_int64)] +
+                [(n, _vp) for n in ("M", "env_parent", "env_rank", "env_token")])
+
+
+class PathsParams(C.Structure):
+    _fields_ = ([(n, C.c_int) for n in ("B", "T_max", "D_max")] +
+                [(n, _vp) for n in ("tree_parent", "tree_size", "path_index", "n_paths")])
 
 
 class AttnParams(C.Structure):
@@ -82,7 +94,8 @@ _lib.graft_device_status.restype = C.c_int
 _lib.graft_device_status.argtypes = [_vp, _vp, C.POINTER(C.c_uint), C.c_int]
 for _name, _typ in (("graft_build_tree", BuildParams), ("graft_tree_verify_attn", AttnParams),
                     ("graft_accept", AcceptParams), ("graft_compact_kv", CompactParams),
-                    ("graft_update_adjacency", UpdateParams)):
+                    ("graft_update_adjacency", UpdateParams), ("graft_retrieve_envelope", EnvelopeParams),
+                    ("graft_path_indices", PathsParams)):
     getattr(_lib, _name).restype = C.c_int
     getattr(_lib, _name).argtypes = [_vp, C.POINTER(_typ), _vp]
 
@@ -165,7 +178,9 @@ def build_tree_params(*, mode: int, K_max: int, V: int, k: int, S_cap: int,
                      draft_token, draft_parent, draft_score, n_draft, seq_len, M=None, keep_count=None, k_max=None,
                      gate_depth: int = 0, node_threshold: float = 0.0, ckpt_depth=None, ckpt_keep=None,
                      ckpt_log_tau=None, tmpl_offset=None, tmpl_parent=None, tmpl_rank=None,
-                     tree_token, tree_parent, tree_pos, tree_src, tree_anc, tree_size) -> None:
+                     tree_token, tree_parent, tree_pos, tree_src, tree_anc, tree_size,
+                     env_token=None, tmpl_env=None) -> BuildParams:
+    """env_token [B, N_env] / tmpl_env [N_tmpl]: take the grafted tokens from a precomputed retrieval envelope."""
     B, N_max = draft_token.shape
     T_max = tree_token.shape[1]
     i32, f32 = torch.int32, torch.float32
@@ -179,7 +194,9 @@ def build_tree_params(*, mode: int, K_max: int, V: int, k: int, S_cap: int,
                     ckpt_log_tau=_ptr(ckpt_log_tau, f32), tmpl_offset=_ptr(tmpl_offset, i32),
                     tmpl_parent=_ptr(tmpl_parent, i32), tmpl_rank=_ptr(tmpl_rank, i32),
                     tree_token=_ptr(tree_token, i32), tree_parent=_ptr(tree_parent, i32), tree_pos=_ptr(tree_pos, i32),
-                    tree_src=_ptr(tree_src, i32), tree_anc=_ptr(tree_anc, torch.int64), tree_size=_ptr(tree_size, i32))
+                    tree_src=_ptr(tree_src, i32), tree_anc=_ptr(tree_anc, torch.int64), tree_size=_ptr(tree_size, i32),
+                    N_env=0 if env_token is None else env_token.shape[1],
+                    env_token=_ptr(env_token, i32), tmpl_env=_ptr(tmpl_env, i32))
     return p
 
 
@@ -248,6 +265,36 @@ def update_adjacency_params(*, logits, tree_token, tree_size, M, target_next=Non
 
 def graft_update_adjacency(ctx: Context, **kw) -> None:
     launch("graft_update_adjacency", ctx, update_adjacency_params(**kw))
+
+
+def retrieve_envelope_params(*, root_token, M, env_parent, env_rank, env_token, root_stride: int = 1) -> EnvelopeParams:
+    """root_token: int32, request b's root at element b * root_stride (draft_token with root_stride = N_max reads the
+    draft trees' node 0 in place); env_token: int32 [B, N_env] out."""
+    i32 = torch.int32
+    B, N_env = env_token.shape
+    V, k = M.shape
+    assert M.is_contiguous() and env_token.is_contiguous() and env_parent.numel() == N_env and env_rank.numel() == N_env
+    assert root_token.numel() > (B - 1) * root_stride
+    return EnvelopeParams(B=B, V=V, k=k, N_env=N_env, root_token=_ptr(root_token, i32), root_stride=root_stride,
+                          M=_ptr(M, i32), env_parent=_ptr(env_parent, i32), env_rank=_ptr(env_rank, i32),
+                          env_token=_ptr(env_token, i32))
+
+
+def graft_retrieve_envelope(ctx: Context, **kw) -> None:
+    launch("graft_retrieve_envelope", ctx, retrieve_envelope_params(**kw))
+
+
+def path_indices_params(*, tree_parent, tree_size, path_index, n_paths) -> PathsParams:
+    """path_index: int32 [B, T_max, D_max] out; n_paths: int32 [B] out."""
+    i32 = torch.int32
+    B, T_max, D_max = path_index.shape
+    assert tree_parent.shape == (B, T_max) and path_index.is_contiguous()
+    return PathsParams(B=B, T_max=T_max, D_max=D_max, tree_parent=_ptr(tree_parent, i32), tree_size=_ptr(tree_size, i32),
+                       path_index=_ptr(path_index, i32), n_paths=_ptr(n_paths, i32))
+
+
+def graft_path_indices(ctx: Context, **kw) -> None:
+    launch("graft_path_indices", ctx, path_indices_params(**kw))
 
 
 def graft_accept(ctx: Context, **kw) -> None:

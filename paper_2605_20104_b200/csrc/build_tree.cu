@@ -3,7 +3,8 @@
 // Thread i owns draft node i, then template node i, then output node i.  Everything a node needs
 // from other nodes goes through shared memory; the only global traffic is one read of the draft
 // arrays, the level-wise gathers from the adjacency matrix (one dependent gather per template
-// depth: the critical path the paper attributes to retrieval), and one write of the outputs.
+// depth: the critical path the paper attributes to retrieval; with a precomputed envelope a single
+// gather), and one write of the outputs.
 #include <limits.h>
 #include <math_constants.h>
 #include "graft_internal.cuh"
@@ -187,7 +188,20 @@ __global__ void __launch_bounds__(kThreads) build_tree_kernel(graft_build_params
             s_opar[K_kept + u] = tp < 0 ? 0 : K_kept + tp;
             o_src[K_kept + u] = -1 - u;
         }
-        const int max_d = block_max_int(u < K_ret ? du : 0, s_i2);
+        if (a.env_token) {
+            // the envelope holds the token of every rank path already: one independent load per node
+            if (u < K_ret) {
+                int x = -1;
+                const int e = a.tmpl_env[t_lo + u];
+                if (e < 0 || e >= a.N_env) flags |= GRAFT_FLAG_BAD_TEMPLATE;
+                else if (ok) {
+                    x = a.env_token[(size_t)b * a.N_env + e];
+                    if (x < -1 || x >= a.V) { x = -1; flags |= GRAFT_FLAG_BAD_TOKEN; }
+                }
+                s_tok[K_kept + u] = x;
+            }
+        }
+        const int max_d = a.env_token ? 0 : block_max_int(u < K_ret ? du : 0, s_i2);
         for (int lvl = 1; lvl <= max_d; ++lvl) {
             if (u < K_ret && du == lvl) {
                 int x = -1;
@@ -233,6 +247,7 @@ extern "C" int graft_build_tree(graft_ctx* ctx, const graft_build_params* p, voi
         return GRAFT_ERR_INVALID_ARG;
     if (p->N_tmpl < 0 || p->n_ckpt < 0) return GRAFT_ERR_INVALID_ARG;
     if (p->mode != GRAFT_PRUNE_NONE && p->N_tmpl > 0 && (!p->M || !p->tmpl_parent || !p->tmpl_rank)) return GRAFT_ERR_INVALID_ARG;
+    if (p->env_token && (!p->tmpl_env || p->N_env <= 0)) return GRAFT_ERR_INVALID_ARG;
     if (p->mode == GRAFT_PRUNE_TOPK && !p->keep_count) return GRAFT_ERR_INVALID_ARG;
     if (p->mode == GRAFT_PRUNE_GATED &&
         (p->n_ckpt > 0 && (!p->ckpt_depth || !p->ckpt_keep || !p->ckpt_log_tau || !p->tmpl_offset)))

@@ -12,7 +12,7 @@ import numpy as np
 import torch
 
 from . import binding as G
-from .workloads import Workload
+from .workloads import Workload, workload_envelope
 
 
 def _dev(a, dtype=None, device="cuda"):
@@ -89,12 +89,48 @@ class VerifyStep:
             cache[key] = make()
         return cache[key]
 
-    def build(self) -> None:
-        G.launch("graft_build_tree", self.ctx, self._cached("build", self._build_params))
+    def retrieve_envelope(self, stream: Optional[torch.cuda.Stream] = None) -> None:
+        """Fills the retrieval envelope of the workload's templates from the draft trees' root tokens; on `stream`
+        (a side stream beside drafting) the next build() waits for it through an event."""
+        if not hasattr(self, "env_token"):
+            ep, er, te = workload_envelope(self.w)
+            self.env_parent, self.env_rank, self.tmpl_env = (_dev(a, device=self.dev) for a in (ep, er, te))
+            self.env_token = torch.empty(self.w.B, len(ep), dtype=torch.int32, device=self.dev) if len(ep) else None
+            self._env_event = torch.cuda.Event()
+        if self.env_token is None:          # the workload grafts nothing
+            return
+        params = self._cached("envelope", lambda: G.retrieve_envelope_params(
+            root_token=self.draft_token, root_stride=self.w.N_max, M=self.M, env_parent=self.env_parent,
+            env_rank=self.env_rank, env_token=self.env_token))
+        if stream is None:
+            G.launch("graft_retrieve_envelope", self.ctx, params)
+        else:
+            stream.wait_stream(torch.cuda.current_stream())
+            with torch.cuda.stream(stream):
+                G.launch("graft_retrieve_envelope", self.ctx, params)
+                self._env_event.record(stream)
+            torch.cuda.current_stream().wait_event(self._env_event)
 
-    def _build_params(self):
+    def path_indices(self, D_max: Optional[int] = None) -> None:
+        """Candidate-path table of the tree build() left: path_index [B, T_max, D_max], n_paths [B]."""
+        D = self.w.T_max if D_max is None else D_max
+        if getattr(self, "path_index", None) is None or self.path_index.shape[2] != D:
+            self.path_index = torch.empty(self.w.B, self.w.T_max, D, dtype=torch.int32, device=self.dev)
+            self.n_paths = torch.empty(self.w.B, dtype=torch.int32, device=self.dev)
+        G.launch("graft_path_indices", self.ctx, self._cached(("paths", self.path_index.data_ptr()), lambda: G.path_indices_params(
+            tree_parent=self.tree_parent, tree_size=self.tree_size, path_index=self.path_index, n_paths=self.n_paths)))
+
+    def build(self, from_envelope: bool = False) -> None:
+        """from_envelope: take the grafted tokens from the envelope retrieve_envelope() filled."""
+        if from_envelope and self.env_token is not None:
+            G.launch("graft_build_tree", self.ctx, self._cached("build_env", lambda: self._build_params(True)))
+        else:
+            G.launch("graft_build_tree", self.ctx, self._cached("build", self._build_params))
+
+    def _build_params(self, from_envelope: bool = False):
         w = self.w
-        return G.build_tree_params(mode=w.mode, K_max=w.K_max, V=w.V, k=w.k, S_cap=w.S_cap,
+        env = dict(env_token=self.env_token, tmpl_env=self.tmpl_env) if from_envelope else {}
+        return G.build_tree_params(**env, mode=w.mode, K_max=w.K_max, V=w.V, k=w.k, S_cap=w.S_cap,
                            draft_token=self.draft_token, draft_parent=self.draft_parent, draft_score=self.draft_score,
                            n_draft=self.n_draft, seq_len=self.seq_len, M=self.M, keep_count=self.keep_count,
                            k_max=self.k_max, gate_depth=w.gate_depth, node_threshold=w.node_threshold,
