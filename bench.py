@@ -197,6 +197,34 @@ def time_update(st, steps, warmup):
             "GBps": byts / (us * 1e-6) / 1e9, "l2": "rotating %d logits buffers" % n_rot}
 
 
+def time_index_kernels(st, steps, warmup):
+    """The small index kernels around tree assembly, each alone: the retrieval envelope, assembly with its own
+    lookups and from the envelope, and the candidate-path table (latency-bound launches of B CTAs)."""
+    vs = st["vs"]
+    vs.retrieve_envelope()
+    calls = {"build_tree": lambda: vs.build(), "path_indices": lambda: vs.path_indices(10)}
+    if vs.env_token is not None:
+        calls["retrieve_envelope"] = lambda: vs.retrieve_envelope()
+        calls["build_tree_from_envelope"] = lambda: vs.build(from_envelope=True)
+    out = {}
+    for name, fn in calls.items():
+        ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(steps)]
+        for _ in range(warmup):
+            fn()
+        torch.cuda.synchronize()
+        torch.cuda._sleep(int(3e6))
+        for a, b in ev:
+            a.record()
+            fn()
+            b.record()
+        torch.cuda.synchronize()
+        out[name + "_us"] = float(np.mean([a.elapsed_time(b) for a, b in ev])) * 1e3
+    out["envelope_nodes"] = 0 if vs.env_token is None else int(vs.env_token.shape[1])
+    vs.build()                       # leave the tree as the step built it
+    torch.cuda.synchronize()
+    return out
+
+
 def run_timed(st, steps):
     # keep the GPU busy for a moment so that the launch queue is full when the timed region starts
     torch.cuda._sleep(int(3e6))
@@ -426,6 +454,7 @@ def main():
         upd = time_update(st, min(args.steps, 50), 5)
         upd["frac_of_measured"] = upd["GBps"] / peak
         line["update_adjacency"] = upd
+        line["index_kernels"] = time_index_kernels(st, min(args.steps, 50), 5)
         extra = []
         del st
         torch.cuda.empty_cache()
