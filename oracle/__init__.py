@@ -236,3 +236,24 @@ def path_indices(tree_parent, tree_size, D_max: int) -> dict:
     flags = fn(C.c_int(B), C.c_int(T), C.c_int(D_max), _p(tp, _i32p, np.int32), _p(ts, _i32p, np.int32),
                _p(out, _i32p, np.int32), _p(n, _i32p, np.int32))
     return dict(path_index=out, n_paths=n, flags=int(flags))
+
+
+def accept_stochastic(logits_bits, temperature: float, tree_token, tree_parent, tree_size, u_accept, u_bonus) -> dict:
+    """logits_bits: uint16 (bf16 bit patterns) [B*T_max, V]; u_accept float32 [B, T_max], u_bonus float32 [B].
+    Returns n_acc, path, best_node, bonus, margin (float64 [B]) and the flag word."""
+    lg = np.ascontiguousarray(logits_bits, np.uint16)
+    tt, tp, ts = _arr(tree_token, np.int32), _arr(tree_parent, np.int32), _arr(tree_size, np.int32)
+    ua, ub = _arr(u_accept, np.float32), _arr(u_bonus, np.float32)
+    B, T = tt.shape
+    V = lg.shape[1]
+    assert lg.shape[0] == B * T and ua.shape == (B, T) and ub.shape == (B,)
+    out = dict(n_acc=np.empty(B, np.int32), best_node=np.empty(B, np.int32), bonus=np.empty(B, np.int32),
+               path=np.empty((B, T), np.int32), margin=np.empty(B, np.float64))
+    fn = lib().orc_accept_stochastic
+    fn.restype = C.c_uint
+    flags = fn(C.c_int(B), C.c_int(T), C.c_int(V), _p(lg, _u16p, np.uint16), C.c_double(temperature),
+               _p(tt, _i32p, np.int32), _p(tp, _i32p, np.int32), _p(ts, _i32p, np.int32), _p(ua, _f32p, np.float32),
+               _p(ub, _f32p, np.float32), _p(out["n_acc"], _i32p, np.int32), _p(out["path"], _i32p, np.int32),
+               _p(out["best_node"], _i32p, np.int32), _p(out["bonus"], _i32p, np.int32), _p(out["margin"], _f64p, np.float64))
+    out["flags"] = int(flags)
+    return out

@@ -18,7 +18,10 @@
  * the retrieval envelope against the lookup equation folded along explicit rank paths, a shift matrix
  * with a closed form, the tree assembly's own lookups and the printed shape of the full template
  * (80 nodes, 8+16+14+11+8+7+6+5+5 over depths 1..9); the candidate-path table against a top-down
- * enumeration, chain and star trees, and acceptance written over paths.
+ * enumeration, chain and star trees, and acceptance written over paths; stochastic acceptance against
+ * a hand-worked three-token example, the empirical distribution of the first emitted token and of the
+ * second given the first over 200000 draws (lossless equivalence), and greedy acceptance in the
+ * low-temperature limit.
  * Parity unpinned: nothing beyond the printed per-depth counts fixes the retrieval
  * templates' exact rank paths; they are inputs here, not computed.
  */
@@ -528,5 +531,89 @@ unsigned orc_path_indices(int B, int T_max, int D_max, const int32_t *tree_paren
         n_paths[b] = n;
     }
     free(up);
+    return flags;
+}
+
+/* ------------------------------------------------------------------------------------------------
+ * Stochastic acceptance (temperature sampling discussion and the lossless-equivalence proposition:
+ * the hybrid tree is verified "with the standard speculative sampling rule", "a rejected position is
+ * resampled from the target correction distribution").  The tree's candidates are fixed tokens (kept
+ * draft nodes and retrieved nodes alike), i.e. point-mass proposals, so the rule at a node u with
+ * target distribution p = softmax(logits[u] / temperature) is the sequential one over u's children in
+ * node order: child c with token x is accepted with probability p(x) / rem, where rem is the mass p
+ * still holds; on rejection p(x) is set to zero and rem shrinks by it (the correction distribution
+ * max(0, p - proposal) renormalised, for a point-mass proposal).  An accepted child becomes the new
+ * u.  When no child is accepted (or u is a leaf) the step ends and the bonus token is drawn from what
+ * is left of p by inverse CDF over increasing ids.  Every emitted token is then distributed as under
+ * plain sampling from the target.
+ *   Random numbers are inputs: u_accept[b, c] in [0, 1) decides child c (accept iff u * rem < p(x)),
+ * u_bonus[b] draws the bonus (smallest id whose running sum of remaining mass exceeds u * rem).
+ * Children with token -1, or with a token a rejected sibling already carried, have probability zero.
+ * margin[b] (optional) is the smallest distance, relative to rem, between a decision's random number
+ * and its boundary: a float32 implementation agrees with this one whenever the margin is well above
+ * float32 rounding of the sums involved.
+ * ------------------------------------------------------------------------------------------------ */
+unsigned orc_accept_stochastic(int B, int T_max, int V, const uint16_t *logits /* bf16 bits [B*T_max, V] */, double temperature,
+                               const int32_t *tree_token, const int32_t *tree_parent, const int32_t *tree_size,
+                               const float *u_accept /* [B, T_max] */, const float *u_bonus /* [B] */,
+                               int32_t *n_acc, int32_t *path /* [B, T_max] */, int32_t *best_node, int32_t *bonus,
+                               double *margin /* [B] or NULL */) {
+    unsigned flags = 0;
+    double *p = (double *)malloc((size_t)V * sizeof(double));
+    for (int b = 0; b < B; ++b) {
+        const int32_t *tok = tree_token + (size_t)b * T_max;
+        const int32_t *par = tree_parent + (size_t)b * T_max;
+        int32_t *pth = path + (size_t)b * T_max;
+        for (int j = 0; j < T_max; ++j) pth[j] = -1;
+        const int T = tree_size[b];
+        if (margin) margin[b] = 1.0;
+        if (T < 1 || T > T_max) { n_acc[b] = 0; best_node[b] = -1; bonus[b] = -1; if (T != 0) flags |= ORC_FLAG_BAD_SIZE; continue; }
+        int u = 0, n = 0;
+        double rem = 1.0;
+        for (;;) {
+            pth[n++] = u;
+            /* p = softmax(logits[u] / temperature) */
+            const uint16_t *row = logits + ((size_t)b * T_max + u) * V;
+            double zmax = -INFINITY, sum = 0.0;
+            for (int v = 0; v < V; ++v) { double z = bf16_to_double(row[v]) / temperature; if (z > zmax) zmax = z; }
+            for (int v = 0; v < V; ++v) { p[v] = exp(bf16_to_double(row[v]) / temperature - zmax); sum += p[v]; }
+            for (int v = 0; v < V; ++v) p[v] /= sum;
+            rem = 1.0;
+            int next = -1;
+            for (int c = u + 1; c < T && next < 0; ++c) {
+                if (par[c] != u) continue;
+                const int x = tok[c];
+                const double px = (x >= 0 && x < V) ? p[x] : 0.0;
+                const double r = (double)u_accept[(size_t)b * T_max + c] * rem;
+                if (margin && px > 0.0) { double m = fabs(r - px) / rem; if (m < margin[b]) margin[b] = m; }
+                if (r < px) { next = c; break; }
+                if (x >= 0 && x < V) { rem -= px; p[x] = 0.0; }
+            }
+            if (next < 0) break;
+            u = next;
+        }
+        /* bonus from what is left of p at u */
+        const double target = (double)u_bonus[b] * rem;
+        double run = 0.0;
+        int pick = -1, last = -1;
+        for (int v = 0; v < V; ++v) {
+            if (p[v] <= 0.0) continue;
+            last = v;
+            const double before = run;
+            run += p[v];
+            if (pick < 0 && run > target) {
+                pick = v;
+                if (margin) {
+                    double m = fmin(target - before, run - target) / rem;
+                    if (m < margin[b]) margin[b] = m;
+                }
+            }
+        }
+        if (pick < 0) pick = last;             /* rounding left the running sum just below the target */
+        n_acc[b] = n;
+        best_node[b] = u;
+        bonus[b] = pick;
+    }
+    free(p);
     return flags;
 }
