@@ -14,7 +14,8 @@
  *     graft_tree_verify_attn  Sec. 3.3: tree attention of the T tree tokens over cache + ancestors
  *     [caller: lm_head gives the target logits of the tree nodes]
  *     graft_update_adjacency  retrieval section / appendix: M[x_i] <- argtopk(p_{i+1}); also target_next
- *     graft_accept            Algorithm 1 "select the accepted path" (greedy, lossless)
+ *     graft_accept            Algorithm 1 "select the accepted path" (greedy, lossless); under temperature
+ *                             sampling graft_accept_stochastic takes its place
  *     graft_compact_kv        Algorithm 1 "append accepted tokens and update target KV cache"
  *
  * Conventions
@@ -312,6 +313,43 @@ typedef struct {
 } graft_accept_params;
 
 int graft_accept(graft_ctx* ctx, const graft_accept_params* p, void* stream);
+
+/* ---- graft_accept_stochastic ------------------------------------------------------------------ */
+/*
+ * Acceptance under temperature sampling (temperature-sampling discussion; lossless-equivalence
+ * proposition: the tree is verified "with the standard speculative sampling rule", a rejected position is
+ * "resampled from the target correction distribution").  The tree's candidates are fixed tokens, so at a
+ * node u with p = softmax(logits[u] / temperature) the children of u are tried in node order: child c with
+ * token x is accepted iff u_accept[b, c] * rem < p(x), where rem (1 at first) is the mass p still holds; a
+ * rejected child's token loses its mass (rem -= p(x), p(x) = 0: the correction distribution for a point-mass
+ * proposal).  An accepted child becomes u.  When no child is accepted, or u is a leaf, the bonus token is
+ * the smallest id whose running sum of the remaining mass (ids in increasing order) exceeds
+ * u_bonus[b] * rem.  Children with token -1 or with a token that a rejected sibling carried are never
+ * accepted.  Outputs as graft_accept: path (root first, -1 padded), n_acc = nodes on it, best_node = its
+ * last node, bonus.  Random numbers are inputs in [0, 1).
+ * Arithmetic is fp32 (row maxima and exponential sums over V entries, running sums of the bonus draw), so
+ * an outcome is only defined up to that rounding when a random number falls within ~1e-5 (relative to
+ * rem) of a decision boundary.
+ * row_stats: caller-provided scratch of 2 floats per row (max of logits / temperature, sum of exponentials).
+ * logits: 16-byte aligned base, row stride a multiple of 8 elements; temperature > 0; T_max <= 64.
+ */
+typedef struct {
+    int B, T_max, V;
+    float temperature;
+    const void* logits; int64_t logits_stride_row;   /* bf16 [B * T_max, V] */
+    const int32_t* tree_token;   /* [B, T_max] */
+    const int32_t* tree_parent;  /* [B, T_max] */
+    const int32_t* tree_size;    /* [B] */
+    const float* u_accept;       /* [B, T_max] */
+    const float* u_bonus;        /* [B] */
+    float* row_stats;            /* scratch [B * T_max, 2] */
+    int32_t* n_acc;              /* out [B] */
+    int32_t* path;               /* out [B, T_max] */
+    int32_t* best_node;          /* out [B] */
+    int32_t* bonus;              /* out [B] */
+} graft_accept_stochastic_params;
+
+int graft_accept_stochastic(graft_ctx* ctx, const graft_accept_stochastic_params* p, void* stream);
 
 /* ---- graft_compact_kv ------------------------------------------------------------------------ */
 /*

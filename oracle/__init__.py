@@ -240,7 +240,7 @@ def path_indices(tree_parent, tree_size, D_max: int) -> dict:
 
 def accept_stochastic(logits_bits, temperature: float, tree_token, tree_parent, tree_size, u_accept, u_bonus) -> dict:
     """logits_bits: uint16 (bf16 bit patterns) [B*T_max, V]; u_accept float32 [B, T_max], u_bonus float32 [B].
-    Returns n_acc, path, best_node, bonus, margin (float64 [B]) and the flag word."""
+    Returns n_acc, path, best_node, bonus, margin (float64 [B, 2]: accept decisions, bonus draw) and the flag word."""
     lg = np.ascontiguousarray(logits_bits, np.uint16)
     tt, tp, ts = _arr(tree_token, np.int32), _arr(tree_parent, np.int32), _arr(tree_size, np.int32)
     ua, ub = _arr(u_accept, np.float32), _arr(u_bonus, np.float32)
@@ -248,7 +248,7 @@ def accept_stochastic(logits_bits, temperature: float, tree_token, tree_parent, 
     V = lg.shape[1]
     assert lg.shape[0] == B * T and ua.shape == (B, T) and ub.shape == (B,)
     out = dict(n_acc=np.empty(B, np.int32), best_node=np.empty(B, np.int32), bonus=np.empty(B, np.int32),
-               path=np.empty((B, T), np.int32), margin=np.empty(B, np.float64))
+               path=np.empty((B, T), np.int32), margin=np.empty((B, 2), np.float64))
     fn = lib().orc_accept_stochastic
     fn.restype = C.c_uint
     flags = fn(C.c_int(B), C.c_int(T), C.c_int(V), _p(lg, _u16p, np.uint16), C.c_double(temperature),

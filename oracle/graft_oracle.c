@@ -549,15 +549,16 @@ unsigned orc_path_indices(int B, int T_max, int D_max, const int32_t *tree_paren
  *   Random numbers are inputs: u_accept[b, c] in [0, 1) decides child c (accept iff u * rem < p(x)),
  * u_bonus[b] draws the bonus (smallest id whose running sum of remaining mass exceeds u * rem).
  * Children with token -1, or with a token a rejected sibling already carried, have probability zero.
- * margin[b] (optional) is the smallest distance, relative to rem, between a decision's random number
- * and its boundary: a float32 implementation agrees with this one whenever the margin is well above
- * float32 rounding of the sums involved.
+ * margin[2b] (optional) is the smallest distance, relative to rem, between an accept decision's random
+ * number and its boundary, margin[2b + 1] that of the bonus draw from the ends of the picked id's interval:
+ * a float32 implementation agrees with this one whenever the margins are well above float32 rounding of
+ * the sums involved.
  * ------------------------------------------------------------------------------------------------ */
 unsigned orc_accept_stochastic(int B, int T_max, int V, const uint16_t *logits /* bf16 bits [B*T_max, V] */, double temperature,
                                const int32_t *tree_token, const int32_t *tree_parent, const int32_t *tree_size,
                                const float *u_accept /* [B, T_max] */, const float *u_bonus /* [B] */,
                                int32_t *n_acc, int32_t *path /* [B, T_max] */, int32_t *best_node, int32_t *bonus,
-                               double *margin /* [B] or NULL */) {
+                               double *margin /* [B, 2] or NULL */) {
     unsigned flags = 0;
     double *p = (double *)malloc((size_t)V * sizeof(double));
     for (int b = 0; b < B; ++b) {
@@ -566,7 +567,7 @@ unsigned orc_accept_stochastic(int B, int T_max, int V, const uint16_t *logits /
         int32_t *pth = path + (size_t)b * T_max;
         for (int j = 0; j < T_max; ++j) pth[j] = -1;
         const int T = tree_size[b];
-        if (margin) margin[b] = 1.0;
+        if (margin) { margin[2 * b] = 1.0; margin[2 * b + 1] = 1.0; }
         if (T < 1 || T > T_max) { n_acc[b] = 0; best_node[b] = -1; bonus[b] = -1; if (T != 0) flags |= ORC_FLAG_BAD_SIZE; continue; }
         int u = 0, n = 0;
         double rem = 1.0;
@@ -585,7 +586,7 @@ unsigned orc_accept_stochastic(int B, int T_max, int V, const uint16_t *logits /
                 const int x = tok[c];
                 const double px = (x >= 0 && x < V) ? p[x] : 0.0;
                 const double r = (double)u_accept[(size_t)b * T_max + c] * rem;
-                if (margin && px > 0.0) { double m = fabs(r - px) / rem; if (m < margin[b]) margin[b] = m; }
+                if (margin && px > 0.0) { double m = fabs(r - px) / rem; if (m < margin[2 * b]) margin[2 * b] = m; }
                 if (r < px) { next = c; break; }
                 if (x >= 0 && x < V) { rem -= px; p[x] = 0.0; }
             }
@@ -604,8 +605,7 @@ unsigned orc_accept_stochastic(int B, int T_max, int V, const uint16_t *logits /
             if (pick < 0 && run > target) {
                 pick = v;
                 if (margin) {
-                    double m = fmin(target - before, run - target) / rem;
-                    if (m < margin[b]) margin[b] = m;
+                    margin[2 * b + 1] = fmin(target - before, run - target) / rem;
                 }
             }
         }

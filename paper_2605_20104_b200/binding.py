@@ -30,7 +30,7 @@ ATTN_AUTO, ATTN_MMA_SYNC, ATTN_TCGEN05, ATTN_TCGEN05_1SM, ATTN_TCGEN05_2SM, ATTN
 EXPORTS = ("graft_workspace_bytes", "graft_create", "graft_destroy", "graft_status_string", "graft_device_status",
            "graft_build_tree", "graft_tree_verify_attn", "graft_accept", "graft_compact_kv",
            "graft_noalloc_scratch_bytes", "graft_tree_verify_attn_noalloc", "graft_update_adjacency",
-           "graft_retrieve_envelope", "graft_path_indices")
+           "graft_retrieve_envelope", "graft_path_indices", "graft_accept_stochastic")
 
 _vp = C.c_void_p
 
@@ -48,6 +48,13 @@ class BuildParams(C.Structure):
 class EnvelopeParams(C.Structure):
     _fields_ = ([(n, C.c_int) for n in ("B", "V", "k", "N_env")] + [("root_token", _vp), ("root_stride", C.c_int64)] +
                 [(n, _vp) for n in ("M", "env_parent", "env_rank", "env_token")])
+
+
+class AcceptStochasticParams(C.Structure):
+    _fields_ = ([(n, C.c_int) for n in ("B", "T_max", "V")] + [("temperature", C.c_float), ("logits", _vp),
+                 ("logits_stride_row", C.c_int64)] +
+                [(n, _vp) for n in ("tree_token", "tree_parent", "tree_size", "u_accept", "u_bonus", "row_stats", "n_acc", "path",
+                                    "best_node", "bonus")])
 
 
 class PathsParams(C.Structure):
@@ -95,7 +102,7 @@ _lib.graft_device_status.argtypes = [_vp, _vp, C.POINTER(C.c_uint), C.c_int]
 for _name, _typ in (("graft_build_tree", BuildParams), ("graft_tree_verify_attn", AttnParams),
                     ("graft_accept", AcceptParams), ("graft_compact_kv", CompactParams),
                     ("graft_update_adjacency", UpdateParams), ("graft_retrieve_envelope", EnvelopeParams),
-                    ("graft_path_indices", PathsParams)):
+                    ("graft_path_indices", PathsParams), ("graft_accept_stochastic", AcceptStochasticParams)):
     getattr(_lib, _name).restype = C.c_int
     getattr(_lib, _name).argtypes = [_vp, C.POINTER(_typ), _vp]
 
@@ -295,6 +302,26 @@ def path_indices_params(*, tree_parent, tree_size, path_index, n_paths) -> Paths
 
 def graft_path_indices(ctx: Context, **kw) -> None:
     launch("graft_path_indices", ctx, path_indices_params(**kw))
+
+
+def accept_stochastic_params(*, logits, temperature: float, tree_token, tree_parent, tree_size, u_accept, u_bonus, row_stats,
+                             n_acc, path, best_node, bonus) -> AcceptStochasticParams:
+    """logits: bf16 [B*T_max, V] (rows may be strided); u_accept float32 [B, T_max], u_bonus float32 [B] in [0, 1);
+    row_stats: float32 scratch [B*T_max, 2]."""
+    i32, f32 = torch.int32, torch.float32
+    B, T_max = tree_token.shape
+    assert logits.dim() == 2 and logits.shape[0] == B * T_max and logits.stride(1) == 1
+    assert u_accept.shape == (B, T_max) and u_bonus.shape == (B,) and row_stats.numel() >= 2 * B * T_max
+    return AcceptStochasticParams(B=B, T_max=T_max, V=logits.shape[1], temperature=temperature, logits=_ptr(logits, torch.bfloat16),
+                                  logits_stride_row=logits.stride(0), tree_token=_ptr(tree_token, i32),
+                                  tree_parent=_ptr(tree_parent, i32), tree_size=_ptr(tree_size, i32),
+                                  u_accept=_ptr(u_accept, f32), u_bonus=_ptr(u_bonus, f32), row_stats=_ptr(row_stats, f32),
+                                  n_acc=_ptr(n_acc, i32), path=_ptr(path, i32), best_node=_ptr(best_node, i32),
+                                  bonus=_ptr(bonus, i32))
+
+
+def graft_accept_stochastic(ctx: Context, **kw) -> None:
+    launch("graft_accept_stochastic", ctx, accept_stochastic_params(**kw))
 
 
 def graft_accept(ctx: Context, **kw) -> None:

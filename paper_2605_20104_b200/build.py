@@ -12,7 +12,7 @@ HERE = os.path.dirname(os.path.abspath(__file__))
 ROOT = os.path.dirname(HERE)
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libgraft.so")
-SOURCES = ["api.cu", "build_tree.cu", "accept.cu", "compact_kv.cu", "attn_mma.cu", "attn_tc.cu", "attn_noalloc.cu", "update_adjacency.cu", "envelope_paths.cu"]
+SOURCES = ["api.cu", "build_tree.cu", "accept.cu", "compact_kv.cu", "attn_mma.cu", "attn_tc.cu", "attn_noalloc.cu", "update_adjacency.cu", "envelope_paths.cu", "accept_stochastic.cu"]
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-O3", "-std=c++17", "-lineinfo", "--use_fast_math",
               "-Xcompiler", "-fPIC", "-I", os.path.join(ROOT, "include"), "-I", CSRC]
 

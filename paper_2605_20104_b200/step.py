@@ -160,6 +160,16 @@ class VerifyStep:
             tree_token=self.tree_token, tree_parent=self.tree_parent, tree_anc=self.tree_anc, tree_size=self.tree_size,
             target_next=self.target_next, n_acc=self.n_acc, path=self.path, best_node=self.best_node, bonus=self.bonus)))
 
+    def accept_stochastic(self, logits: torch.Tensor, temperature: float, u_accept: torch.Tensor, u_bonus: torch.Tensor) -> None:
+        """Acceptance under temperature sampling: logits bf16 [B*T_max, V], random numbers float32 [B, T_max] and [B]."""
+        if getattr(self, "row_stats", None) is None:
+            self.row_stats = torch.empty(self.w.B * self.w.T_max, 2, dtype=torch.float32, device=self.dev)
+        key = ("accept_s", logits.data_ptr(), u_accept.data_ptr(), u_bonus.data_ptr(), temperature)
+        G.launch("graft_accept_stochastic", self.ctx, self._cached(key, lambda: G.accept_stochastic_params(
+            logits=logits, temperature=temperature, tree_token=self.tree_token, tree_parent=self.tree_parent,
+            tree_size=self.tree_size, u_accept=u_accept, u_bonus=u_bonus, row_stats=self.row_stats, n_acc=self.n_acc,
+            path=self.path, best_node=self.best_node, bonus=self.bonus)))
+
     def compact(self) -> None:
         key = ("compact", self.Kc.data_ptr(), self.Vc.data_ptr())
         G.launch("graft_compact_kv", self.ctx, self._cached(key, lambda: G.compact_kv_params(

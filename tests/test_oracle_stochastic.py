@@ -40,7 +40,8 @@ def test_hand_worked_example():
     assert r["path"][0].tolist() == [0, 2, -1] and r["best_node"][0] == 2
     r = go(0.6, 0.6, 0.3)                 # both rejected (0.6 * 0.5 >= 0.25): bonus from {2: 0.25}
     assert r["n_acc"][0] == 1 and r["best_node"][0] == 0 and r["bonus"][0] == 2
-    assert abs(r["margin"][0] - 0.1) < 1e-6      # |0.6 - 0.5| / 1 is the closest call
+    assert abs(r["margin"][0, 0] - 0.1) < 1e-6   # |0.6 - 0.5| / 1 is the closest accept decision
+    assert abs(r["margin"][0, 1] - 0.3) < 1e-6   # the bonus draw: 0.3 * 0.25 sits 0.3 (of rem) inside token 2's interval
 
 
 def test_duplicate_sibling_and_empty_token():
