@@ -197,6 +197,37 @@ def time_update(st, steps, warmup):
             "GBps": byts / (us * 1e-6) / 1e9, "l2": "rotating %d logits buffers" % n_rot}
 
 
+def time_accept_stochastic(st, steps, warmup):
+    """graft_accept_stochastic alone (row statistics of every valid node's logits + walk + bonus draw) on the
+    workload's trees, generator-shaped logits in rotation (> L2 together), fresh uniform numbers."""
+    from paper_2605_20104_b200 import binding as G
+    w, vs = st["w"], st["vs"]
+    lg = torch.from_numpy(W.make_logits(w.B, w.T_max, w.V, seed=w.seed + 23).view(np.int16)).view(torch.bfloat16)
+    n_rot = max(2, int(np.ceil(3 * L2_BYTES / (lg.numel() * 2))))
+    bufs = [lg.to(vs.dev).clone() for _ in range(n_rot)]
+    g = torch.Generator(device=vs.dev)
+    g.manual_seed(5)
+    ua = torch.rand(w.B, w.T_max, device=vs.dev, generator=g)
+    ub = torch.rand(w.B, device=vs.dev, generator=g)
+    ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(steps)]
+    for i in range(warmup):
+        vs.accept_stochastic(bufs[i % n_rot], 1.0, ua, ub)
+    torch.cuda.synchronize()
+    torch.cuda._sleep(int(3e6))
+    for i in range(steps):
+        ev[i][0].record()
+        vs.accept_stochastic(bufs[i % n_rot], 1.0, ua, ub)
+        ev[i][1].record()
+    torch.cuda.synchronize()
+    us = float(np.mean([a.elapsed_time(b) for a, b in ev])) * 1e3
+    rows = int(st["tree"]["tree_size"].sum())
+    byts = rows * w.V * 2
+    vs.accept()                      # leave the greedy result the step produced
+    torch.cuda.synchronize()
+    return {"us_per_call": us, "rows": rows, "V": int(w.V), "algorithmic_bytes": byts, "GBps": byts / (us * 1e-6) / 1e9,
+            "l2": "rotating %d logits buffers" % n_rot}
+
+
 def time_index_kernels(st, steps, warmup):
     """The small index kernels around tree assembly, each alone: the retrieval envelope, assembly with its own
     lookups and from the envelope, and the candidate-path table (latency-bound launches of B CTAs)."""
@@ -455,6 +486,9 @@ def main():
         upd["frac_of_measured"] = upd["GBps"] / peak
         line["update_adjacency"] = upd
         line["index_kernels"] = time_index_kernels(st, min(args.steps, 50), 5)
+        acs = time_accept_stochastic(st, min(args.steps, 50), 5)
+        acs["frac_of_measured"] = acs["GBps"] / peak
+        line["accept_stochastic"] = acs
         extra = []
         del st
         torch.cuda.empty_cache()

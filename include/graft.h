@@ -330,8 +330,9 @@ int graft_accept(graft_ctx* ctx, const graft_accept_params* p, void* stream);
  * Arithmetic is fp32 (row maxima and exponential sums over V entries, running sums of the bonus draw), so
  * an outcome is only defined up to that rounding when a random number falls within ~1e-5 (relative to
  * rem) of a decision boundary.
- * row_stats: caller-provided scratch of 2 floats per row (max of logits / temperature, sum of exponentials).
- * logits: 16-byte aligned base, row stride a multiple of 8 elements; temperature > 0; T_max <= 64.
+ * row_stats: caller-provided scratch of graft_accept_stochastic_scratch_floats(B, T_max, V) floats (per row the
+ * max of logits / temperature and the sum of exponentials, of the whole row and of every 256 ids).
+ * logits: 16-byte aligned base, row stride a multiple of 8 elements; temperature > 0; T_max <= 64; V <= 524288.
  */
 typedef struct {
     int B, T_max, V;
@@ -342,13 +343,14 @@ typedef struct {
     const int32_t* tree_size;    /* [B] */
     const float* u_accept;       /* [B, T_max] */
     const float* u_bonus;        /* [B] */
-    float* row_stats;            /* scratch [B * T_max, 2] */
+    float* row_stats;            /* scratch, see above */
     int32_t* n_acc;              /* out [B] */
     int32_t* path;               /* out [B, T_max] */
     int32_t* best_node;          /* out [B] */
     int32_t* bonus;              /* out [B] */
 } graft_accept_stochastic_params;
 
+size_t graft_accept_stochastic_scratch_floats(int B, int T_max, int V);     /* host only; 0 for invalid sizes */
 int graft_accept_stochastic(graft_ctx* ctx, const graft_accept_stochastic_params* p, void* stream);
 
 /* ---- graft_compact_kv ------------------------------------------------------------------------ */

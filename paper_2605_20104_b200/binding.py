@@ -30,7 +30,8 @@ ATTN_AUTO, ATTN_MMA_SYNC, ATTN_TCGEN05, ATTN_TCGEN05_1SM, ATTN_TCGEN05_2SM, ATTN
 EXPORTS = ("graft_workspace_bytes", "graft_create", "graft_destroy", "graft_status_string", "graft_device_status",
            "graft_build_tree", "graft_tree_verify_attn", "graft_accept", "graft_compact_kv",
            "graft_noalloc_scratch_bytes", "graft_tree_verify_attn_noalloc", "graft_update_adjacency",
-           "graft_retrieve_envelope", "graft_path_indices", "graft_accept_stochastic")
+           "graft_retrieve_envelope", "graft_path_indices", "graft_accept_stochastic",
+           "graft_accept_stochastic_scratch_floats")
 
 _vp = C.c_void_p
 
@@ -109,6 +110,8 @@ for _name, _typ in (("graft_build_tree", BuildParams), ("graft_tree_verify_attn"
 
 _lib.graft_noalloc_scratch_bytes.restype = C.c_size_t
 _lib.graft_noalloc_scratch_bytes.argtypes = []
+_lib.graft_accept_stochastic_scratch_floats.restype = C.c_size_t
+_lib.graft_accept_stochastic_scratch_floats.argtypes = [C.c_int] * 3
 _lib.graft_tree_verify_attn_noalloc.restype = C.c_int
 _lib.graft_tree_verify_attn_noalloc.argtypes = [C.POINTER(AttnParams), _vp, _vp]
 
@@ -307,17 +310,22 @@ def graft_path_indices(ctx: Context, **kw) -> None:
 def accept_stochastic_params(*, logits, temperature: float, tree_token, tree_parent, tree_size, u_accept, u_bonus, row_stats,
                              n_acc, path, best_node, bonus) -> AcceptStochasticParams:
     """logits: bf16 [B*T_max, V] (rows may be strided); u_accept float32 [B, T_max], u_bonus float32 [B] in [0, 1);
-    row_stats: float32 scratch [B*T_max, 2]."""
+    row_stats: float32 scratch of graft_accept_stochastic_scratch_floats(B, T_max, V) elements."""
     i32, f32 = torch.int32, torch.float32
     B, T_max = tree_token.shape
     assert logits.dim() == 2 and logits.shape[0] == B * T_max and logits.stride(1) == 1
-    assert u_accept.shape == (B, T_max) and u_bonus.shape == (B,) and row_stats.numel() >= 2 * B * T_max
+    assert u_accept.shape == (B, T_max) and u_bonus.shape == (B,)
+    assert row_stats.numel() >= graft_accept_stochastic_scratch_floats(B, T_max, logits.shape[1])
     return AcceptStochasticParams(B=B, T_max=T_max, V=logits.shape[1], temperature=temperature, logits=_ptr(logits, torch.bfloat16),
                                   logits_stride_row=logits.stride(0), tree_token=_ptr(tree_token, i32),
                                   tree_parent=_ptr(tree_parent, i32), tree_size=_ptr(tree_size, i32),
                                   u_accept=_ptr(u_accept, f32), u_bonus=_ptr(u_bonus, f32), row_stats=_ptr(row_stats, f32),
                                   n_acc=_ptr(n_acc, i32), path=_ptr(path, i32), best_node=_ptr(best_node, i32),
                                   bonus=_ptr(bonus, i32))
+
+
+def graft_accept_stochastic_scratch_floats(B: int, T_max: int, V: int) -> int:
+    return int(_lib.graft_accept_stochastic_scratch_floats(B, T_max, V))
 
 
 def graft_accept_stochastic(ctx: Context, **kw) -> None:

@@ -1,15 +1,16 @@
 // graft_accept_stochastic: acceptance under temperature sampling, two kernels.
 //
 //   softmax_stats_kernel   one CTA per tree node streams that node's V logits once and leaves the row's
-//                          (max of logit / temperature, sum of exponentials) pair: which rows the walk
-//                          will need is only known while walking, so all valid rows are done at once, in
-//                          parallel (HBM-bound: V * 2 bytes per valid node, as the adjacency refresh);
+//                          (max of logit / temperature, sum of exponentials) pair and the same pair for
+//                          every step of 256 ids: which rows the walk will need is only known while
+//                          walking, so all valid rows are done at once, in parallel (HBM-bound: V * 2 bytes
+//                          per valid node, as the adjacency refresh);
 //   accept_walk_kernel     one CTA per request: every thread of the first T computes the probability of
 //                          its node's token under the parent's distribution (one gather each), one thread
 //                          walks the tree with those (sequential rejection over a node's children), then
-//                          the whole CTA draws the bonus token from the last node's remaining distribution:
-//                          contiguous chunks per thread, block scan of the chunk sums, and the warp of the
-//                          chunk that holds the target splits it once more.
+//                          the CTA draws the bonus token from the last node's remaining distribution: a scan
+//                          over that row's step sums (rejected tokens taken out) finds the step that crosses
+//                          the target, one warp loads its 256 ids and finds the lane and the id.
 #include <cuda_bf16.h>
 #include <math_constants.h>
 #include "graft_internal.cuh"
@@ -17,10 +18,15 @@
 namespace {
 
 constexpr int ST = 512;        // threads of the statistics kernel
-constexpr int WT = 256;        // threads of the walk kernel
+constexpr int WT = 1024;       // threads of the walk kernel
+constexpr int kStep = 256;     // ids per step: eight per lane of a warp
+constexpr int kMaxSteps = 2 * WT;   // steps of a row the walk kernel can scan: V <= 524288
 
 __device__ __forceinline__ float lo_f(uint32_t w) { return __uint_as_float(w << 16); }
 __device__ __forceinline__ float hi_f(uint32_t w) { return __uint_as_float(w & 0xffff0000u); }
+__host__ __device__ __forceinline__ int steps_of(int V) { return (V + kStep - 1) / kStep; }
+// scratch of a row: (m, s) of the row, then (m, s) of every step
+__host__ __device__ __forceinline__ size_t row_floats(int V) { return 2 + 2 * (size_t)steps_of(V); }
 
 // (m, s) <- (m, s) (+) (m2, s2): s counts exponentials relative to m
 __device__ __forceinline__ void combine(float& m, float& s, float m2, float s2) {
@@ -30,7 +36,21 @@ __device__ __forceinline__ void combine(float& m, float& s, float m2, float s2) 
     m = mn;
 }
 
-__global__ void __launch_bounds__(ST, 2) softmax_stats_kernel(graft_accept_stochastic_params p, unsigned* status) {
+// eight scaled logits of a lane: ids v0 .. v0 + 7 of the row, -inf past its end
+__device__ __forceinline__ void scaled8(const __nv_bfloat16* row, int v0, int V, float inv_t, float (&z)[8]) {
+    if (v0 + 8 <= V) {
+        const uint4 q = __ldcs(reinterpret_cast<const uint4*>(row + v0));
+        z[0] = lo_f(q.x) * inv_t; z[1] = hi_f(q.x) * inv_t; z[2] = lo_f(q.y) * inv_t; z[3] = hi_f(q.y) * inv_t;
+        z[4] = lo_f(q.z) * inv_t; z[5] = hi_f(q.z) * inv_t; z[6] = lo_f(q.w) * inv_t; z[7] = hi_f(q.w) * inv_t;
+    } else {
+#pragma unroll
+        for (int e = 0; e < 8; ++e) z[e] = v0 + e < V ? __bfloat162float(row[v0 + e]) * inv_t : -CUDART_INF_F;
+    }
+}
+
+// One CTA per tree node; a warp takes a step of 256 ids at a time (four in flight), leaves the step's
+// (max, sum of exponentials relative to it) and folds it into its running pair.
+__global__ void __launch_bounds__(ST, 2) softmax_stats_kernel(graft_accept_stochastic_params p) {
     __shared__ float s_m[ST / 32], s_s[ST / 32];
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int r = blockIdx.x, b = r / p.T_max, i = r % p.T_max;
@@ -39,29 +59,38 @@ __global__ void __launch_bounds__(ST, 2) softmax_stats_kernel(graft_accept_stoch
     if (i >= T) return;
     const float inv_t = 1.f / p.temperature;
     const __nv_bfloat16* row = reinterpret_cast<const __nv_bfloat16*>(p.logits) + (size_t)r * p.logits_stride_row;
-    const int nvec = p.V >> 3;
+    float* out = p.row_stats + (size_t)r * row_floats(p.V);
+    const int nsteps = steps_of(p.V);
     float m = -CUDART_INF_F, s = 0.f;
-    for (int j = tid; j < nvec; j += ST) {
-        const uint4 q = __ldcs(reinterpret_cast<const uint4*>(row) + j);
-        float z[8] = {lo_f(q.x) * inv_t, hi_f(q.x) * inv_t, lo_f(q.y) * inv_t, hi_f(q.y) * inv_t,
-                      lo_f(q.z) * inv_t, hi_f(q.z) * inv_t, lo_f(q.w) * inv_t, hi_f(q.w) * inv_t};
-        float vm = z[0];
+    constexpr int NWS = ST / 32, kFlight = 4;          // steps a warp has in flight
+    for (int st = warp; st < nsteps; st += kFlight * NWS) {
+        float z[kFlight][8];
 #pragma unroll
-        for (int e = 1; e < 8; ++e) vm = fmaxf(vm, z[e]);
-        const float mn = fmaxf(m, vm);
-        if (mn > -CUDART_INF_F) {
-            float add = 0.f;
+        for (int h = 0; h < kFlight; ++h)
+            if (st + h * NWS < nsteps) scaled8(row, (st + h * NWS) * kStep + lane * 8, p.V, inv_t, z[h]);
 #pragma unroll
-            for (int e = 0; e < 8; ++e) add += __expf(z[e] - mn);
-            s = s * __expf(m - mn) + add;
-            m = mn;
+        for (int h = 0; h < kFlight; ++h) {
+            const int sx = st + h * NWS;
+            if (sx < nsteps) {
+                float vm = z[h][0];
+#pragma unroll
+                for (int e = 1; e < 8; ++e) vm = fmaxf(vm, z[h][e]);
+#pragma unroll
+                for (int o = 16; o; o >>= 1) vm = fmaxf(vm, __shfl_xor_sync(0xffffffffu, vm, o));
+                float add = 0.f;
+                if (vm > -CUDART_INF_F) {
+#pragma unroll
+                    for (int e = 0; e < 8; ++e) add += __expf(z[h][e] - vm);
+                }
+#pragma unroll
+                for (int o = 16; o; o >>= 1) add += __shfl_xor_sync(0xffffffffu, add, o);
+                if (lane == 0) {
+                    out[2 + 2 * sx] = vm;
+                    out[2 + 2 * sx + 1] = add;
+                }
+                combine(m, s, vm, add);
+            }
         }
-    }
-    for (int v = (nvec << 3) + tid; v < p.V; v += ST) combine(m, s, __bfloat162float(row[v]) * inv_t, 1.f);
-#pragma unroll
-    for (int o = 16; o; o >>= 1) {
-        const float m2 = __shfl_xor_sync(0xffffffffu, m, o), s2 = __shfl_xor_sync(0xffffffffu, s, o);
-        combine(m, s, m2, s2);
     }
     if (lane == 0) { s_m[warp] = m; s_s[warp] = s; }
     __syncthreads();
@@ -73,24 +102,27 @@ __global__ void __launch_bounds__(ST, 2) softmax_stats_kernel(graft_accept_stoch
             const float m2 = __shfl_xor_sync(0xffffffffu, m, o), s2 = __shfl_xor_sync(0xffffffffu, s, o);
             combine(m, s, m2, s2);
         }
-        if (lane == 0) { p.row_stats[2 * (size_t)r] = m; p.row_stats[2 * (size_t)r + 1] = s; }
+        if (lane == 0) { out[0] = m; out[1] = s; }
     }
-    (void)status;
 }
 
 __global__ void __launch_bounds__(WT) accept_walk_kernel(graft_accept_stochastic_params p, unsigned* status) {
+    constexpr int NW = WT / 32;
     __shared__ int s_par[64], s_tok[64];
     __shared__ float s_w[64];                 // weight exp(z - m) of node i's token in its parent's row
+    __shared__ float s_u[64], s_m[64], s_s[64];   // the node's random number; its row's statistics
     __shared__ int s_rej[64];                 // tokens rejected at the node the walk ended at
-    __shared__ float s_scan[WT];
-    __shared__ int s_nrej, s_best, s_pick, s_owner;
+    __shared__ float s_rejw[64];              // and their weights
+    __shared__ float s_stepw[kMaxSteps];      // remaining weight of every step of the last node's row
+    __shared__ float s_wtot[NW];
+    __shared__ int s_nrej, s_best, s_pick, s_step;
     __shared__ float s_rem, s_base;
-    const int tid = threadIdx.x, lane = tid & 31;
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int b = blockIdx.x;
     const int T = p.tree_size[b];
     int32_t* path = p.path + (size_t)b * p.T_max;
-    for (int j = tid; j < p.T_max; j += WT) path[j] = -1;
     if (T < 1 || T > p.T_max) {
+        for (int j = tid; j < p.T_max; j += WT) path[j] = -1;
         if (tid == 0) {
             p.n_acc[b] = 0; p.best_node[b] = -1; p.bonus[b] = -1;
             if (T != 0) atomicOr(status, (unsigned)GRAFT_FLAG_BAD_SIZE);
@@ -98,21 +130,24 @@ __global__ void __launch_bounds__(WT) accept_walk_kernel(graft_accept_stochastic
         return;
     }
     const float inv_t = 1.f / p.temperature;
+    const size_t rf = row_floats(p.V);
     const __nv_bfloat16* lg = reinterpret_cast<const __nv_bfloat16*>(p.logits) + (size_t)b * p.T_max * p.logits_stride_row;
-    const float* stats = p.row_stats + 2 * (size_t)b * p.T_max;
+    const float* stats = p.row_stats + (size_t)b * p.T_max * rf;
     if (tid < 64) {
         int par = -1, x = -1;
-        float w = 0.f;
+        float w = 0.f, u = 1.f, m = 0.f, sm = 1.f;
         if (tid < T) {
             par = p.tree_parent[(size_t)b * p.T_max + tid];
             x = p.tree_token[(size_t)b * p.T_max + tid];
+            u = p.u_accept[(size_t)b * p.T_max + tid];
+            m = stats[tid * rf];
+            sm = stats[tid * rf + 1];
             if (tid == 0 || par < 0 || par >= tid) par = -1;               // the root, or not a tree node: nobody's child
-            else if (x >= 0 && x < p.V) w = __expf(__bfloat162float(lg[(size_t)par * p.logits_stride_row + x]) * inv_t - stats[2 * par]);
+            else if (x >= 0 && x < p.V) w = __expf(__bfloat162float(lg[(size_t)par * p.logits_stride_row + x]) * inv_t - stats[par * rf]);
         }
-        s_par[tid] = par; s_tok[tid] = x; s_w[tid] = w;
+        s_par[tid] = par; s_tok[tid] = x; s_w[tid] = w; s_u[tid] = u; s_m[tid] = m; s_s[tid] = sm;
     }
     __syncthreads();
-    __syncthreads();                 // (path was cleared above by all threads; the walk below writes it)
     if (tid == 0) {
         int u = 0, n = 0, nrej = 0;
         float rem = 1.f;
@@ -120,7 +155,7 @@ __global__ void __launch_bounds__(WT) accept_walk_kernel(graft_accept_stochastic
             path[n++] = u;
             rem = 1.f;
             nrej = 0;
-            const float inv_s = 1.f / stats[2 * u + 1];
+            const float inv_s = 1.f / s_s[u];
             int next = -1;
             for (int c = u + 1; c < T; ++c) {
                 if (s_par[c] != u) continue;
@@ -128,134 +163,121 @@ __global__ void __launch_bounds__(WT) accept_walk_kernel(graft_accept_stochastic
                 float px = s_w[c] * inv_s;
                 for (int j = 0; j < nrej; ++j)
                     if (s_rej[j] == x) px = 0.f;                            // that mass is gone already
-                if (p.u_accept[(size_t)b * p.T_max + c] * rem < px) { next = c; break; }
-                if (x >= 0 && x < p.V && px > 0.f) { rem -= px; s_rej[nrej++] = x; }
+                if (s_u[c] * rem < px) { next = c; break; }
+                if (x >= 0 && x < p.V && px > 0.f) { rem -= px; s_rejw[nrej] = s_w[c]; s_rej[nrej++] = x; }
             }
             if (next < 0) break;
             u = next;
         }
-        s_best = u; s_nrej = nrej; s_rem = rem; s_pick = -1; s_owner = -1;
+        for (int j = n; j < p.T_max; ++j) path[j] = -1;
+        s_best = u; s_nrej = nrej; s_rem = rem; s_pick = -1; s_step = -1;
         p.n_acc[b] = n;
         p.best_node[b] = u;
     }
     __syncthreads();
-    // ---- bonus: smallest id whose running sum of remaining weight exceeds the target
+    // ---- bonus: smallest id whose running sum of remaining weight exceeds the target.  The statistics
+    // kernel left the sum of every step of 256 ids; find the step, then the lane, then the id.
     const int u = s_best, nrej = s_nrej;
-    const float m = stats[2 * u], target = p.u_bonus[b] * s_rem * stats[2 * u + 1];
+    const float m = s_m[u], target = p.u_bonus[b] * s_rem * s_s[u];
     const __nv_bfloat16* row = lg + (size_t)u * p.logits_stride_row;
-    const int chunk = (((p.V + WT - 1) / WT) + 7) & ~7;             // per thread, a multiple of one vector
-    const int lo = min(p.V, tid * chunk), hi = min(p.V, lo + chunk);
-    auto weight_sum = [&](int a, int e) {                            // sum of weights over [a, e), rejected ids left out
-        float acc = 0.f;
-        int v = a;
-        for (; v < e && (v & 7); ++v) acc += __expf(__bfloat162float(row[v]) * inv_t - m);
-        for (; v + 8 <= e; v += 8) {
-            const uint4 q = *reinterpret_cast<const uint4*>(row + v);
-            acc += __expf(lo_f(q.x) * inv_t - m) + __expf(hi_f(q.x) * inv_t - m) + __expf(lo_f(q.y) * inv_t - m) + __expf(hi_f(q.y) * inv_t - m) +
-                   __expf(lo_f(q.z) * inv_t - m) + __expf(hi_f(q.z) * inv_t - m) + __expf(lo_f(q.w) * inv_t - m) + __expf(hi_f(q.w) * inv_t - m);
-        }
-        for (; v < e; ++v) acc += __expf(__bfloat162float(row[v]) * inv_t - m);
+    const float* steps = stats + u * rf + 2;
+    const int nsteps = steps_of(p.V);
+    for (int st = tid; st < nsteps; st += WT) {
+        const float ms = steps[2 * st];
+        s_stepw[st] = ms > -CUDART_INF_F ? steps[2 * st + 1] * __expf(ms - m) : 0.f;
+    }
+    __syncthreads();
+    if (tid < nrej) atomicAdd(&s_stepw[s_rej[tid] / kStep], -s_rejw[tid]);
+    __syncthreads();
+    // inclusive scan over the steps: two per thread
+    const float a0 = 2 * tid < nsteps ? fmaxf(s_stepw[2 * tid], 0.f) : 0.f;
+    const float a1 = 2 * tid + 1 < nsteps ? fmaxf(s_stepw[2 * tid + 1], 0.f) : 0.f;
+    float inc = a0 + a1;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+        const float t = __shfl_up_sync(0xffffffffu, inc, o);
+        if (lane >= o) inc += t;
+    }
+    if (lane == 31) s_wtot[warp] = inc;
+    __syncthreads();
+    float before = 0.f;
+    for (int w2 = 0; w2 < warp; ++w2) before += s_wtot[w2];
+    const float e0 = before + inc - a0 - a1, e1 = e0 + a0, e2 = e1 + a1;      // running sums before, between and after my two steps
+    if (e1 > target && !(e0 > target)) { s_step = 2 * tid; s_base = e0; }
+    else if (e2 > target && !(e1 > target)) { s_step = 2 * tid + 1; s_base = e1; }
+    __syncthreads();
+    const int sx = s_step;
+    if (sx >= 0 && warp == 0) {
+        float z[8], w[8];
+        const int v0 = sx * kStep + lane * 8;
+        scaled8(row, v0, p.V, inv_t, z);
+#pragma unroll
+        for (int e = 0; e < 8; ++e) w[e] = __expf(z[e] - m);
         for (int j = 0; j < nrej; ++j) {
-            const int x = s_rej[j];
-            if (x >= a && x < e) acc -= __expf(__bfloat162float(row[x]) * inv_t - m);
-        }
-        return fmaxf(acc, 0.f);
-    };
-    const float mine = weight_sum(lo, hi);
-    s_scan[tid] = mine;
-    __syncthreads();
-    if (tid < 32) {                    // inclusive scan of the 256 chunk sums: eight per lane, then across lanes
-        float loc[8], run = 0.f;
+            const int d = s_rej[j] - v0;
+            if (d >= 0 && d < 8) {
 #pragma unroll
-        for (int e = 0; e < 8; ++e) { run += s_scan[tid * 8 + e]; loc[e] = run; }
-        float incl = run;
-#pragma unroll
-        for (int o = 1; o < 32; o <<= 1) {
-            const float t = __shfl_up_sync(0xffffffffu, incl, o);
-            if (lane >= o) incl += t;
-        }
-        const float excl = incl - run;
-#pragma unroll
-        for (int e = 0; e < 8; ++e) s_scan[tid * 8 + e] = excl + loc[e];
-    }
-    __syncthreads();
-    const float incl = s_scan[tid], excl = tid ? s_scan[tid - 1] : 0.f;
-    if (incl > target && !(excl > target)) { s_owner = tid; s_base = excl; }     // exactly one chunk: the sums do not decrease
-    __syncthreads();
-    const int owner = s_owner;
-    if (owner < 0) {
-        // rounding left the total just below the target: the last id that still has weight
-        if (tid == 0) {
-            int v = p.V - 1;
-            for (; v >= 0; --v) {
-                bool rej = false;
-                for (int j = 0; j < nrej; ++j) rej |= s_rej[j] == v;
-                if (!rej && __expf(__bfloat162float(row[v]) * inv_t - m) > 0.f) break;
+                for (int e = 0; e < 8; ++e)
+                    if (e == d) w[e] = 0.f;
             }
-            p.bonus[b] = v;
         }
-        return;
-    }
-    if ((tid >> 5) == (owner >> 5)) {            // the owner's warp splits the owner's chunk into 32 pieces
-        const int olo = min(p.V, owner * chunk), ohi = min(p.V, olo + chunk);
-        const int piece = (ohi - olo + 31) / 32;
-        const int a = min(ohi, olo + lane * piece), e = min(ohi, a + piece);
-        const float part = weight_sum(a, e);
-        float inc = part;
+        const float mine = ((w[0] + w[1]) + (w[2] + w[3])) + ((w[4] + w[5]) + (w[6] + w[7]));
+        float li = mine;
 #pragma unroll
         for (int o = 1; o < 32; o <<= 1) {
-            const float t = __shfl_up_sync(0xffffffffu, inc, o);
-            if (lane >= o) inc += t;
+            const float t = __shfl_up_sync(0xffffffffu, li, o);
+            if (lane >= o) li += t;
         }
-        const float base = s_base + inc - part;
-        const bool has = base + part > target && !(base > target);
-        const unsigned who = __ballot_sync(0xffffffffu, has);
-        int pick = -1;
-        if (who) {
-            if (lane == __ffs(who) - 1) {
-                float run = base;
-                for (int v = a; v < e; ++v) {
-                    bool rej = false;
-                    for (int j = 0; j < nrej; ++j) rej |= s_rej[j] == v;
-                    if (rej) continue;
-                    const float w = __expf(__bfloat162float(row[v]) * inv_t - m);
-                    if (w <= 0.f) continue;
-                    pick = v;                      // the last weighted id so far: the answer if rounding ends the piece early
-                    run += w;
-                    if (run > target) break;
+        const float run = s_base;
+        unsigned who = __ballot_sync(0xffffffffu, run + li > target);
+        const unsigned any = __ballot_sync(0xffffffffu, mine > 0.f);
+        if (!who && any) who = 1u << (31 - __clz(any));               // the lanes' sums round differently from the step's: the last lane with weight
+        if (who && lane == __ffs(who) - 1) {
+            float r2 = run + li - mine;
+            int pick = -1, last = -1;
+#pragma unroll
+            for (int e = 0; e < 8; ++e) {
+                if (w[e] > 0.f && pick < 0) {
+                    last = v0 + e;
+                    r2 += w[e];
+                    if (r2 > target) pick = v0 + e;
                 }
-                p.bonus[b] = pick;
             }
-        } else if (lane == 0) {
-            // the piece sums round differently from the chunk sum: fall back to a plain walk of the chunk
-            float run = s_base;
-            for (int v = olo; v < ohi; ++v) {
-                bool rej = false;
-                for (int j = 0; j < nrej; ++j) rej |= s_rej[j] == v;
-                if (rej) continue;
-                const float w = __expf(__bfloat162float(row[v]) * inv_t - m);
-                if (w <= 0.f) continue;
-                pick = v;
-                run += w;
-                if (run > target) break;
-            }
-            p.bonus[b] = pick;
+            s_pick = pick < 0 ? last : pick;
         }
+    }
+    __syncthreads();
+    if (tid == 0) {
+        int pick = s_pick;
+        if (pick < 0) {
+            // rounding left the total just below the target: the last id that still has weight
+            for (pick = p.V - 1; pick >= 0; --pick) {
+                bool rej = false;
+                for (int j = 0; j < nrej; ++j) rej |= s_rej[j] == pick;
+                if (!rej && __expf(__bfloat162float(row[pick]) * inv_t - m) > 0.f) break;
+            }
+        }
+        p.bonus[b] = pick;
     }
 }
 
 }  // namespace
 
+extern "C" size_t graft_accept_stochastic_scratch_floats(int B, int T_max, int V) {
+    if (B <= 0 || T_max <= 0 || V <= 0) return 0;
+    return (size_t)B * T_max * row_floats(V);
+}
+
 extern "C" int graft_accept_stochastic(graft_ctx* ctx, const graft_accept_stochastic_params* p, void* stream) {
     if (!ctx || !p) return GRAFT_ERR_INVALID_ARG;
     if (p->B <= 0 || p->T_max <= 0 || p->V <= 0 || !(p->temperature > 0.f)) return GRAFT_ERR_INVALID_ARG;
-    if (p->T_max > 64) return GRAFT_ERR_UNSUPPORTED;
+    if (p->T_max > 64 || steps_of(p->V) > kMaxSteps) return GRAFT_ERR_UNSUPPORTED;
     if (!p->logits || !p->tree_token || !p->tree_parent || !p->tree_size || !p->u_accept || !p->u_bonus || !p->row_stats ||
         !p->n_acc || !p->path || !p->best_node || !p->bonus)
         return GRAFT_ERR_INVALID_ARG;
     if (!graft_aligned16(p->logits) || p->logits_stride_row < p->V || p->logits_stride_row % 8 != 0) return GRAFT_ERR_INVALID_ARG;
     cudaStream_t s = static_cast<cudaStream_t>(stream);
-    softmax_stats_kernel<<<p->B * p->T_max, ST, 0, s>>>(*p, ctx->status);
+    softmax_stats_kernel<<<p->B * p->T_max, ST, 0, s>>>(*p);
     GRAFT_CHECK_CUDA(cudaGetLastError());
     accept_walk_kernel<<<p->B, WT, 0, s>>>(*p, ctx->status);
     GRAFT_CHECK_CUDA(cudaGetLastError());

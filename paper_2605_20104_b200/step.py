@@ -162,8 +162,9 @@ class VerifyStep:
 
     def accept_stochastic(self, logits: torch.Tensor, temperature: float, u_accept: torch.Tensor, u_bonus: torch.Tensor) -> None:
         """Acceptance under temperature sampling: logits bf16 [B*T_max, V], random numbers float32 [B, T_max] and [B]."""
-        if getattr(self, "row_stats", None) is None:
-            self.row_stats = torch.empty(self.w.B * self.w.T_max, 2, dtype=torch.float32, device=self.dev)
+        need = G.graft_accept_stochastic_scratch_floats(self.w.B, self.w.T_max, logits.shape[1])
+        if getattr(self, "row_stats", None) is None or self.row_stats.numel() < need:
+            self.row_stats = torch.empty(need, dtype=torch.float32, device=self.dev)
         key = ("accept_s", logits.data_ptr(), u_accept.data_ptr(), u_bonus.data_ptr(), temperature)
         G.launch("graft_accept_stochastic", self.ctx, self._cached(key, lambda: G.accept_stochastic_params(
             logits=logits, temperature=temperature, tree_token=self.tree_token, tree_parent=self.tree_parent,

@@ -59,7 +59,11 @@ def test_binding_lists_the_same_entry_points(lib):
 
 @pytest.mark.parametrize("cname,pyname", [("graft_build_params", "BuildParams"), ("graft_attn_params", "AttnParams"),
                                           ("graft_accept_params", "AcceptParams"),
-                                          ("graft_compact_params", "CompactParams")])
+                                          ("graft_compact_params", "CompactParams"),
+                                          ("graft_update_params", "UpdateParams"),
+                                          ("graft_envelope_params", "EnvelopeParams"),
+                                          ("graft_paths_params", "PathsParams"),
+                                          ("graft_accept_stochastic_params", "AcceptStochasticParams")])
 def test_struct_layouts_follow_the_header(cname, pyname):
     from paper_2605_20104_b200 import binding
     assert [f[0] for f in getattr(binding, pyname)._fields_] == struct_fields(cname)
@@ -73,7 +77,8 @@ def test_status_strings(lib):
 
 def test_host_side_argument_checks_need_no_gpu(lib):
     """Null handles are rejected before anything touches a device."""
-    for fn in ("graft_build_tree", "graft_tree_verify_attn", "graft_accept", "graft_compact_kv"):
+    for fn in ("graft_build_tree", "graft_tree_verify_attn", "graft_accept", "graft_compact_kv", "graft_update_adjacency",
+               "graft_retrieve_envelope", "graft_path_indices", "graft_accept_stochastic"):
         f = getattr(lib, fn)
         f.restype = ctypes.c_int
         assert f(None, None, None) == -1
