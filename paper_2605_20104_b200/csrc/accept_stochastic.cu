@@ -62,35 +62,60 @@ __global__ void __launch_bounds__(ST, 2) softmax_stats_kernel(graft_accept_stoch
     float* out = p.row_stats + (size_t)r * row_floats(p.V);
     const int nsteps = steps_of(p.V);
     float m = -CUDART_INF_F, s = 0.f;
-    constexpr int NWS = ST / 32, kFlight = 4;          // steps a warp has in flight
+    constexpr int NWS = ST / 32, kFlight = 4;          // steps a warp has in flight; they share one reference maximum
     for (int st = warp; st < nsteps; st += kFlight * NWS) {
         float z[kFlight][8];
+        float vm = -CUDART_INF_F;
+        if ((st + (kFlight - 1) * NWS + 1) * kStep <= p.V) {
+            // all four steps lie inside the row: four unconditional 16-byte loads in flight
+            uint4 q[kFlight];
 #pragma unroll
-        for (int h = 0; h < kFlight; ++h)
-            if (st + h * NWS < nsteps) scaled8(row, (st + h * NWS) * kStep + lane * 8, p.V, inv_t, z[h]);
+            for (int h = 0; h < kFlight; ++h) q[h] = __ldcs(reinterpret_cast<const uint4*>(row + (st + h * NWS) * kStep + lane * 8));
+#pragma unroll
+            for (int h = 0; h < kFlight; ++h) {
+                z[h][0] = lo_f(q[h].x) * inv_t; z[h][1] = hi_f(q[h].x) * inv_t; z[h][2] = lo_f(q[h].y) * inv_t; z[h][3] = hi_f(q[h].y) * inv_t;
+                z[h][4] = lo_f(q[h].z) * inv_t; z[h][5] = hi_f(q[h].z) * inv_t; z[h][6] = lo_f(q[h].w) * inv_t; z[h][7] = hi_f(q[h].w) * inv_t;
+#pragma unroll
+                for (int e = 0; e < 8; ++e) vm = fmaxf(vm, z[h][e]);
+            }
+        } else {
+#pragma unroll
+            for (int h = 0; h < kFlight; ++h) {
+                if (st + h * NWS < nsteps) {
+                    scaled8(row, (st + h * NWS) * kStep + lane * 8, p.V, inv_t, z[h]);
+#pragma unroll
+                    for (int e = 0; e < 8; ++e) vm = fmaxf(vm, z[h][e]);
+                } else {
+#pragma unroll
+                    for (int e = 0; e < 8; ++e) z[h][e] = -CUDART_INF_F;
+                }
+            }
+        }
+#pragma unroll
+        for (int o = 16; o; o >>= 1) vm = fmaxf(vm, __shfl_xor_sync(0xffffffffu, vm, o));
+        float add[kFlight];
+#pragma unroll
+        for (int h = 0; h < kFlight; ++h) {
+            add[h] = 0.f;
+            if (vm > -CUDART_INF_F) {
+#pragma unroll
+                for (int e = 0; e < 8; ++e) add[h] += __expf(z[h][e] - vm);
+            }
+        }
+#pragma unroll
+        for (int o = 16; o; o >>= 1)
+#pragma unroll
+            for (int h = 0; h < kFlight; ++h) add[h] += __shfl_xor_sync(0xffffffffu, add[h], o);
+        float tot = 0.f;
 #pragma unroll
         for (int h = 0; h < kFlight; ++h) {
             const int sx = st + h * NWS;
             if (sx < nsteps) {
-                float vm = z[h][0];
-#pragma unroll
-                for (int e = 1; e < 8; ++e) vm = fmaxf(vm, z[h][e]);
-#pragma unroll
-                for (int o = 16; o; o >>= 1) vm = fmaxf(vm, __shfl_xor_sync(0xffffffffu, vm, o));
-                float add = 0.f;
-                if (vm > -CUDART_INF_F) {
-#pragma unroll
-                    for (int e = 0; e < 8; ++e) add += __expf(z[h][e] - vm);
-                }
-#pragma unroll
-                for (int o = 16; o; o >>= 1) add += __shfl_xor_sync(0xffffffffu, add, o);
-                if (lane == 0) {
-                    out[2 + 2 * sx] = vm;
-                    out[2 + 2 * sx + 1] = add;
-                }
-                combine(m, s, vm, add);
+                if (lane == h) { out[2 + 2 * sx] = vm; out[2 + 2 * sx + 1] = add[h]; }
+                tot += add[h];
             }
         }
+        combine(m, s, vm, tot);
     }
     if (lane == 0) { s_m[warp] = m; s_s[warp] = s; }
     __syncthreads();
