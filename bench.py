@@ -169,6 +169,37 @@ def time_workload(name, steps, warmup, device, variant, rank=0):
                 flags=flags, tree=tree)
 
 
+def time_graph_replay(st, steps, warmup, variant):
+    """The same step captured once per rotating cache in a CUDA graph and replayed: device time per step without
+    the launch gaps of four separate calls (the launch configuration is fixed by the shapes, so a serving loop
+    can do this)."""
+    vs, caches, n_rot = st["vs"], st["caches"], st["n_rot"]
+    graphs = []
+    side = torch.cuda.Stream()
+    for kc, vc in caches:
+        vs.Kc, vs.Vc = kc, vc
+        side.wait_stream(torch.cuda.current_stream())
+        with torch.cuda.stream(side):                 # every launch once outside a capture (module loading, attributes)
+            vs.build(); vs.attn(variant); vs.accept(); vs.compact()
+        torch.cuda.current_stream().wait_stream(side)
+        torch.cuda.synchronize()
+        g = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(g):
+            vs.build(); vs.attn(variant); vs.accept(); vs.compact()
+        graphs.append(g)
+    for i in range(warmup):
+        graphs[i % n_rot].replay()
+    torch.cuda.synchronize()
+    t0, t1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    torch.cuda._sleep(int(3e6))
+    t0.record()
+    for i in range(steps):
+        graphs[i % n_rot].replay()
+    t1.record()
+    torch.cuda.synchronize()
+    return t0.elapsed_time(t1) / steps * 1e3
+
+
 def time_update(st, steps, warmup):
     """graft_update_adjacency (the matrix refresh that follows the verify pass) alone, on the workload's trees and
     generator-shaped target logits; three logits buffers in rotation (> L2 together)."""
@@ -491,6 +522,7 @@ def main():
         upd["frac_of_measured"] = upd["GBps"] / peak
         line["update_adjacency"] = upd
         line["index_kernels"] = time_index_kernels(st, min(args.steps, 50), 5)
+        line["graph_replay_us_per_step"] = time_graph_replay(st, min(args.steps, 100), 5, variant)
         acs = time_accept_stochastic(st, min(args.steps, 50), 5)
         acs["frac_of_measured"] = acs["GBps"] / peak
         line["accept_stochastic"] = acs

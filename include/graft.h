@@ -35,6 +35,9 @@
  *   - Padding (so that whole buffers compare bit for bit): nodes i >= T_b have token -1, parent -1,
  *     pos 0, anc 0, src INT32_MIN; path[j >= n_acc] = -1; O rows t >= T_b are zero, LSE there -inf.
  *   - One graft_ctx per stream; calls on one ctx must not overlap on the GPU.
+ *   - Launch configurations depend only on the scalars of a params struct (shapes, variant), never on device
+ *     data, and no call keeps per-call state on the host: a sequence of calls can be captured in a CUDA graph
+ *     once and replayed after the contents of its buffers changed (lengths, trees, K/V, random numbers).
  */
 #ifndef GRAFT_H_
 #define GRAFT_H_

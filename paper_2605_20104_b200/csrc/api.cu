@@ -35,7 +35,6 @@ extern "C" int graft_create(graft_ctx** out, int device, void* workspace, size_t
     c->ws = workspace;
     c->ws_bytes = workspace_bytes;
     c->status = static_cast<unsigned*>(workspace);
-    c->epoch = 0;
     *out = c;
     return GRAFT_OK;
 }

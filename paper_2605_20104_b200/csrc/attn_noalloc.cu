@@ -24,7 +24,6 @@ struct DeviceSetup {
     bool ready = false;
     void* scratch = nullptr;       // device address of g_noalloc_scratch on this device
     int num_sms = 0;
-    unsigned epoch = 0;            // attention calls made on this device's scratch so far
 };
 DeviceSetup g_setup[kMaxDevices];
 std::mutex g_setup_mutex;
@@ -83,14 +82,12 @@ extern "C" int graft_tree_verify_attn_noalloc(const graft_attn_params* p, void* 
     ctx.ws = s->scratch;
     ctx.ws_bytes = kScratchBytes;
     ctx.status = static_cast<unsigned*>(s->scratch);
-    ctx.epoch = s->epoch;
 
     cudaStream_t st = static_cast<cudaStream_t>(stream);
-    // the array keeps the previous call's contents; only the status word has to start at zero
-    // (partials are always written before they are read)
-    GRAFT_CHECK_CUDA(cudaMemsetAsync(ctx.status, 0, GRAFT_WS_HEADER, st));
+    // the array keeps the previous call's contents (among them the number of the last call, in the header);
+    // only the status word has to start at zero (partials are always written before they are read)
+    GRAFT_CHECK_CUDA(cudaMemsetAsync(ctx.status, 0, 16, st));
     rc = graft_tree_verify_attn(&ctx, p, stream);
-    s->epoch = ctx.epoch;
     if (rc == GRAFT_ERR_WORKSPACE_TOO_SMALL) return GRAFT_ERR_SCRATCH_LIMIT;
     if (rc != GRAFT_OK) return rc;
     if (device_flags_out)

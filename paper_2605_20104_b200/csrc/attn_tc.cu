@@ -80,7 +80,8 @@ struct TcArgs {
     CutHeader* cut;     // this call's cut, followed by B SeqEntry records
     float* partial;     // 2 slots per CTA
     int* counters;      // [B * Hkv * 8 * 2] arrivals per (item, 128-row half) for the in-kernel merge: (epoch << 8) | count
-    unsigned epoch;     // number of this call (24 bits): stale counts of earlier calls are ignored
+    unsigned epoch;     // number of this call (24 bits): stale counts of earlier calls are ignored; every kernel reads it from call_no
+    unsigned* call_no;  // [0] number of the last finished call on this workspace, [1] CTAs of the running call that are done
     int inkernel;       // the kernel merges the parts of an item itself (last arrival); else merge_streamk_kernel follows
     int G;
     int q_tma;          // Q tiles are fetched by TMA (group size divides 128); otherwise threads copy them
@@ -221,6 +222,21 @@ __device__ __forceinline__ int item_id(const graft_attn_params& p, int b, int h,
 // what a slot descriptor holds: the item, stamped with the call's number, so that a descriptor left by an earlier call
 // (a worker that has not yet reset its own in this call) never matches
 __device__ __forceinline__ int item_tag(const TcArgs& a, int id) { return id | (int)((a.epoch & 0x7fu) << 24); }
+// The number of a call lives in the workspace, not in a kernel argument, so that a captured launch can be
+// replayed: every CTA of the attention kernel takes "last finished call + 1" on entry, and the last CTA to
+// leave publishes it (the merge kernel, which runs after the whole grid, reads it back).
+__device__ __forceinline__ unsigned next_call_no(const TcArgs& a) {
+    const unsigned e = (__ldcg(a.call_no) + 1u) & 0xffffffu;
+    return e ? e : 1u;
+}
+__device__ __forceinline__ void cta_leaves(const TcArgs& a) {          // one thread per CTA, after the CTA's last use of the number
+    __threadfence();
+    if (atomicAdd(a.call_no + 1, 1u) == gridDim.x - 1) {
+        a.call_no[1] = 0u;
+        __threadfence();
+        atomicExch(a.call_no, a.epoch);
+    }
+}
 
 struct Seg {
     int b, h, rb;            // item
@@ -563,10 +579,14 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap kmap, const __grid_constant__
                 tma_load_5d(sQ + blk * TILE_BYTES + half * HALF_BYTES, &qmap, half * 64, 0, (row0 + blk * 128) / G, sg.h, sg.b, bar(BAR_Q));
     };
 
+    a.epoch = next_call_no(a);
     if (warp == 0) plan_first(a, G, (int)blockIdx.x, (int)gridDim.x, blockIdx.x == 0, true, s_plan);
     if (threadIdx.x == 0) s_abort = 0;
     __syncthreads();
-    if (s_nseg == 0) return;                      // nothing for this CTA (short batch)
+    if (s_nseg == 0) {                            // nothing for this CTA (short batch)
+        if (threadIdx.x == 0) cta_leaves(a);
+        return;
+    }
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");      // the merge kernel may be set up from now on (it waits for this grid to end)
 
     // ring load n of a segment's tile t: K (which = 0) or V (which = 1)
@@ -932,6 +952,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap kmap, const __grid_constant__
         tc_fence_after();
         asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(512u) : "memory");
     }
+    if (threadIdx.x == 0) cta_leaves(a);
 }
 
 // Rows of padding nodes (t >= T_b; all rows of a sequence whose sizes are out of range) are zero with LSE -inf.
@@ -1405,8 +1426,9 @@ attn_tc_pair_kernel(const __grid_constant__ CUtensorMap kmap, const __grid_const
     const uint32_t rank = cluster_ctarank();          // 0: leader (issues the MMAs), 1: peer
     const int worker = (int)(blockIdx.x >> 1), nworkers = (int)(gridDim.x >> 1);
 
+    a.epoch = next_call_no(a);
     if ((smem_u32(smem_raw) & 1023u) != 0) {          // the tiles would miss their alignment: refuse to run (both CTAs alike)
-        if (threadIdx.x == 0) atomicOr(status, (unsigned)GRAFT_FLAG_INTERNAL);
+        if (threadIdx.x == 0) { atomicOr(status, (unsigned)GRAFT_FLAG_INTERNAL); cta_leaves(a); }
         return;
     }
     const uint32_t sQ = smem_u32(smem_raw) + kCtrlBytes;
@@ -1421,7 +1443,10 @@ attn_tc_pair_kernel(const __grid_constant__ CUtensorMap kmap, const __grid_const
     if (warp == 0) plan_first(a, G, worker, nworkers, blockIdx.x == 0, rank == 0, plan);
     if (threadIdx.x == 0) ctrl.abort = 0;
     __syncthreads();
-    if (plan.nseg == 0) return;                       // nothing for this pair (short batch); no cluster operation was started
+    if (plan.nseg == 0) {                             // nothing for this pair (short batch); no cluster operation was started
+        if (threadIdx.x == 0) cta_leaves(a);
+        return;
+    }
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");      // the merge kernel may be set up from now on (it waits for this grid to end)
 
     if (threadIdx.x == 0) {
@@ -1587,6 +1612,7 @@ attn_tc_pair_kernel(const __grid_constant__ CUtensorMap kmap, const __grid_const
         tc_fence_after();
         asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(512u) : "memory");
     }
+    if (threadIdx.x == 0) cta_leaves(a);
 }
 
 // ---------------------------------------------------------------------------------------------------
@@ -1625,8 +1651,9 @@ attn_tc_rb_kernel(const __grid_constant__ CUtensorMap kmap, const __grid_constan
     const int rank = (int)(blockIdx.x & 1);           // which 128-row block of an item
     const int worker = (int)(blockIdx.x >> 1), nworkers = (int)(gridDim.x >> 1);
 
+    a.epoch = next_call_no(a);
     if ((smem_u32(smem_raw) & 1023u) != 0) {          // the tiles would miss their alignment: refuse to run
-        if (threadIdx.x == 0) atomicOr(status, (unsigned)GRAFT_FLAG_INTERNAL);
+        if (threadIdx.x == 0) { atomicOr(status, (unsigned)GRAFT_FLAG_INTERNAL); cta_leaves(a); }
         return;
     }
     const uint32_t sQ = smem_u32(smem_raw) + kCtrlBytes;
@@ -1641,7 +1668,10 @@ attn_tc_rb_kernel(const __grid_constant__ CUtensorMap kmap, const __grid_constan
     if (warp == 0) plan_first(a, G, worker, nworkers, blockIdx.x == 0, rank == 0, plan);
     if (threadIdx.x == 0) ctrl.abort = 0;
     __syncthreads();
-    if (plan.nseg == 0) return;                       // nothing for this worker (short batch)
+    if (plan.nseg == 0) {                             // nothing for this worker (short batch)
+        if (threadIdx.x == 0) cta_leaves(a);
+        return;
+    }
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");      // the merge kernel may be set up from now on (it waits for this grid to end)
 
     if (threadIdx.x == 0) {
@@ -1827,6 +1857,7 @@ attn_tc_rb_kernel(const __grid_constant__ CUtensorMap kmap, const __grid_constan
         tc_fence_after();
         asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(512u) : "memory");
     }
+    if (threadIdx.x == 0) cta_leaves(a);
 }
 
 // ---------------------------------------------------------------------------------------------------
@@ -1840,6 +1871,7 @@ constexpr int kMergeWarps = 8;       // warps per CTA; rows per CTA is a launch 
 
 __global__ void __launch_bounds__(kMergeWarps * 32, 4) merge_streamk_kernel(TcArgs a, int rows_per_cta, unsigned* status) {
     asm volatile("griddepcontrol.wait;" ::: "memory");      // launched early: nothing is read before the attention kernel is complete
+    a.epoch = __ldcg(a.call_no);                            // the call the attention kernel just finished
     const graft_attn_params& p = a.p;
     const int G = a.G;
     const int rows_pad = p.T_max * G;
@@ -2080,9 +2112,8 @@ int graft_attn_tc_launch(graft_ctx* ctx, const graft_attn_params* p, cudaStream_
     a.cut = reinterpret_cast<CutHeader*>(reinterpret_cast<char*>(ctx->ws) + GRAFT_WS_HEADER + kDescBytes);
     a.counters = reinterpret_cast<int*>(reinterpret_cast<char*>(ctx->ws) + GRAFT_WS_HEADER + kDescBytes + cut_bytes(p->B));
     a.partial = reinterpret_cast<float*>(reinterpret_cast<char*>(ctx->ws) + GRAFT_WS_HEADER + kDescBytes + cut_bytes(p->B) + counter_bytes(p->B, p->Hkv));
-    ctx->epoch = (ctx->epoch + 1u) & 0xffffffu;
-    if (ctx->epoch == 0u) ctx->epoch = 1u;
-    a.epoch = ctx->epoch;
+    a.epoch = 0u;
+    a.call_no = ctx->status + 4;            // two words of the workspace header
     // Merge in the kernel (by the last part of an item to arrive) when items are cut into two or three parts: that CTA
     // reads all parts of its 128 rows alone, which then beats a second launch (measured: -15 % on a batch of eight 4K
     // contexts, -10 % on the ragged batch of sixteen; but +2 % on four 64K sequences cut into five parts each and

@@ -10,7 +10,6 @@ struct graft_ctx {
     void* ws;           // caller-owned device workspace
     size_t ws_bytes;
     unsigned* status;   // device status word = first word of the workspace
-    unsigned epoch;     // number of the last attention call on this context (stamps the in-kernel merge's counters)
 };
 
 // the first GRAFT_WS_HEADER bytes of the workspace are reserved (status word)
