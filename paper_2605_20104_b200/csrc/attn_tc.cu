@@ -83,6 +83,7 @@ struct TcArgs {
     unsigned epoch;     // number of this call (24 bits): stale counts of earlier calls are ignored; every kernel reads it from call_no
     unsigned* call_no;  // [0] number of the last finished call on this workspace, [1] CTAs of the running call that are done
     int inkernel;       // the kernel merges the parts of an item itself (last arrival); else merge_streamk_kernel follows
+    int single;         // row-block kernel: every item has one 128-row block (T_max * G <= 128), so every CTA is a worker of its own
     int G;
     int q_tma;          // Q tiles are fetched by TMA (group size divides 128); otherwise threads copy them
     int prof_cta;       // experiments: CTA whose timeline is recorded
@@ -1648,8 +1649,10 @@ attn_tc_rb_kernel(const __grid_constant__ CUtensorMap kmap, const __grid_constan
     const graft_attn_params& p = a.p;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int G = a.G;
-    const int rank = (int)(blockIdx.x & 1);           // which 128-row block of an item
-    const int worker = (int)(blockIdx.x >> 1), nworkers = (int)(gridDim.x >> 1);
+    // two CTAs per worker, one 128-row block each; with a single block per item (chains and other small trees) a
+    // partner would only repeat the copies, so every CTA walks its own tiles
+    const int rank = a.single ? 0 : (int)(blockIdx.x & 1);           // which 128-row block of an item
+    const int worker = a.single ? (int)blockIdx.x : (int)(blockIdx.x >> 1), nworkers = a.single ? (int)gridDim.x : (int)(gridDim.x >> 1);
 
     a.epoch = next_call_no(a);
     if ((smem_u32(smem_raw) & 1023u) != 0) {          // the tiles would miss their alignment: refuse to run
@@ -2121,7 +2124,9 @@ int graft_attn_tc_launch(graft_ctx* ctx, const graft_attn_params* p, cudaStream_
     // sequence, so there are about workers / (B * H_kv) + 1 parts per item; the kernel merges when that is below 2.5.
     a.G = G;
     a.q_tma = q_tma ? 1 : 0;
-    a.inkernel = (use_pair || use_rb) && ctx->num_sms / 2 <= 2 * (long long)p->B * p->Hkv ? 1 : 0;
+    a.single = use_rb && p->T_max * G <= 128 ? 1 : 0;
+    const int workers = a.single ? ctx->num_sms : ctx->num_sms / 2;
+    a.inkernel = (use_pair || use_rb) && workers <= 2 * (long long)p->B * p->Hkv ? 1 : 0;
     a.prof_cta = 0;
 #ifdef GRAFT_TC_EXPERIMENTS
     if (getenv("GRAFT_TC_PROF_CTA")) a.prof_cta = atoi(getenv("GRAFT_TC_PROF_CTA"));
@@ -2135,7 +2140,7 @@ int graft_attn_tc_launch(graft_ctx* ctx, const graft_attn_params* p, cudaStream_
         if (pairs > ctx->num_sms / 2) pairs = ctx->num_sms / 2;       // the workspace has two slots per SM
         attn_tc_pair_kernel<<<2 * pairs, P_NTHREADS, P_SMEM_DYN, stream>>>(kmap, vmap, qmap, a, ctx->status);
     } else if (use_rb) {
-        attn_tc_rb_kernel<<<ctx->num_sms & ~1, R_NTHREADS, R_SMEM_DYN, stream>>>(kmap, vmap, qmap, a, ctx->status);
+        attn_tc_rb_kernel<<<a.single ? ctx->num_sms : ctx->num_sms & ~1, R_NTHREADS, R_SMEM_DYN, stream>>>(kmap, vmap, qmap, a, ctx->status);
     } else
     attn_tc_kernel<<<grid, NTHREADS, SMEM_DYN, stream>>>(kmap, vmap, qmap, a, ctx->status);
     GRAFT_CHECK_CUDA(cudaGetLastError());

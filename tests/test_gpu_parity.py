@@ -402,3 +402,16 @@ def test_invalid_sequence_inside_a_batch(orc, G, Step):
             err = np.abs(O[b, :20] - out["O"][b, :20])
             assert err.max() <= MAX_ABS and err.mean() <= MEAN_ABS
             assert (O[b, 20:] == 0).all()
+
+
+@pytest.mark.parametrize("variant", ["auto", "l2pair", "one", "pair", "mma"])
+@pytest.mark.parametrize("B,L0", [(1, 20000), (6, 3000)])
+def test_chain_only_trees(orc, G, Step, variant, B, L0):
+    """Chains of 16 nodes (the tail-block proposals): one 128-row block per KV head, the case in which every CTA of the
+    row-block kernel walks tiles of its own; a single long sequence is cut across all of them, a batch merges in place."""
+    rng = np.random.default_rng(B)
+    parents = [W.chain_parents(int(n)) for n in ([16] if B == 1 else rng.integers(1, 17, size=B))]
+    L = [L0] if B == 1 else [int(x) for x in rng.integers(100, L0, size=B)]
+    w = W.custom(parents, Hq=40, Hkv=8, d=128, L=L, T_max=16, seed=40 + B)
+    rows = sample_rows(np.random.default_rng(B), orc.build_tree(w)["tree_size"], w.Hq, 300)
+    full_case(orc, G, Step, w, variant, rows=rows)
