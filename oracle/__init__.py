@@ -47,7 +47,7 @@ class _BuildArgs(C.Structure):
         ("ckpt_depth", _i32p), ("ckpt_keep", _i32p), ("ckpt_log_tau", _f32p), ("tmpl_offset", _i32p),
         ("tmpl_parent", _i32p), ("tmpl_rank", _i32p),
         ("tree_token", _i32p), ("tree_parent", _i32p), ("tree_pos", _i32p), ("tree_src", _i32p),
-        ("tree_anc", _u64p), ("tree_size", _i32p)]
+        ("tree_anc", _u64p), ("tree_size", _i32p), ("attach_tail", C.c_int)]
 
 
 class _AttnArgs(C.Structure):
@@ -122,7 +122,8 @@ def build_tree(w) -> dict:
                    tmpl_parent=_p(keep["tp"], _i32p, np.int32), tmpl_rank=_p(keep["tr"], _i32p, np.int32),
                    tree_token=_p(out["tree_token"], _i32p, np.int32), tree_parent=_p(out["tree_parent"], _i32p, np.int32),
                    tree_pos=_p(out["tree_pos"], _i32p, np.int32), tree_src=_p(out["tree_src"], _i32p, np.int32),
-                   tree_anc=_p(out["tree_anc"], _u64p, np.uint64), tree_size=_p(out["tree_size"], _i32p, np.int32))
+                   tree_anc=_p(out["tree_anc"], _u64p, np.uint64), tree_size=_p(out["tree_size"], _i32p, np.int32),
+                   attach_tail=int(bool(getattr(w, "attach_tail", False))))
     out["flags"] = int(lib().orc_build_tree(C.byref(a)))
     return out
 

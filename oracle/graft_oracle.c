@@ -69,6 +69,7 @@ typedef struct {
     int32_t *tree_token, *tree_parent, *tree_pos, *tree_src; /* [B, T_max] */
     uint64_t *tree_anc;                                      /* [B, T_max] */
     int32_t *tree_size;                                      /* [B] */
+    int attach_tail;         /* 0: template nodes with parent -1 hang off the root; 1: off the last kept node (tail grafting) */
 } orc_build_args;
 
 static int popcount64(uint64_t x) {
@@ -208,7 +209,10 @@ unsigned orc_build_tree(const orc_build_args *a) {
                 int tp = a->tmpl_parent[t_lo + u], r = a->tmpl_rank[t_lo + u];
                 int j = K_kept + u, ok = 1;
                 if (tp < -1 || tp >= u || r < 0 || r >= a->k) { ok = 0; flags |= ORC_FLAG_BAD_TEMPLATE; }
-                int p = (!ok || tp == -1) ? 0 : K_kept + tp;
+                /* root-centred template, or (block drafters' "keep the reliable prefix and attach retrieved tokens to the
+                   tail of the remaining chain") the template continues the last kept node */
+                const int attach = a->attach_tail ? K_kept - 1 : 0;
+                int p = (!ok || tp == -1) ? attach : K_kept + tp;
                 int ptok = o_tok[p], x = -1;
                 if (ok && ptok >= 0) {
                     x = a->M[(size_t)ptok * a->k + r];

@@ -191,6 +191,7 @@ class Workload:
     tmpl_offset: Optional[np.ndarray] = None     # int32 [n_ckpt + 1]
     tmpl_parent: np.ndarray = field(default_factory=lambda: np.zeros(0, np.int32))
     tmpl_rank: np.ndarray = field(default_factory=lambda: np.zeros(0, np.int32))
+    attach_tail: bool = False                    # template nodes with parent -1 continue the last kept node instead of the root
     # acceptance recipe
     p_draft: float = 0.75
     p_graft: float = 0.9
@@ -438,6 +439,22 @@ def config(cfg: str, *, B: Optional[int] = None, L: Optional[int] = None,
                         keep_count=((T_b + 1) // 2).astype(np.int32), k_max=T_b,
                         tmpl_parent=tp, tmpl_rank=tr, p_draft=0.65, p_graft=0.65, seed=seed)
     raise KeyError(cfg)
+
+
+def tail_block(B: int = 4, L: int = 65536, block: int = 16, *, Hq: int = 40, Hkv: int = 8, d: int = 128, V: int = 151936,
+               k: int = 8, seed: int = 16) -> Workload:
+    """Block drafter with tail grafting: a drafted chain of `block` tokens whose cumulative scores fall along the
+    chain, the first keep_count[b] ~ U{4..block} of them are kept (top-k by score on a chain = a prefix) and the
+    rank-0 chain of retrieved tokens fills the block from the last kept token on."""
+    rng = np.random.default_rng(np.random.PCG64(seed))
+    tok, par, sc, nd = _pack_trees([chain_parents(block)] * B, block, V, rng)
+    sc[:] = -np.cumsum(rng.random((B, block)).astype(np.float32), axis=1)       # strictly decreasing along the chain
+    tp, tr = chains_template([block])
+    return Workload(name="tail-block", B=B, Hq=Hq, Hkv=Hkv, d=d, S_cap=L + block, T_max=block, N_max=block, K_max=block,
+                    V=V, k=k, scale=float(np.float32(1.0 / math.sqrt(d))), seq_len=np.full(B, L, np.int32),
+                    draft_token=tok, draft_parent=par, draft_score=sc, n_draft=nd, M=_random_M(rng, V, k, 0.02),
+                    mode=MODE_TOPK, keep_count=rng.integers(4, block + 1, size=B).astype(np.int32), tmpl_parent=tp,
+                    tmpl_rank=tr, attach_tail=True, p_draft=0.8, p_graft=0.7, seed=seed, std=0.5)
 
 
 def custom(parents: List[np.ndarray], *, Hq: int, Hkv: int, d: int, L: Sequence[int], V: int = 1000,

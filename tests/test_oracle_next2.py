@@ -181,3 +181,28 @@ def test_acceptance_over_paths_equals_acceptance_over_parents(cfg):
             best = max(best, n)
         # the accepted path counts the root
         assert int(acc["n_acc"][b]) == (best + 1 if tree["tree_size"][b] > 0 else 0)
+
+
+def test_tail_grafting_continues_the_kept_prefix():
+    """Block drafter with tail grafting: the kept prefix of the drafted chain, then the rank-0 chain of the
+    adjacency matrix from the last kept token on; the result is again one chain of the block's length."""
+    w = W.tail_block(B=6, L=300, block=16, V=997)
+    tree = oracle.build_tree(w)
+    assert tree["flags"] == 0
+    for b in range(w.B):
+        keep = int(w.keep_count[b])
+        assert tree["tree_size"][b] == 16
+        assert tree["tree_parent"][b].tolist() == [-1] + list(range(15))            # one chain
+        assert tree["tree_token"][b, :keep].tolist() == w.draft_token[b, :keep].tolist()
+        x = int(w.draft_token[b, keep - 1])
+        for i in range(keep, 16):                                                     # x_{i} = M[x_{i-1}, 0], -1 propagates
+            x = int(w.M[x, 0]) if x >= 0 else -1
+            assert tree["tree_token"][b, i] == x
+        assert tree["tree_pos"][b].tolist() == list(range(300, 316))
+        assert tree["tree_src"][b].tolist() == list(range(keep)) + [-1 - u for u in range(16 - keep)]
+    # the same template hung off the root instead gives a star of two chains
+    w.attach_tail = False
+    root = oracle.build_tree(w)
+    b = int(np.argmin(w.keep_count))
+    keep = int(w.keep_count[b])
+    assert root["tree_parent"][b, keep] == 0 and root["tree_token"][b, keep] == w.M[w.draft_token[b, 0], 0]
