@@ -164,6 +164,11 @@ typedef struct {
     int N_env;
     const int32_t* env_token;    /* [B, N_env] or NULL */
     const int32_t* tmpl_env;     /* [N_tmpl] */
+    /* tail grafting for block drafters (the block-drafter appendix: keep the reliable prefix of the drafted chain
+       "and attach retrieved tokens to the tail of the remaining chain"): with attach_tail != 0 a template node
+       whose parent is -1 hangs off the last kept node (index K_kept - 1) instead of the root, and its token is
+       looked up from that node's token.  Not together with env_token (the envelope is root-centred). */
+    int attach_tail;
 } graft_build_params;
 
 int graft_build_tree(graft_ctx* ctx, const graft_build_params* p, void* stream);

@@ -211,7 +211,7 @@ unsigned orc_build_tree(const orc_build_args *a) {
                 if (tp < -1 || tp >= u || r < 0 || r >= a->k) { ok = 0; flags |= ORC_FLAG_BAD_TEMPLATE; }
                 /* root-centred template, or (block drafters' "keep the reliable prefix and attach retrieved tokens to the
                    tail of the remaining chain") the template continues the last kept node */
-                const int attach = a->attach_tail ? K_kept - 1 : 0;
+                const int attach = a->attach_tail && K_kept > 0 ? K_kept - 1 : 0;
                 int p = (!ok || tp == -1) ? attach : K_kept + tp;
                 int ptok = o_tok[p], x = -1;
                 if (ok && ptok >= 0) {

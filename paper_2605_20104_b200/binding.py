@@ -43,7 +43,7 @@ class BuildParams(C.Structure):
                                     "k_max", "ckpt_depth", "ckpt_keep", "ckpt_log_tau", "tmpl_offset", "tmpl_parent",
                                     "tmpl_rank", "tree_token", "tree_parent", "tree_pos", "tree_src", "tree_anc",
                                     "tree_size")] +
-                [("N_env", C.c_int), ("env_token", _vp), ("tmpl_env", _vp)])
+                [("N_env", C.c_int), ("env_token", _vp), ("tmpl_env", _vp), ("attach_tail", C.c_int)])
 
 
 class EnvelopeParams(C.Structure):
@@ -189,7 +189,7 @@ def build_tree_params(*, mode: int, K_max: int, V: int, k: int, S_cap: int,
                      gate_depth: int = 0, node_threshold: float = 0.0, ckpt_depth=None, ckpt_keep=None,
                      ckpt_log_tau=None, tmpl_offset=None, tmpl_parent=None, tmpl_rank=None,
                      tree_token, tree_parent, tree_pos, tree_src, tree_anc, tree_size,
-                     env_token=None, tmpl_env=None) -> BuildParams:
+                     env_token=None, tmpl_env=None, attach_tail: bool = False) -> BuildParams:
     """env_token [B, N_env] / tmpl_env [N_tmpl]: take the grafted tokens from a precomputed retrieval envelope."""
     B, N_max = draft_token.shape
     T_max = tree_token.shape[1]
@@ -206,7 +206,7 @@ def build_tree_params(*, mode: int, K_max: int, V: int, k: int, S_cap: int,
                     tree_token=_ptr(tree_token, i32), tree_parent=_ptr(tree_parent, i32), tree_pos=_ptr(tree_pos, i32),
                     tree_src=_ptr(tree_src, i32), tree_anc=_ptr(tree_anc, torch.int64), tree_size=_ptr(tree_size, i32),
                     N_env=0 if env_token is None else env_token.shape[1],
-                    env_token=_ptr(env_token, i32), tmpl_env=_ptr(tmpl_env, i32))
+                    env_token=_ptr(env_token, i32), tmpl_env=_ptr(tmpl_env, i32), attach_tail=int(attach_tail))
     return p
 
 

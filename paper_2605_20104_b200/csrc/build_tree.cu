@@ -168,6 +168,7 @@ __global__ void __launch_bounds__(kThreads) build_tree_kernel(graft_build_params
     int T = K_kept;
     if (graft) {
         const int K_ret = max(0, min(t_hi - t_lo, budget - K_kept));
+        const int attach = a.attach_tail && K_kept > 0 ? K_kept - 1 : 0;      // where template nodes without a template parent hang
         T += K_ret;
         const int u = i;
         int tp = -1, r = 0, du = 0;
@@ -185,7 +186,7 @@ __global__ void __launch_bounds__(kThreads) build_tree_kernel(graft_build_params
                 ++du;
                 if (j >= u) { break; }       // cannot happen after the check above; bounds the loop
             }
-            s_opar[K_kept + u] = tp < 0 ? 0 : K_kept + tp;
+            s_opar[K_kept + u] = tp < 0 ? attach : K_kept + tp;
             o_src[K_kept + u] = -1 - u;
         }
         if (a.env_token) {
@@ -205,7 +206,7 @@ __global__ void __launch_bounds__(kThreads) build_tree_kernel(graft_build_params
         for (int lvl = 1; lvl <= max_d; ++lvl) {
             if (u < K_ret && du == lvl) {
                 int x = -1;
-                const int ptok = s_tok[tp < 0 ? 0 : K_kept + tp];
+                const int ptok = s_tok[tp < 0 ? attach : K_kept + tp];
                 if (ok && ptok >= 0) {
                     x = a.M[(size_t)ptok * a.k + r];
                     if (x < -1 || x >= a.V) { x = -1; flags |= GRAFT_FLAG_BAD_TOKEN; }
@@ -247,7 +248,7 @@ extern "C" int graft_build_tree(graft_ctx* ctx, const graft_build_params* p, voi
         return GRAFT_ERR_INVALID_ARG;
     if (p->N_tmpl < 0 || p->n_ckpt < 0) return GRAFT_ERR_INVALID_ARG;
     if (p->mode != GRAFT_PRUNE_NONE && p->N_tmpl > 0 && (!p->M || !p->tmpl_parent || !p->tmpl_rank)) return GRAFT_ERR_INVALID_ARG;
-    if (p->env_token && (!p->tmpl_env || p->N_env <= 0)) return GRAFT_ERR_INVALID_ARG;
+    if (p->env_token && (!p->tmpl_env || p->N_env <= 0 || p->attach_tail)) return GRAFT_ERR_INVALID_ARG;
     if (p->mode == GRAFT_PRUNE_TOPK && !p->keep_count) return GRAFT_ERR_INVALID_ARG;
     if (p->mode == GRAFT_PRUNE_GATED &&
         (p->n_ckpt > 0 && (!p->ckpt_depth || !p->ckpt_keep || !p->ckpt_log_tau || !p->tmpl_offset)))

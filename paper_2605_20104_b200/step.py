@@ -130,7 +130,7 @@ class VerifyStep:
     def _build_params(self, from_envelope: bool = False):
         w = self.w
         env = dict(env_token=self.env_token, tmpl_env=self.tmpl_env) if from_envelope else {}
-        return G.build_tree_params(**env, mode=w.mode, K_max=w.K_max, V=w.V, k=w.k, S_cap=w.S_cap,
+        return G.build_tree_params(**env, attach_tail=getattr(w, "attach_tail", False), mode=w.mode, K_max=w.K_max, V=w.V, k=w.k, S_cap=w.S_cap,
                            draft_token=self.draft_token, draft_parent=self.draft_parent, draft_score=self.draft_score,
                            n_draft=self.n_draft, seq_len=self.seq_len, M=self.M, keep_count=self.keep_count,
                            k_max=self.k_max, gate_depth=w.gate_depth, node_threshold=w.node_threshold,

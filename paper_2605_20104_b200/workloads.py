@@ -318,9 +318,11 @@ def config(cfg: str, *, B: Optional[int] = None, L: Optional[int] = None,
            seed: Optional[int] = None) -> Workload:
     """Build the named workload's integer inputs (call make_qkv for the tensors).
 
-    cfg in {"1", "2", "3", "3p", "4", "5"}.  B and L override batch and context length
+    cfg in {"1", "2", "3", "3p", "4", "5", "tail"}.  B and L override batch and context length
     (used by the tests to shrink a shape without changing its structure).
     """
+    if cfg == "tail":
+        return tail_block(B=B or 4, L=L or 65536, seed=16 if seed is None else seed)
     if cfg == "1":
         seed = 0 if seed is None else seed
         rng = np.random.default_rng(np.random.PCG64(seed))

@@ -157,3 +157,21 @@ def test_path_indices_bad_size_flag():
     G.graft_path_indices(ctx, tree_parent=parent, tree_size=torch.tensor([9], dtype=torch.int32, device="cuda"), path_index=out, n_paths=n)
     torch.cuda.synchronize()
     assert ctx.device_status() == G.FLAG_BAD_SIZE and int(n[0]) == 0 and (out == -1).all()
+
+
+@pytest.mark.parametrize("block,V", [(16, 151936), (8, 500)])
+def test_tail_grafting_block_drafter(block, V):
+    """Keep the reliable prefix of a drafted chain, continue it with the matrix's rank-0 chain (tail grafting)."""
+    w = W.tail_block(B=9, L=700, block=block, V=V)
+    ref = oracle.build_tree(w)
+    vs = VerifyStep(w, upload_qkv=False)
+    vs.build()
+    torch.cuda.synchronize()
+    got = vs.tree_host()
+    for key in TREE_KEYS:
+        assert (got[key] == ref[key]).all(), key
+    assert vs.ctx.device_status() == ref["flags"]
+    assert (ref["tree_src"] < 0).any() and (got["tree_parent"][:, 1:block] == np.arange(block - 1)).all()
+    with pytest.raises(G.GraftError):            # the envelope is root-centred: not together with tail grafting
+        vs.retrieve_envelope()
+        vs.build(from_envelope=True)
