@@ -41,6 +41,7 @@ WORKLOADS = {
     "cfg4-B4": ("4", 4, 65536),
     "cfg5": ("5", None, None),
     "tail16-B4": ("tail", 4, 65536),      # block drafter with tail grafting: chains of 16 on the 64K Qwen3-14B shape
+    "tail16-B1-32k": ("tail", 1, 32768),  # the same at a size an ncu capture may hold
 }
 DEFAULT_WORKLOAD = "cfg4-B4"          # the 64K-context point the metric's target is stated on
 EXTRA_WORKLOADS = ["cfg2", "cfg3", "cfg4-B1-32k", "cfg4-B1", "cfg5", "tail16-B4"]
