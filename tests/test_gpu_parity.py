@@ -415,3 +415,30 @@ def test_chain_only_trees(orc, G, Step, variant, B, L0):
     w = W.custom(parents, Hq=40, Hkv=8, d=128, L=L, T_max=16, seed=40 + B)
     rows = sample_rows(np.random.default_rng(B), orc.build_tree(w)["tree_size"], w.Hq, 300)
     full_case(orc, G, Step, w, variant, rows=rows)
+
+
+@pytest.mark.parametrize("Hq,Hkv,T", [(32, 8, 32), (40, 8, 48)])
+def test_kernels_take_turns_on_one_workspace(orc, G, Step, Hq, Hkv, T):
+    """All attention kernels share one workspace (slot descriptors, arrival counters, the call number): a dozen calls
+    in a row, the kernel and the lengths changing from call to call, every one exact.  The first shape gives one
+    128-row block per item (every CTA its own tiles in the row-block kernel), the second two."""
+    rng = np.random.default_rng(Hq)
+    B = 6
+    parents = [W.random_tree_parents(rng, int(rng.integers(T // 2, T + 1))) for _ in range(B)]
+    L0 = [2500, 1800, 900, 2200, 600, 1500]
+    w = W.custom(parents, Hq=Hq, Hkv=Hkv, d=128, L=L0, T_max=T, seed=Hq)
+    tree = orc.build_tree(w)
+    W.make_qkv(w, tree["tree_size"], poison=True)
+    vs = Step(w)
+    vs.build()
+    order = ["l2pair", "pair", "one", "auto", "mma", "pair", "l2pair", "l2pair", "one", "pair", "auto", "l2pair"]
+    for n, variant in enumerate(order):
+        # lengths only ever shrink: the cache is poisoned past the first call's ends
+        w.seq_len = np.maximum(1, np.asarray(L0) - rng.integers(0, 500, size=B) * (n > 0)).astype(np.int32)
+        vs.seq_len.copy_(torch.from_numpy(w.seq_len))
+        vs.O.fill_(float("nan"))
+        vs.attn(variant_id(G, variant, w))
+        torch.cuda.synchronize()
+        rows = sample_rows(np.random.default_rng(n), tree["tree_size"], w.Hq, 200)
+        check_attn(orc, w, vs, tree, rows)
+    assert vs.ctx.device_status() == 0
