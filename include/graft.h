@@ -245,6 +245,13 @@ typedef struct {
     const int32_t* seq_len;                          /* [B] */
     const int32_t* tree_size;                        /* [B] */
     const uint64_t* tree_anc;                        /* [B, T_max] */
+    /* paged caches (optional; serving-shaped variant).  With block_table set, Kc / Vc are pools
+       [n_blocks, Hkv, page_size, d] (kv_stride_b = elements between blocks) and cache slot s of sequence b
+       lives in block block_table[b * blocks_per_seq + s / page_size] at row s % page_size.  page_size is a
+       multiple of 128; S_cap <= blocks_per_seq * page_size.  A table entry outside [0, n_blocks) reads as
+       zeros and sets GRAFT_FLAG_BAD_SIZE.  Slots past L_b + T_b may hold anything, as in the contiguous layout. */
+    const int32_t* block_table;                      /* [B, blocks_per_seq] or NULL */
+    int page_size, blocks_per_seq, n_blocks;
 } graft_attn_params;
 
 int graft_tree_verify_attn(graft_ctx* ctx, const graft_attn_params* p, void* stream);
@@ -377,6 +384,9 @@ typedef struct {
     const int32_t* n_acc;        /* [B] */
     const int32_t* path;         /* [B, T_max] */
     int32_t* new_seq_len;        /* out [B] */
+    /* paged caches, as in graft_attn_params (one table for all layers; layer_stride between the layers' pools) */
+    const int32_t* block_table;  /* [B, blocks_per_seq] or NULL */
+    int page_size, blocks_per_seq, n_blocks;
 } graft_compact_params;
 
 int graft_compact_kv(graft_ctx* ctx, const graft_compact_params* p, void* stream);

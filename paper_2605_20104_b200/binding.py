@@ -70,7 +70,8 @@ class AttnParams(C.Structure):
                  ("Kc", _vp), ("Vc", _vp),
                  ("kv_stride_b", C.c_int64), ("kv_stride_h", C.c_int64), ("kv_stride_s", C.c_int64),
                  ("O", _vp), ("o_stride_b", C.c_int64), ("o_stride_t", C.c_int64), ("o_stride_h", C.c_int64),
-                 ("LSE", _vp), ("seq_len", _vp), ("tree_size", _vp), ("tree_anc", _vp)])
+                 ("LSE", _vp), ("seq_len", _vp), ("tree_size", _vp), ("tree_anc", _vp),
+                 ("block_table", _vp), ("page_size", C.c_int), ("blocks_per_seq", C.c_int), ("n_blocks", C.c_int)])
 
 
 class AcceptParams(C.Structure):
@@ -87,7 +88,8 @@ class UpdateParams(C.Structure):
 class CompactParams(C.Structure):
     _fields_ = ([(n, C.c_int) for n in ("B", "Hkv", "d", "S_cap", "T_max", "n_layers")] +
                 [(n, C.c_int64) for n in ("layer_stride", "kv_stride_b", "kv_stride_h", "kv_stride_s")] +
-                [(n, _vp) for n in ("Kc", "Vc", "seq_len", "n_acc", "path", "new_seq_len")])
+                [(n, _vp) for n in ("Kc", "Vc", "seq_len", "n_acc", "path", "new_seq_len", "block_table")] +
+                [(n, C.c_int) for n in ("page_size", "blocks_per_seq", "n_blocks")])
 
 
 _lib.graft_workspace_bytes.restype = C.c_size_t
@@ -215,12 +217,22 @@ def graft_build_tree(ctx: Context, **kw) -> None:
 
 
 def tree_verify_attn_params(*, Q, Kc, Vc, O, seq_len, tree_size, tree_anc, scale: float,
-                            LSE=None, variant: int = ATTN_AUTO) -> AttnParams:
+                            LSE=None, variant: int = ATTN_AUTO, block_table=None, S_cap: Optional[int] = None) -> AttnParams:
     """Q, O: bf16 [B, T_max, Hq, d]; Kc, Vc: bf16 [B, Hkv, S_cap, d] (any strides with a contiguous
-    last axis); tree_anc: int64 [B, T_max] holding the 64-bit masks."""
+    last axis); tree_anc: int64 [B, T_max] holding the 64-bit masks.
+    Paged caches: block_table int32 [B, blocks_per_seq] and Kc, Vc pools [n_blocks, Hkv, page_size, d];
+    S_cap (logical slots per sequence) then defaults to blocks_per_seq * page_size."""
     bf = torch.bfloat16
     B, T_max, Hq, d = Q.shape
-    _, Hkv, S_cap, _ = Kc.shape
+    paged = {}
+    if block_table is None:
+        _, Hkv, S_cap, _ = Kc.shape
+    else:
+        n_blocks, Hkv, page_size, _ = Kc.shape
+        assert block_table.shape[0] == B and block_table.is_contiguous()
+        S_cap = block_table.shape[1] * page_size if S_cap is None else S_cap
+        paged = dict(block_table=_ptr(block_table, torch.int32), page_size=page_size, blocks_per_seq=block_table.shape[1],
+                     n_blocks=n_blocks)
     assert Q.stride(3) == 1 and Kc.stride(3) == 1 and Vc.stride(3) == 1 and O.stride(3) == 1
     assert Kc.stride() == Vc.stride() and Kc.shape == Vc.shape and O.shape == Q.shape
     p = AttnParams(B=B, T_max=T_max, Hq=Hq, Hkv=Hkv, d=d, S_cap=S_cap, scale=scale, variant=variant,
@@ -229,7 +241,7 @@ def tree_verify_attn_params(*, Q, Kc, Vc, O, seq_len, tree_size, tree_anc, scale
                    kv_stride_s=Kc.stride(2),
                    O=_ptr(O, bf), o_stride_b=O.stride(0), o_stride_t=O.stride(1), o_stride_h=O.stride(2),
                    LSE=_ptr(LSE, torch.float32), seq_len=_ptr(seq_len, torch.int32),
-                   tree_size=_ptr(tree_size, torch.int32), tree_anc=_ptr(tree_anc, torch.int64))
+                   tree_size=_ptr(tree_size, torch.int32), tree_anc=_ptr(tree_anc, torch.int64), **paged)
     return p
 
 
@@ -336,19 +348,27 @@ def graft_accept(ctx: Context, **kw) -> None:
     launch("graft_accept", ctx, accept_params(**kw))
 
 
-def compact_kv_params(*, Kc, Vc, seq_len, n_acc, path, new_seq_len) -> CompactParams:
-    """Kc, Vc: bf16 [B, Hkv, S_cap, d] or [n_layers, B, Hkv, S_cap, d], compacted in place."""
+def compact_kv_params(*, Kc, Vc, seq_len, n_acc, path, new_seq_len, block_table=None, S_cap: Optional[int] = None) -> CompactParams:
+    """Kc, Vc: bf16 [B, Hkv, S_cap, d] or [n_layers, B, Hkv, S_cap, d], compacted in place.
+    Paged caches: block_table int32 [B, blocks_per_seq] and pools [n_blocks, Hkv, page_size, d] (or with a leading
+    layer axis)."""
     bf, i32 = torch.bfloat16, torch.int32
     if Kc.dim() == 4:
         n_layers, layer_stride, off = 1, 0, 0
     else:
         n_layers, layer_stride, off = Kc.shape[0], Kc.stride(0), 1
-    B, Hkv, S_cap, d = Kc.shape[off:]
+    B, Hkv, S_cap_, d = Kc.shape[off:]
+    paged = {}
+    if block_table is not None:
+        n_blocks, page_size, B = B, S_cap_, block_table.shape[0]
+        S_cap_ = block_table.shape[1] * page_size if S_cap is None else S_cap
+        paged = dict(block_table=_ptr(block_table, i32), page_size=page_size, blocks_per_seq=block_table.shape[1], n_blocks=n_blocks)
+    S_cap = S_cap_
     assert Kc.stride() == Vc.stride() and Kc.stride(-1) == 1
     p = CompactParams(B=B, Hkv=Hkv, d=d, S_cap=S_cap, T_max=path.shape[1], n_layers=n_layers, layer_stride=layer_stride,
                       kv_stride_b=Kc.stride(off), kv_stride_h=Kc.stride(off + 1), kv_stride_s=Kc.stride(off + 2),
                       Kc=_ptr(Kc, bf), Vc=_ptr(Vc, bf), seq_len=_ptr(seq_len, i32), n_acc=_ptr(n_acc, i32),
-                      path=_ptr(path, i32), new_seq_len=_ptr(new_seq_len, i32))
+                      path=_ptr(path, i32), new_seq_len=_ptr(new_seq_len, i32), **paged)
     return p
 
 

@@ -79,6 +79,10 @@ extern "C" int graft_tree_verify_attn(graft_ctx* ctx, const graft_attn_params* p
     for (int64_t s : strides)
         if (s < 0 || s % 8 != 0) return GRAFT_ERR_INVALID_ARG;
     if (p->kv_stride_s < p->d || p->q_stride_h < p->d || p->o_stride_h < p->d) return GRAFT_ERR_INVALID_ARG;
+    if (p->block_table) {
+        if (p->page_size <= 0 || p->page_size % 128 != 0 || p->blocks_per_seq <= 0 || p->n_blocks <= 0) return GRAFT_ERR_INVALID_ARG;
+        if ((long long)p->blocks_per_seq * p->page_size < p->S_cap) return GRAFT_ERR_INVALID_ARG;
+    }
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     switch (p->variant) {
         case GRAFT_ATTN_MMA_SYNC: return graft_attn_mma_launch(ctx, p, s);

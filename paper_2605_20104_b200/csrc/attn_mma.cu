@@ -55,22 +55,41 @@ __device__ __forceinline__ uint32_t swz(int row, int chunk) {
 
 using MmaArgs = graft_merge::AttnArgs;
 
-template <int D>
-__device__ __forceinline__ void load_kv_tile(uint32_t sK, uint32_t sV, const __nv_bfloat16* Kg, const __nv_bfloat16* Vg,
-                                             int64_t stride_s, int key0, int n_keys) {
-    constexpr int CH = D / 8;
-    for (int c = threadIdx.x; c < BN * CH; c += NTHREADS) {
-        const int row = c / CH, ch = c % CH;
-        const int key = key0 + row;
-        const bool ok = key < n_keys;
-        const size_t off = (size_t)(ok ? key : 0) * stride_s + ch * 8;
-        cp_async16(sK + swz<D>(row, ch), Kg + off, ok);
-        cp_async16(sV + swz<D>(row, ch), Vg + off, ok);
-    }
+// where a sequence's cache slots live: one contiguous run, or pages of a pool looked up in the sequence's block table
+struct KvPlace {
+    const int32_t* table;      // the sequence's row of the block table, or nullptr
+    int page_size, n_blocks;
+    int64_t stride_b, stride_s;
+};
+// element offset of cache slot `key` (from the KV head's base); false if its table entry is out of range
+__device__ __forceinline__ bool kv_offset(const KvPlace& pl, int key, size_t& off) {
+    if (!pl.table) { off = (size_t)key * pl.stride_s; return true; }
+    const int blk = pl.table[key / pl.page_size];
+    if (blk < 0 || blk >= pl.n_blocks) return false;
+    off = (size_t)blk * pl.stride_b + (size_t)(key % pl.page_size) * pl.stride_s;
+    return true;
 }
 
 template <int D>
-__global__ void __launch_bounds__(NTHREADS, 2) attn_mma_kernel(MmaArgs a) {
+__device__ __forceinline__ bool load_kv_tile(uint32_t sK, uint32_t sV, const __nv_bfloat16* Kg, const __nv_bfloat16* Vg,
+                                             const KvPlace& pl, int key0, int n_keys) {
+    constexpr int CH = D / 8;
+    bool all_ok = true;
+    for (int c = threadIdx.x; c < BN * CH; c += NTHREADS) {
+        const int row = c / CH, ch = c % CH;
+        const int key = key0 + row;
+        bool ok = key < n_keys;
+        size_t off = 0;
+        if (ok && !kv_offset(pl, key, off)) { ok = false; all_ok = false; }
+        off = ok ? off + ch * 8 : 0;
+        cp_async16(sK + swz<D>(row, ch), Kg + off, ok);
+        cp_async16(sV + swz<D>(row, ch), Vg + off, ok);
+    }
+    return all_ok;
+}
+
+template <int D>
+__global__ void __launch_bounds__(NTHREADS, 2) attn_mma_kernel(MmaArgs a, unsigned* status) {
     extern __shared__ __align__(128) unsigned char smem[];
     const graft_attn_params& p = a.p;
     constexpr int TILE_BYTES = BN * D * 2;
@@ -94,8 +113,12 @@ __global__ void __launch_bounds__(NTHREADS, 2) attn_mma_kernel(MmaArgs a) {
     const int n_keys = w.L + w.T;
     const __nv_bfloat16* Qg = reinterpret_cast<const __nv_bfloat16*>(p.Q) + (size_t)w.b * p.q_stride_b +
                               (size_t)w.h * G * p.q_stride_h;
-    const __nv_bfloat16* Kg = reinterpret_cast<const __nv_bfloat16*>(p.Kc) + (size_t)w.b * p.kv_stride_b + (size_t)w.h * p.kv_stride_h;
-    const __nv_bfloat16* Vg = reinterpret_cast<const __nv_bfloat16*>(p.Vc) + (size_t)w.b * p.kv_stride_b + (size_t)w.h * p.kv_stride_h;
+    const size_t seq_off = p.block_table ? 0 : (size_t)w.b * p.kv_stride_b;          // pages are found through the table
+    const __nv_bfloat16* Kg = reinterpret_cast<const __nv_bfloat16*>(p.Kc) + seq_off + (size_t)w.h * p.kv_stride_h;
+    const __nv_bfloat16* Vg = reinterpret_cast<const __nv_bfloat16*>(p.Vc) + seq_off + (size_t)w.h * p.kv_stride_h;
+    const KvPlace place = {p.block_table ? p.block_table + (size_t)w.b * p.blocks_per_seq : nullptr, p.page_size, p.n_blocks,
+                           p.kv_stride_b, p.kv_stride_s};
+    bool table_ok = true;
 
     // ---- prologue: Q rows and the first two K/V tiles
     {
@@ -108,10 +131,10 @@ __global__ void __launch_bounds__(NTHREADS, 2) attn_mma_kernel(MmaArgs a) {
             cp_async16(sQ + swz<D>(row, ch), Qg + (size_t)t * p.q_stride_t + (size_t)g * p.q_stride_h + ch * 8, ok);
         }
     }
-    load_kv_tile<D>(sKV, sKV + TILE_BYTES, Kg, Vg, p.kv_stride_s, w.tile_lo * BN, n_keys);
+    table_ok &= load_kv_tile<D>(sKV, sKV + TILE_BYTES, Kg, Vg, place, w.tile_lo * BN, n_keys);
     cp_async_commit();
     if (w.tile_lo + 1 < w.tile_hi)
-        load_kv_tile<D>(sKV + 2 * TILE_BYTES, sKV + 3 * TILE_BYTES, Kg, Vg, p.kv_stride_s, (w.tile_lo + 1) * BN, n_keys);
+        table_ok &= load_kv_tile<D>(sKV + 2 * TILE_BYTES, sKV + 3 * TILE_BYTES, Kg, Vg, place, (w.tile_lo + 1) * BN, n_keys);
     cp_async_commit();
 
     // ---- per-thread rows: lane/4 and lane/4 + 8 of the warp's 16
@@ -219,10 +242,11 @@ __global__ void __launch_bounds__(NTHREADS, 2) attn_mma_kernel(MmaArgs a) {
             }
         }
         __syncthreads();
-        if (tile + 2 < w.tile_hi) load_kv_tile<D>(sK, sV, Kg, Vg, p.kv_stride_s, (tile + 2) * BN, n_keys);
+        if (tile + 2 < w.tile_hi) table_ok &= load_kv_tile<D>(sK, sV, Kg, Vg, place, (tile + 2) * BN, n_keys);
         cp_async_commit();
     }
     cp_async_wait<0>();
+    if (!table_ok) atomicOr(status, (unsigned)GRAFT_FLAG_BAD_SIZE);          // a block-table entry outside the pool: its keys read as zeros
 
     // ---- epilogue: quad-reduce the row sums, then either the final result or a partial
     lA += __shfl_xor_sync(0xffffffffu, lA, 1);
@@ -291,7 +315,7 @@ static int launch(graft_ctx* ctx, const graft_attn_params* p, cudaStream_t strea
     a.dbg = 0;
     const int grid = max_slots(ctx->num_sms, p->B, p->Hq, p->Hkv, p->T_max);
     const size_t smem = (size_t)BR * D * 2 + 4 * (size_t)BN * D * 2;
-    attn_mma_kernel<D><<<grid, NTHREADS, smem, stream>>>(a);
+    attn_mma_kernel<D><<<grid, NTHREADS, smem, stream>>>(a, ctx->status);
     GRAFT_CHECK_CUDA(cudaGetLastError());
     return graft_merge::launch<D, BR, BN>(a, ctx->status, stream);
 }

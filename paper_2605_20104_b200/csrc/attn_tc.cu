@@ -2080,6 +2080,7 @@ bool graft_attn_tc_pair_supported(const graft_ctx* ctx, const graft_attn_params*
 
 bool graft_attn_tc_supported(const graft_ctx* ctx, const graft_attn_params* p) {
     if (p->d != D) return false;
+    if (p->block_table) return false;                                    // paged caches go through the register-tile kernel
     if ((long long)p->B * p->Hkv * 8 >= (1ll << 24)) return false;      // item ids share a word with the call stamp
     // TMA: 16-byte aligned base and strides (checked by the caller), strides below 2^40 bytes
     if (p->kv_stride_s * 2 >= (1ll << 40) || p->kv_stride_h * 2 >= (1ll << 40) || p->kv_stride_b * 2 >= (1ll << 40)) return false;

@@ -40,18 +40,34 @@ __global__ void __launch_bounds__(kThreads) compact_kernel(graft_compact_params 
     if (first) a.new_seq_len[b] = L + n;
 
     uint16_t* base = reinterpret_cast<uint16_t*>(which ? a.Vc : a.Kc) + (size_t)layer * a.layer_stride +
-                     (size_t)b * a.kv_stride_b + (size_t)h * a.kv_stride_h;
+                     (a.block_table ? 0 : (size_t)b * a.kv_stride_b) + (size_t)h * a.kv_stride_h;
+    // element offset of cache slot s of this sequence: contiguous, or through the block table (-1: entry out of range)
+    const int32_t* table = a.block_table ? a.block_table + (size_t)b * a.blocks_per_seq : nullptr;
+    auto slot = [&](int s) -> long long {
+        if (!table) return (long long)s * a.kv_stride_s;
+        const int blk = table[s / a.page_size];
+        if (blk < 0 || blk >= a.n_blocks) return -1;
+        return (long long)blk * a.kv_stride_b + (long long)(s % a.page_size) * a.kv_stride_s;
+    };
+    bool table_ok = true;
     for (int c = threadIdx.x; c < n * chunks; c += kThreads) {
         const int j = c / chunks, part = c % chunks;
-        if (s_path[j] != j)
-            stage[c] = *reinterpret_cast<const uint4*>(base + (size_t)(L + s_path[j]) * a.kv_stride_s + part * 8);
+        if (s_path[j] != j) {
+            const long long src = slot(L + s_path[j]);
+            if (src < 0) { table_ok = false; stage[c] = make_uint4(0u, 0u, 0u, 0u); }
+            else stage[c] = *reinterpret_cast<const uint4*>(base + src + part * 8);
+        }
     }
     __syncthreads();
     for (int c = threadIdx.x; c < n * chunks; c += kThreads) {
         const int j = c / chunks, part = c % chunks;
-        if (s_path[j] != j)
-            *reinterpret_cast<uint4*>(base + (size_t)(L + j) * a.kv_stride_s + part * 8) = stage[c];
+        if (s_path[j] != j) {
+            const long long dst = slot(L + j);
+            if (dst < 0) table_ok = false;
+            else *reinterpret_cast<uint4*>(base + dst + part * 8) = stage[c];
+        }
     }
+    if (!table_ok) atomicOr(status, (unsigned)GRAFT_FLAG_BAD_SIZE);
 }
 
 }  // namespace
@@ -65,6 +81,10 @@ extern "C" int graft_compact_kv(graft_ctx* ctx, const graft_compact_params* p, v
     if (!graft_aligned16(p->Kc) || !graft_aligned16(p->Vc) || p->layer_stride % 8 || p->kv_stride_b % 8 ||
         p->kv_stride_h % 8 || p->kv_stride_s % 8 || p->kv_stride_s < p->d)
         return GRAFT_ERR_INVALID_ARG;
+    if (p->block_table) {
+        if (p->page_size <= 0 || p->page_size % 128 != 0 || p->blocks_per_seq <= 0 || p->n_blocks <= 0) return GRAFT_ERR_INVALID_ARG;
+        if ((long long)p->blocks_per_seq * p->page_size < p->S_cap) return GRAFT_ERR_INVALID_ARG;
+    }
     const long long ctas = 2ll * p->B * p->Hkv * p->n_layers;
     if (ctas > 0x7fffffffll) return GRAFT_ERR_UNSUPPORTED;
     const size_t smem = (size_t)p->T_max * (p->d / 8) * sizeof(uint4);     // <= 32 KB
