@@ -171,6 +171,40 @@ def time_workload(name, steps, warmup, device, variant, rank=0):
                 flags=flags, tree=tree)
 
 
+def time_paged_attention(st, steps, warmup, variant, page_size=256):
+    """The attention call on the same K/V scattered over a paged pool (random block table), alone."""
+    from paper_2605_20104_b200 import binding as G
+    w, vs = st["w"], st["vs"]
+    Kc, Vc = st["caches"][0]
+    B, Hkv, S_cap, d = Kc.shape
+    per_seq = (S_cap + page_size - 1) // page_size
+    n_blocks = B * per_seq + 7
+    g = torch.Generator(device="cpu")
+    g.manual_seed(11)
+    table = torch.randperm(n_blocks, generator=g)[:B * per_seq].reshape(B, per_seq).to(torch.int32).to(vs.dev)
+    Kp = torch.zeros(n_blocks, Hkv, page_size, d, dtype=torch.bfloat16, device=vs.dev)
+    Vp = torch.zeros_like(Kp)
+    pad = per_seq * page_size - S_cap
+    for src, dst in ((Kc, Kp), (Vc, Vp)):
+        x = torch.nn.functional.pad(src, (0, 0, 0, pad)).reshape(B, Hkv, per_seq, page_size, d).permute(0, 2, 1, 3, 4)
+        dst[table.long().reshape(-1)] = x.reshape(B * per_seq, Hkv, page_size, d)
+    prm = G.tree_verify_attn_params(Q=vs.Q, Kc=Kp, Vc=Vp, O=vs.O, seq_len=vs.seq_len, tree_size=vs.tree_size, tree_anc=vs.tree_anc,
+                                    scale=w.scale, LSE=vs.LSE, variant=variant, block_table=table, S_cap=S_cap)
+    ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(steps)]
+    for _ in range(warmup):
+        G.launch("graft_tree_verify_attn", vs.ctx, prm)
+    torch.cuda.synchronize()
+    torch.cuda._sleep(int(3e6))
+    for a, b in ev:
+        a.record()
+        G.launch("graft_tree_verify_attn", vs.ctx, prm)
+        b.record()
+    torch.cuda.synchronize()
+    us = float(np.mean([a.elapsed_time(b) for a, b in ev])) * 1e3
+    del Kp, Vp
+    return {"us_per_call": us, "page_size": page_size, "device_flags": vs.ctx.device_status()}
+
+
 def time_graph_replay(st, steps, warmup, variant):
     """The same step captured once per rotating cache in a CUDA graph and replayed: device time per step without
     the launch gaps of four separate calls (the launch configuration is fixed by the shapes, so a serving loop
@@ -525,6 +559,8 @@ def main():
         line["update_adjacency"] = upd
         line["index_kernels"] = time_index_kernels(st, min(args.steps, 50), 5)
         line["graph_replay_us_per_step"] = time_graph_replay(st, min(args.steps, 100), 5, variant)
+        if st["n_rot"] == 1:
+            line["paged_attention"] = time_paged_attention(st, min(args.steps, 50), 5, variant)
         acs = time_accept_stochastic(st, min(args.steps, 50), 5)
         acs["frac_of_measured"] = acs["GBps"] / peak
         line["accept_stochastic"] = acs

@@ -90,7 +90,7 @@ extern "C" int graft_tree_verify_attn(graft_ctx* ctx, const graft_attn_params* p
             if (!graft_attn_tc_supported(ctx, p)) return GRAFT_ERR_UNSUPPORTED;
             return graft_attn_tc_launch(ctx, p, s);
         case GRAFT_ATTN_TCGEN05_1SM:
-            if (!graft_attn_tc_supported(ctx, p)) return GRAFT_ERR_UNSUPPORTED;
+            if (!graft_attn_tc_supported(ctx, p) || p->block_table) return GRAFT_ERR_UNSUPPORTED;     // this kernel takes contiguous caches only
             return graft_attn_tc_launch(ctx, p, s, 0);
         case GRAFT_ATTN_TCGEN05_2SM:
             if (!graft_attn_tc_pair_supported(ctx, p)) return GRAFT_ERR_UNSUPPORTED;

@@ -1155,14 +1155,27 @@ struct SoftmaxBars {
     int S, P, O;             // barrier indices: score buffer ready (x3), P written (x3), all MMAs of the segment complete
     int pv_done, pv_mod;     // barrier whose phase tile/pv_mod of index pv_done + tile % pv_mod completes with P V of `tile`
     bool remote;             // P barriers live in CTA 0 of the cluster
+    // where this CTA's part of a V tile sits in shared memory (paged caches: rows past a sequence's keys are zeroed there)
+    uint32_t v_base;         // slot 0
+    int v_slot_bytes, v_nslot, v_boxes, v_box_stride;
+    int v_full;              // barrier that tells a V slot has landed, or -1 when the score barrier implies it
 };
 // first key and number of already-covered columns of tile t of an item: the last tile is fetched at keys
 // [L+T-128, L+T), so it never reaches past the sequence's keys (rows before key 0 are zero-filled by the copy)
-__device__ __forceinline__ int tile_key0(const Seg& sg, int t, int& overlap) {
+// pool block of the page that holds cache slot `key` of sequence b (paged caches); an entry outside the pool gives
+// n_blocks, a coordinate past the tensor map's end that the copy fills with zeros, and raises the flag
+__device__ __forceinline__ int page_block(const graft_attn_params& p, int b, int key, unsigned* status) {
+    const int blk = __ldg(p.block_table + (size_t)b * p.blocks_per_seq + key / p.page_size);
+    if (blk < 0 || blk >= p.n_blocks) { atomicOr(status, (unsigned)GRAFT_FLAG_BAD_SIZE); return p.n_blocks; }
+    return blk;
+}
+// With paged caches a tile must not straddle two pages, so the last tile stays aligned; what it holds past the
+// sequence's keys is masked in the scores and zeroed in the V tile before P V reads it.
+__device__ __forceinline__ int tile_key0(const Seg& sg, int t, int& overlap, bool paged) {
     const int n_keys = sg.L + sg.T;
     const int ntiles = (n_keys + BN - 1) / BN;
     overlap = 0;
-    if (t < ntiles - 1) return t * BN;
+    if (paged || t < ntiles - 1) return t * BN;
     overlap = ntiles * BN - n_keys;
     return n_keys - BN;
 }
@@ -1209,10 +1222,23 @@ __device__ __forceinline__ void softmax_rows_split(const TcArgs& a, const Plan& 
             const uint32_t tS = tmem + lane_bits + (gt % P_NSBUF) * 128 + half * 64;      // this thread's 64 score columns
             const uint32_t tP = tmem + lane_bits + (gt % P_NSBUF) * 128 + half * 32;      // its 64 P values (bf16 pairs)
             int overlap;
-            const int key0 = tile_key0(sg, sg.tile_lo + j, overlap);
+            const bool paged = p.block_table != nullptr;
+            const int key0 = tile_key0(sg, sg.tile_lo + j, overlap, paged);
             const bool masked = key0 + BN > sg.L || overlap > 0;
+            const int n_valid = sg.L + sg.T - key0;         // keys of this tile that exist (paged caches: may be < 128 in the last tile)
             mbar_wait(bar(lay.S + gt % P_NSBUF), (gt / P_NSBUF) & 1, abort_flag, status);
             tc_fence_after();
+            const bool sanitize = paged && n_valid < BN;
+            if (sanitize) {
+                // the rows of the V tile past the sequence's keys may hold anything (0 x NaN would poison O): zero them
+                if (lay.v_full >= 0) mbar_wait(bar(lay.v_full + gt % lay.v_nslot), (gt / lay.v_nslot) & 1, abort_flag, status);
+                const uint32_t vs = lay.v_base + (gt % lay.v_nslot) * lay.v_slot_bytes + (uint32_t)n_valid * 128u;
+                const int nchunk = (BN - n_valid) * 8;       // 16-byte pieces per 64-column box
+                for (int bx = 0; bx < lay.v_boxes; ++bx)
+                    for (int c = (int)threadIdx.x - 128; c < nchunk; c += 256)
+                        asm volatile("st.shared.v4.b32 [%0], {%1, %1, %1, %1};" ::"r"(vs + bx * lay.v_box_stride + c * 16), "r"(0u) : "memory");
+                fence_async_smem();
+            }
             uint32_t x[2][32];
 #pragma unroll
             for (int c = 0; c < 2; ++c) tmem_ld32(tS + c * 32, x[c]);
@@ -1289,7 +1315,9 @@ __device__ __forceinline__ void softmax_rows_split(const TcArgs& a, const Plan& 
             tc_fence_before();
             __syncwarp();
             if (lane == 0) {                               // one arrival per warp
-                if (lay.remote) mbar_arrive_remote(map_to_cta(bar(lay.P + gt % P_NSBUF), 0u));
+                if (lay.remote && sanitize)                // the zeroed rows must be visible to the MMA the leader issues: release at cluster scope
+                    asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(map_to_cta(bar(lay.P + gt % P_NSBUF), 0u)) : "memory");
+                else if (lay.remote) mbar_arrive_remote(map_to_cta(bar(lay.P + gt % P_NSBUF), 0u));
                 else mbar_arrive(bar(lay.P + gt % P_NSBUF));
             }
         }
@@ -1486,16 +1514,19 @@ attn_tc_pair_kernel(const __grid_constant__ CUtensorMap kmap, const __grid_const
                     const Seg sg = plan.seg[si];
                     for (int t = sg.tile_lo; t < sg.tile_hi; ++t, ++jt) {
                         int overlap;
-                        const int key0 = tile_key0(sg, t, overlap);
+                        const bool paged = p.block_table != nullptr;
+                        const int key0 = tile_key0(sg, t, overlap, paged);
+                        // paged caches: the copy addresses (row of the page, block of the pool) instead of (slot, sequence)
+                        const int krow = paged ? key0 % p.page_size : key0, kblk = paged ? page_block(p, sg.b, key0, status) : sg.b;
                         const int slot = jt % P_NSLOT, use = jt / P_NSLOT;
                         if (use > 0) mbar_wait(bar(PB_EMPTY + slot), (use - 1) & 1, abort_flag, status);
                         if (rank == 0) mbar_expect_tx(bar(PB_FULL + slot), 2 * P_SLOT_BYTES);      // K and V halves of both CTAs
                         const uint32_t dst = sRing + slot * P_SLOT_BYTES;
                         const uint32_t fb = leader_bar(PB_FULL + slot);
                         // 64 keys of the K tile, all of d (two 64-column boxes); all keys of the V tile, 64 columns of d
-                        tma_pair_4d_hint(dst, &kmap, 0, key0 + 64 * (int)rank, sg.h, sg.b, fb, stream_once);
-                        tma_pair_4d_hint(dst + P_HALF_TILE / 2, &kmap, 64, key0 + 64 * (int)rank, sg.h, sg.b, fb, stream_once);
-                        tma_pair_4d_hint(dst + P_HALF_TILE, &vmap, 64 * (int)rank, key0, sg.h, sg.b, fb, stream_once);
+                        tma_pair_4d_hint(dst, &kmap, 0, krow + 64 * (int)rank, sg.h, kblk, fb, stream_once);
+                        tma_pair_4d_hint(dst + P_HALF_TILE / 2, &kmap, 64, krow + 64 * (int)rank, sg.h, kblk, fb, stream_once);
+                        tma_pair_4d_hint(dst + P_HALF_TILE, &vmap, 64 * (int)rank, krow, sg.h, kblk, fb, stream_once);
                     }
                 }
             }
@@ -1591,7 +1622,8 @@ attn_tc_pair_kernel(const __grid_constant__ CUtensorMap kmap, const __grid_const
             }
         } else if (warp >= 4) {
             // =============================== softmax, results (both CTAs) ===============================
-            const SoftmaxBars lay = {PB_S, PB_P, PB_O, PB_EMPTY, P_NSLOT, true};
+            // this CTA's half of a V tile: all 128 keys, 64 of the d columns, behind the K half of the slot
+            const SoftmaxBars lay = {PB_S, PB_P, PB_O, PB_EMPTY, P_NSLOT, true, sRing + P_HALF_TILE, P_SLOT_BYTES, P_NSLOT, 1, 0, -1};
             softmax_rows_split(a, plan, lay, bar0, tmem, (int)rank, split, &ctrl.merge_flag, jt, n_seg_done, abort_flag, status);
         }
 
@@ -1721,7 +1753,9 @@ attn_tc_rb_kernel(const __grid_constant__ CUtensorMap kmap, const __grid_constan
                     Seg sg;
                     int t = 0, overlap;
                     locate(idx, sg, t);
-                    const int key0 = tile_key0(sg, t, overlap);
+                    const bool paged = p.block_table != nullptr;
+                    const int key0 = tile_key0(sg, t, overlap, paged);
+                    const int krow = paged ? key0 % p.page_size : key0, kblk = paged ? page_block(p, sg.b, key0, status) : sg.b;
                     const int g = jt + idx;              // global tile number
                     const int nslot = is_v ? R_NV : R_NK;
                     const int slot = g % nslot, use = g / nslot;
@@ -1730,8 +1764,8 @@ attn_tc_rb_kernel(const __grid_constant__ CUtensorMap kmap, const __grid_constan
                     mbar_expect_tx(bar(full), TILE_BYTES);
                     const uint32_t dst = (is_v ? sV : sK) + slot * TILE_BYTES;
                     const CUtensorMap* map = is_v ? &vmap : &kmap;
-                    tma_load_4d(dst, map, 0, key0, sg.h, sg.b, bar(full));
-                    tma_load_4d(dst + HALF_BYTES, map, 64, key0, sg.h, sg.b, bar(full));
+                    tma_load_4d(dst, map, 0, krow, sg.h, kblk, bar(full));
+                    tma_load_4d(dst + HALF_BYTES, map, 64, krow, sg.h, kblk, bar(full));
                 };
                 for (int i = 0; i <= total; ++i) {
                     if (i < total) load(i, false);
@@ -1835,7 +1869,7 @@ attn_tc_rb_kernel(const __grid_constant__ CUtensorMap kmap, const __grid_constan
             }
         } else if (warp >= 4) {
             // =============================== softmax, results ===============================
-            const SoftmaxBars lay = {RB_S, RB_P, RB_O, RB_EMPTYV, R_NV, false};
+            const SoftmaxBars lay = {RB_S, RB_P, RB_O, RB_EMPTYV, R_NV, false, sV, TILE_BYTES, R_NV, 2, HALF_BYTES, RB_FULLV};
             softmax_rows_split(a, plan, lay, bar0, tmem, rank, split, &ctrl.merge_flag, jt, n_seg_done, abort_flag, status);
         }
 
@@ -1995,7 +2029,9 @@ constexpr int kMaxDevices = 64;
 int g_pair_clusters[kMaxDevices] = {0};      // resident 2-CTA clusters of the pair kernel per device (0: not asked yet)
 
 int make_kv_map(CUtensorMap* map, const void* base, const graft_attn_params* p, int box_rows = BN) {
-    const cuuint64_t dims[4] = {(cuuint64_t)p->d, (cuuint64_t)p->S_cap, (cuuint64_t)p->Hkv, (cuuint64_t)p->B};
+    // contiguous caches: (d, slot, KV head, sequence); paged: (d, row of the page, KV head, block of the pool)
+    const cuuint64_t dims[4] = {(cuuint64_t)p->d, (cuuint64_t)(p->block_table ? p->page_size : p->S_cap), (cuuint64_t)p->Hkv,
+                                (cuuint64_t)(p->block_table ? p->n_blocks : p->B)};
     const cuuint64_t strides[3] = {(cuuint64_t)p->kv_stride_s * 2, (cuuint64_t)p->kv_stride_h * 2, (cuuint64_t)p->kv_stride_b * 2};
     const cuuint32_t box[4] = {64, (cuuint32_t)box_rows, 1, 1};
     const cuuint32_t estr[4] = {1, 1, 1, 1};
@@ -2080,7 +2116,6 @@ bool graft_attn_tc_pair_supported(const graft_ctx* ctx, const graft_attn_params*
 
 bool graft_attn_tc_supported(const graft_ctx* ctx, const graft_attn_params* p) {
     if (p->d != D) return false;
-    if (p->block_table) return false;                                    // paged caches go through the register-tile kernel
     if ((long long)p->B * p->Hkv * 8 >= (1ll << 24)) return false;      // item ids share a word with the call stamp
     // TMA: 16-byte aligned base and strides (checked by the caller), strides below 2^40 bytes
     if (p->kv_stride_s * 2 >= (1ll << 40) || p->kv_stride_h * 2 >= (1ll << 40) || p->kv_stride_b * 2 >= (1ll << 40)) return false;

@@ -39,7 +39,8 @@ def gather_pool(Kp, table, S_cap):
     return out
 
 
-@pytest.mark.parametrize("cfg,kw,page", [("1", dict(), 128), ("5", dict(), 256), ("4", dict(B=2, L=3000), 128), ("2", dict(), 512)])
+@pytest.mark.parametrize("cfg,kw,page", [("1", dict(), 128), ("5", dict(), 256), ("4", dict(B=2, L=3000), 128), ("2", dict(), 512),
+                                         ("4", dict(B=1, L=20000), 1024), ("3", dict(B=8, L=1111), 128), ("tail", dict(B=3, L=5000), 256)])
 def test_paged_attention_and_compaction(cfg, kw, page):
     w = W.config(cfg, **kw)
     tree = oracle.build_tree(w)
@@ -57,7 +58,8 @@ def test_paged_attention_and_compaction(cfg, kw, page):
     vs.Q = w.Q.cuda()
     vs.build()
     Kd, Vd, td = Kp.cuda(), Vp.cuda(), torch.from_numpy(table).cuda()
-    for variant in (G.ATTN_AUTO, G.ATTN_MMA_SYNC):
+    tc = (G.ATTN_TCGEN05_2SM, G.ATTN_TCGEN05_L2PAIR) if w.d == 128 else ()
+    for variant in (G.ATTN_AUTO, G.ATTN_MMA_SYNC) + tc:
         vs.O.fill_(float("nan"))
         G.graft_tree_verify_attn(vs.ctx, Q=vs.Q, Kc=Kd, Vc=Vd, O=vs.O, seq_len=vs.seq_len, tree_size=vs.tree_size,
                                  tree_anc=vs.tree_anc, scale=w.scale, LSE=vs.LSE, variant=variant, block_table=td, S_cap=w.S_cap)
