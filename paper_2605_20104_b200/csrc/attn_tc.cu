@@ -1192,6 +1192,7 @@ struct SplitShared {
     float mx[2][2][128];     // [tile parity][half][row]; the idle parity carries the row sums at the end of a segment
 };
 
+template <bool PAGED>
 __device__ __forceinline__ void softmax_rows_split(const TcArgs& a, const Plan& plan, const SoftmaxBars lay, uint32_t bar0, uint32_t tmem, int rank,
                                              SplitShared& sh, volatile int* merge_flag, int& jt, int& n_seg_done, volatile int* abort_flag, unsigned* status) {
     const graft_attn_params& p = a.p;
@@ -1222,28 +1223,32 @@ __device__ __forceinline__ void softmax_rows_split(const TcArgs& a, const Plan& 
             const uint32_t tS = tmem + lane_bits + (gt % P_NSBUF) * 128 + half * 64;      // this thread's 64 score columns
             const uint32_t tP = tmem + lane_bits + (gt % P_NSBUF) * 128 + half * 32;      // its 64 P values (bf16 pairs)
             int overlap;
-            const bool paged = p.block_table != nullptr;
-            const int key0 = tile_key0(sg, sg.tile_lo + j, overlap, paged);
+            const int key0 = tile_key0(sg, sg.tile_lo + j, overlap, PAGED);
             const bool masked = key0 + BN > sg.L || overlap > 0;
-            const int n_valid = sg.L + sg.T - key0;         // keys of this tile that exist (paged caches: may be < 128 in the last tile)
             mbar_wait(bar(lay.S + gt % P_NSBUF), (gt / P_NSBUF) & 1, abort_flag, status);
             tc_fence_after();
-            const bool sanitize = paged && n_valid < BN;
-            if (sanitize) {
-                // the rows of the V tile past the sequence's keys may hold anything (0 x NaN would poison O): zero them
-                if (lay.v_full >= 0) mbar_wait(bar(lay.v_full + gt % lay.v_nslot), (gt / lay.v_nslot) & 1, abort_flag, status);
-                const uint32_t vs = lay.v_base + (gt % lay.v_nslot) * lay.v_slot_bytes + (uint32_t)n_valid * 128u;
-                const int nchunk = (BN - n_valid) * 8;       // 16-byte pieces per 64-column box
-                for (int bx = 0; bx < lay.v_boxes; ++bx)
-                    for (int c = (int)threadIdx.x - 128; c < nchunk; c += 256)
-                        asm volatile("st.shared.v4.b32 [%0], {%1, %1, %1, %1};" ::"r"(vs + bx * lay.v_box_stride + c * 16), "r"(0u) : "memory");
-                fence_async_smem();
-            }
             uint32_t x[2][32];
 #pragma unroll
             for (int c = 0; c < 2; ++c) tmem_ld32(tS + c * 32, x[c]);
             tmem_wait_ld();
             if (masked) {
+                if (PAGED) {
+                    // paged caches: an item's last tile may reach past the sequence's keys
+                    const int n_valid = sg.L + sg.T - key0;
+                    if (n_valid < BN) {
+                        // the rows of the V tile past the sequence's keys may hold anything (0 x NaN would poison O): zero them
+                        if (lay.v_full >= 0) mbar_wait(bar(lay.v_full + gt % lay.v_nslot), (gt / lay.v_nslot) & 1, abort_flag, status);
+                        const uint32_t vs = lay.v_base + (gt % lay.v_nslot) * lay.v_slot_bytes + (uint32_t)n_valid * 128u;
+                        const int nchunk = (BN - n_valid) * 8;       // 16-byte pieces per 64-column box
+                        for (int bx = 0; bx < lay.v_boxes; ++bx)
+                            for (int c = (int)threadIdx.x - 128; c < nchunk; c += 256)
+                                asm volatile("st.shared.v4.b32 [%0], {%1, %1, %1, %1};" ::"r"(vs + bx * lay.v_box_stride + c * 16), "r"(0u) : "memory");
+                        fence_async_smem();
+                        // the MMA that reads these rows is issued from the pair's leader after the P barrier: order the
+                        // stores before this thread's (relaxed) arrival there at cluster scope
+                        if (lay.remote) asm volatile("fence.acq_rel.cluster;" ::: "memory");
+                    }
+                }
                 // per 32-column chunk one word of allowed columns: cached keys not yet covered, ancestors in the tree
 #pragma unroll
                 for (int c = 0; c < 2; ++c) {
@@ -1315,9 +1320,7 @@ __device__ __forceinline__ void softmax_rows_split(const TcArgs& a, const Plan& 
             tc_fence_before();
             __syncwarp();
             if (lane == 0) {                               // one arrival per warp
-                if (lay.remote && sanitize)                // the zeroed rows must be visible to the MMA the leader issues: release at cluster scope
-                    asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(map_to_cta(bar(lay.P + gt % P_NSBUF), 0u)) : "memory");
-                else if (lay.remote) mbar_arrive_remote(map_to_cta(bar(lay.P + gt % P_NSBUF), 0u));
+                if (lay.remote) mbar_arrive_remote(map_to_cta(bar(lay.P + gt % P_NSBUF), 0u));
                 else mbar_arrive(bar(lay.P + gt % P_NSBUF));
             }
         }
@@ -1443,6 +1446,7 @@ __device__ __forceinline__ void softmax_rows_split(const TcArgs& a, const Plan& 
 }
 
 
+template <bool PAGED>
 __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(P_NTHREADS, 1)
 attn_tc_pair_kernel(const __grid_constant__ CUtensorMap kmap, const __grid_constant__ CUtensorMap vmap, const __grid_constant__ CUtensorMap qmap,
                     TcArgs a, unsigned* status) {
@@ -1512,12 +1516,15 @@ attn_tc_pair_kernel(const __grid_constant__ CUtensorMap kmap, const __grid_const
                 asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(stream_once));
                 for (int si = 0; si < nseg; ++si) {
                     const Seg sg = plan.seg[si];
+                    // paged caches: the block of the next tile is looked up one tile ahead, so that the table's latency
+                    // hides behind the wait for a free slot
+                    int blk_next = PAGED && sg.tile_lo < sg.tile_hi ? page_block(p, sg.b, sg.tile_lo * BN, status) : 0;
                     for (int t = sg.tile_lo; t < sg.tile_hi; ++t, ++jt) {
                         int overlap;
-                        const bool paged = p.block_table != nullptr;
-                        const int key0 = tile_key0(sg, t, overlap, paged);
+                        const int key0 = tile_key0(sg, t, overlap, PAGED);
                         // paged caches: the copy addresses (row of the page, block of the pool) instead of (slot, sequence)
-                        const int krow = paged ? key0 % p.page_size : key0, kblk = paged ? page_block(p, sg.b, key0, status) : sg.b;
+                        const int krow = PAGED ? key0 % p.page_size : key0, kblk = PAGED ? blk_next : sg.b;
+                        if (PAGED && t + 1 < sg.tile_hi) blk_next = page_block(p, sg.b, (t + 1) * BN, status);
                         const int slot = jt % P_NSLOT, use = jt / P_NSLOT;
                         if (use > 0) mbar_wait(bar(PB_EMPTY + slot), (use - 1) & 1, abort_flag, status);
                         if (rank == 0) mbar_expect_tx(bar(PB_FULL + slot), 2 * P_SLOT_BYTES);      // K and V halves of both CTAs
@@ -1624,7 +1631,7 @@ attn_tc_pair_kernel(const __grid_constant__ CUtensorMap kmap, const __grid_const
             // =============================== softmax, results (both CTAs) ===============================
             // this CTA's half of a V tile: all 128 keys, 64 of the d columns, behind the K half of the slot
             const SoftmaxBars lay = {PB_S, PB_P, PB_O, PB_EMPTY, P_NSLOT, true, sRing + P_HALF_TILE, P_SLOT_BYTES, P_NSLOT, 1, 0, -1};
-            softmax_rows_split(a, plan, lay, bar0, tmem, (int)rank, split, &ctrl.merge_flag, jt, n_seg_done, abort_flag, status);
+            softmax_rows_split<PAGED>(a, plan, lay, bar0, tmem, (int)rank, split, &ctrl.merge_flag, jt, n_seg_done, abort_flag, status);
         }
 
         // ---- next round (only batches with very many short sequences need more than one)
@@ -1669,9 +1676,11 @@ struct RbCtrl {
     uint32_t tmem;
     int abort;
     int merge_flag;
+    int blk[8];              // paged caches: pool block of the last few tiles (K looks it up, V reuses it)
 };
 static_assert(sizeof(RbCtrl) <= kCtrlBytes, "control block too large");
 
+template <bool PAGED>
 __global__ void __launch_bounds__(R_NTHREADS, 1)
 attn_tc_rb_kernel(const __grid_constant__ CUtensorMap kmap, const __grid_constant__ CUtensorMap vmap, const __grid_constant__ CUtensorMap qmap,
                   TcArgs a, unsigned* status) {
@@ -1749,13 +1758,29 @@ attn_tc_rb_kernel(const __grid_constant__ CUtensorMap kmap, const __grid_constan
                         idx -= n;
                     }
                 };
+                int pre_idx = -1, pre_blk = 0;
                 auto load = [&](int idx, bool is_v) {
                     Seg sg;
                     int t = 0, overlap;
                     locate(idx, sg, t);
-                    const bool paged = p.block_table != nullptr;
-                    const int key0 = tile_key0(sg, t, overlap, paged);
-                    const int krow = paged ? key0 % p.page_size : key0, kblk = paged ? page_block(p, sg.b, key0, status) : sg.b;
+                    const int key0 = tile_key0(sg, t, overlap, PAGED);
+                    // paged caches: K of tile idx looks the block up (one tile ahead of its use) and leaves it for V of the same tile
+                    int kblk = sg.b;
+                    if (PAGED) {
+                        if (is_v) kblk = ctrl.blk[idx & 7];
+                        else {
+                            kblk = idx == pre_idx ? pre_blk : page_block(p, sg.b, key0, status);
+                            ctrl.blk[idx & 7] = kblk;
+                            if (idx + 1 < total) {
+                                Seg s2;
+                                int t2 = 0;
+                                locate(idx + 1, s2, t2);
+                                pre_idx = idx + 1;
+                                pre_blk = page_block(p, s2.b, t2 * BN, status);
+                            }
+                        }
+                    }
+                    const int krow = PAGED ? key0 % p.page_size : key0;
                     const int g = jt + idx;              // global tile number
                     const int nslot = is_v ? R_NV : R_NK;
                     const int slot = g % nslot, use = g / nslot;
@@ -1870,7 +1895,7 @@ attn_tc_rb_kernel(const __grid_constant__ CUtensorMap kmap, const __grid_constan
         } else if (warp >= 4) {
             // =============================== softmax, results ===============================
             const SoftmaxBars lay = {RB_S, RB_P, RB_O, RB_EMPTYV, R_NV, false, sV, TILE_BYTES, R_NV, 2, HALF_BYTES, RB_FULLV};
-            softmax_rows_split(a, plan, lay, bar0, tmem, rank, split, &ctrl.merge_flag, jt, n_seg_done, abort_flag, status);
+            softmax_rows_split<PAGED>(a, plan, lay, bar0, tmem, rank, split, &ctrl.merge_flag, jt, n_seg_done, abort_flag, status);
         }
 
         // ---- next round (only batches with very many short sequences need more than one)
@@ -2076,8 +2101,10 @@ int graft_attn_tc_init() {
     }
     GRAFT_CHECK_CUDA(cudaFuncSetAttribute(attn_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_DYN));
     // pair kernel: how many 2-CTA clusters fit on the device at once (SMs that cannot be paired stay idle)
-    GRAFT_CHECK_CUDA(cudaFuncSetAttribute(attn_tc_pair_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, P_SMEM_DYN));
-    GRAFT_CHECK_CUDA(cudaFuncSetAttribute(attn_tc_rb_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, R_SMEM_DYN));
+    GRAFT_CHECK_CUDA(cudaFuncSetAttribute(attn_tc_pair_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, P_SMEM_DYN));
+    GRAFT_CHECK_CUDA(cudaFuncSetAttribute(attn_tc_pair_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, P_SMEM_DYN));
+    GRAFT_CHECK_CUDA(cudaFuncSetAttribute(attn_tc_rb_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, R_SMEM_DYN));
+    GRAFT_CHECK_CUDA(cudaFuncSetAttribute(attn_tc_rb_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, R_SMEM_DYN));
     int dev = 0;
     GRAFT_CHECK_CUDA(cudaGetDevice(&dev));
     if (dev >= 0 && dev < kMaxDevices && g_pair_clusters[dev] == 0) {
@@ -2095,7 +2122,7 @@ int graft_attn_tc_init() {
         cfg.attrs = &attr;
         cfg.numAttrs = 1;
         int n = 0;
-        if (cudaOccupancyMaxActiveClusters(&n, attn_tc_pair_kernel, &cfg) != cudaSuccess) { (void)cudaGetLastError(); n = 0; }
+        if (cudaOccupancyMaxActiveClusters(&n, attn_tc_pair_kernel<false>, &cfg) != cudaSuccess) { (void)cudaGetLastError(); n = 0; }
         g_pair_clusters[dev] = n > 0 ? (n < sms / 2 ? n : sms / 2) : -1;      // -1: the pair kernel cannot run here
     }
     return GRAFT_OK;
@@ -2174,9 +2201,12 @@ int graft_attn_tc_launch(graft_ctx* ctx, const graft_attn_params* p, cudaStream_
     if (use_pair) {
         int pairs = pair_clusters();
         if (pairs > ctx->num_sms / 2) pairs = ctx->num_sms / 2;       // the workspace has two slots per SM
-        attn_tc_pair_kernel<<<2 * pairs, P_NTHREADS, P_SMEM_DYN, stream>>>(kmap, vmap, qmap, a, ctx->status);
+        if (p->block_table) attn_tc_pair_kernel<true><<<2 * pairs, P_NTHREADS, P_SMEM_DYN, stream>>>(kmap, vmap, qmap, a, ctx->status);
+        else attn_tc_pair_kernel<false><<<2 * pairs, P_NTHREADS, P_SMEM_DYN, stream>>>(kmap, vmap, qmap, a, ctx->status);
     } else if (use_rb) {
-        attn_tc_rb_kernel<<<a.single ? ctx->num_sms : ctx->num_sms & ~1, R_NTHREADS, R_SMEM_DYN, stream>>>(kmap, vmap, qmap, a, ctx->status);
+        const int rb_grid = a.single ? ctx->num_sms : ctx->num_sms & ~1;
+        if (p->block_table) attn_tc_rb_kernel<true><<<rb_grid, R_NTHREADS, R_SMEM_DYN, stream>>>(kmap, vmap, qmap, a, ctx->status);
+        else attn_tc_rb_kernel<false><<<rb_grid, R_NTHREADS, R_SMEM_DYN, stream>>>(kmap, vmap, qmap, a, ctx->status);
     } else
     attn_tc_kernel<<<grid, NTHREADS, SMEM_DYN, stream>>>(kmap, vmap, qmap, a, ctx->status);
     GRAFT_CHECK_CUDA(cudaGetLastError());
