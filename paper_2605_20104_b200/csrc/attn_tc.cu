@@ -42,6 +42,8 @@
 #include <cuda_bf16.h>
 #include <math_constants.h>
 #include <stdlib.h>
+#include <climits>
+#include <type_traits>
 #include "graft_internal.cuh"
 
 namespace {
@@ -1218,13 +1220,15 @@ __device__ __forceinline__ void softmax_rows_split(const TcArgs& a, const Plan& 
         const unsigned long long allowed = sg.T >= 64 ? anc : (anc & ((1ull << sg.T) - 1ull));
         float m_ref = -CUDART_INF_F, l = 0.f;
 
-        for (int j = 0; j < nt; ++j) {
+        // Tiles that lie entirely among the cached keys need no mask at all; they come first and take the loop body
+        // without the masking code (the loop is sensitive to every instruction in it), the boundary tiles the full one.
+        auto one_tile = [&](int j, auto masked_tag) {
             const int gt = jt + j;
             const uint32_t tS = tmem + lane_bits + (gt % P_NSBUF) * 128 + half * 64;      // this thread's 64 score columns
             const uint32_t tP = tmem + lane_bits + (gt % P_NSBUF) * 128 + half * 32;      // its 64 P values (bf16 pairs)
-            int overlap;
-            const int key0 = tile_key0(sg, sg.tile_lo + j, overlap, PAGED);
-            const bool masked = key0 + BN > sg.L || overlap > 0;
+            constexpr bool masked = decltype(masked_tag)::value;
+            int overlap = 0;
+            const int key0 = masked ? tile_key0(sg, sg.tile_lo + j, overlap, PAGED) : 0;
             mbar_wait(bar(lay.S + gt % P_NSBUF), (gt / P_NSBUF) & 1, abort_flag, status);
             tc_fence_after();
             uint32_t x[2][32];
@@ -1323,7 +1327,12 @@ __device__ __forceinline__ void softmax_rows_split(const TcArgs& a, const Plan& 
                 if (lay.remote) mbar_arrive_remote(map_to_cta(bar(lay.P + gt % P_NSBUF), 0u));
                 else mbar_arrive(bar(lay.P + gt % P_NSBUF));
             }
-        }
+        };
+        const int n_keys_seg = sg.L + sg.T;
+        const int first_masked = min(sg.L / BN, PAGED ? INT_MAX : (n_keys_seg + BN - 1) / BN - 1);      // first tile of the item that needs the mask
+        const int j_plain = max(0, min(nt, first_masked - sg.tile_lo));
+        for (int j = 0; j < j_plain; ++j) one_tile(j, std::false_type{});
+        for (int j = j_plain; j < nt; ++j) one_tile(j, std::true_type{});
 
         // ---- results of the segment: the two halves of the row sum, then 64 O columns each: final rows or a partial
         const int last = (jt + nt - 1) & 1;          // the exchange buffer of the other parity is idle
