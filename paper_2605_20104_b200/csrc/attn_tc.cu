@@ -1222,14 +1222,19 @@ __device__ __forceinline__ void softmax_rows_split(const TcArgs& a, const Plan& 
 
         // Tiles that lie entirely among the cached keys need no mask at all; they come first and take the loop body
         // without the masking code (the loop is sensitive to every instruction in it), the boundary tiles the full one.
+        // score buffer and barrier phase of the tile at hand: kept as running values (gt % 3 and gt / 3 cost a dozen
+        // instructions each time)
+        int sb = jt % P_NSBUF;
+        uint32_t sph = (uint32_t)(jt / P_NSBUF) & 1u;
+        const uint32_t p_bar0 = lay.remote ? map_to_cta(bar(lay.P), 0u) : bar(lay.P);
         auto one_tile = [&](int j, auto masked_tag) {
             const int gt = jt + j;
-            const uint32_t tS = tmem + lane_bits + (gt % P_NSBUF) * 128 + half * 64;      // this thread's 64 score columns
-            const uint32_t tP = tmem + lane_bits + (gt % P_NSBUF) * 128 + half * 32;      // its 64 P values (bf16 pairs)
+            const uint32_t tS = tmem + lane_bits + sb * 128 + half * 64;      // this thread's 64 score columns
+            const uint32_t tP = tmem + lane_bits + sb * 128 + half * 32;      // its 64 P values (bf16 pairs)
             constexpr bool masked = decltype(masked_tag)::value;
             int overlap = 0;
             const int key0 = masked ? tile_key0(sg, sg.tile_lo + j, overlap, PAGED) : 0;
-            mbar_wait(bar(lay.S + gt % P_NSBUF), (gt / P_NSBUF) & 1, abort_flag, status);
+            mbar_wait(bar(lay.S + sb), sph, abort_flag, status);
             tc_fence_after();
             uint32_t x[2][32];
 #pragma unroll
@@ -1324,9 +1329,10 @@ __device__ __forceinline__ void softmax_rows_split(const TcArgs& a, const Plan& 
             tc_fence_before();
             __syncwarp();
             if (lane == 0) {                               // one arrival per warp
-                if (lay.remote) mbar_arrive_remote(map_to_cta(bar(lay.P + gt % P_NSBUF), 0u));
-                else mbar_arrive(bar(lay.P + gt % P_NSBUF));
+                if (lay.remote) mbar_arrive_remote(p_bar0 + 8u * (uint32_t)sb);
+                else mbar_arrive(p_bar0 + 8u * (uint32_t)sb);
             }
+            if (++sb == P_NSBUF) { sb = 0; sph ^= 1u; }
         };
         const int n_keys_seg = sg.L + sg.T;
         const int first_masked = min(sg.L / BN, PAGED ? INT_MAX : (n_keys_seg + BN - 1) / BN - 1);      // first tile of the item that needs the mask
