@@ -341,50 +341,118 @@ def run_timed(st, steps):
 
 
 def run_e2e(st, steps, warmup, variant):
-    """The same step with its inputs arriving from pinned host memory and its results read back.
-    The cached prefix is resident state (it was produced by earlier steps); the step's own inputs
-    are the draft arrays, Q, the tree tokens' K/V rows and the target's ids."""
-    w, vs = st["w"], st["vs"]
-    pin = lambda t: t.cpu().pin_memory()
+    """The same step with its inputs arriving from pinned host memory and its results read back on the host, every
+    step.  The cached prefix is resident state (it was produced by earlier steps); the step's own inputs are the
+    draft arrays, Q, the tree tokens' K/V rows and the target's ids; its results O, n_acc, path, bonus, new_seq_len.
+    Two sets of step buffers are in flight, as a serving loop keeps them: the copies of step i+1 (host to device) and
+    of step i-1 (device to host) run on their own streams beside the kernels of step i, and the host takes the
+    results of step i-1 (it waits for their copy) while step i runs."""
+    from paper_2605_20104_b200.step import VerifyStep
+    w, vs0 = st["w"], st["vs"]
     B, T = w.B, w.T_max
-    h_in = dict(draft_token=pin(vs.draft_token), draft_parent=pin(vs.draft_parent), draft_score=pin(vs.draft_score),
-                n_draft=pin(vs.n_draft), seq_len=pin(vs.seq_len), Q=pin(vs.Q), target_next=pin(vs.target_next))
-    L0 = int(w.seq_len.min())
-    h_k = torch.randn(B, w.Hkv, T, w.d).to(torch.bfloat16).pin_memory()
-    h_v = torch.randn(B, w.Hkv, T, w.d).to(torch.bfloat16).pin_memory()
-    d_k, d_v = torch.empty_like(h_k, device=vs.dev), torch.empty_like(h_v, device=vs.dev)
+    in_names = ("draft_token", "draft_parent", "draft_score", "n_draft", "seq_len", "Q", "target_next")
+    out_names = ("O", "n_acc", "path", "bonus", "new_seq_len")
     seq = [int(x) for x in w.seq_len]
-    h_out = dict(O=torch.empty_like(vs.O, device="cpu").pin_memory(), n_acc=pin(vs.n_acc), path=pin(vs.path),
-                 bonus=pin(vs.bonus), new_seq_len=pin(vs.new_seq_len))
-    h2d = sum(t.numel() * t.element_size() for t in h_in.values()) + h_k.numel() * 2 * 2
-    d2h = sum(t.numel() * t.element_size() for t in h_out.values())
+    same_len = len(set(seq)) == 1
 
-    def one(i):
+    def arena(tensors):
+        """One device buffer and one pinned host buffer that hold all `tensors` (name -> device tensor) back to back;
+        returns them and the typed device / host views.  One copy then moves the lot."""
+        offs, total = {}, 0
+        for k, t in tensors.items():
+            offs[k] = total
+            total += (t.numel() * t.element_size() + 255) // 256 * 256
+        dev = torch.empty(total, dtype=torch.uint8, device=vs0.dev)
+        host = torch.empty(total, dtype=torch.uint8).pin_memory()
+        view = lambda buf, k, t: buf[offs[k]:offs[k] + t.numel() * t.element_size()].view(t.dtype).view(t.shape)
+        dv = {k: view(dev, k, t) for k, t in tensors.items()}
+        hv = {k: view(host, k, t) for k, t in tensors.items()}
+        for k, t in tensors.items():
+            dv[k].copy_(t)
+            hv[k].copy_(t.cpu())
+        return dev, host, dv, hv
+
+    sets = []
+    rows_k = torch.randn(B, w.Hkv, T, w.d, device=vs0.dev).to(torch.bfloat16)     # the tree tokens' K/V rows (same every step)
+    rows_v = torch.randn(B, w.Hkv, T, w.d, device=vs0.dev).to(torch.bfloat16)
+    for n in range(2):
+        vs = vs0 if n == 0 else VerifyStep(w, device=torch.device(vs0.dev).index, upload_qkv=False)
+        if n:
+            vs.Q = vs0.Q.clone()
+        ins = {k: getattr(vs0, k) for k in in_names}
+        ins["d_k"], ins["d_v"] = rows_k, rows_v
+        d_in, h_in, dv_in, _ = arena(ins)
+        d_out, h_out, dv_out, hv_out = arena({k: getattr(vs, k) for k in out_names})
+        for k in in_names:                                   # the step's tensors are views of the two arenas from now on
+            setattr(vs, k, dv_in[k])
+        for k in out_names:
+            setattr(vs, k, dv_out[k])
+        vs.__dict__["_params"] = {}                          # marshalled argument structs pointed at the old tensors
+        sets.append(dict(vs=vs, d_in=d_in, h_in=h_in, d_out=d_out, h_out=h_out, hv_out=hv_out, d_k=dv_in["d_k"], d_v=dv_in["d_v"],
+                         in_ready=torch.cuda.Event(), cmp_done=torch.cuda.Event(), out_done=torch.cuda.Event()))
+    h2d = sum(getattr(vs0, k).numel() * getattr(vs0, k).element_size() for k in in_names) + 2 * sets[0]["d_k"].numel() * 2
+    d2h = sum(getattr(vs0, k).numel() * getattr(vs0, k).element_size() for k in out_names)
+    s_in, s_out, s_cmp = torch.cuda.Stream(), torch.cuda.Stream(), torch.cuda.current_stream()
+
+    def copy_in(i):
+        z = sets[i % 2]
+        s_in.wait_event(z["cmp_done"])                       # the kernels of step i-2 have read this set
+        with torch.cuda.stream(s_in):
+            z["d_in"].copy_(z["h_in"], non_blocking=True)
+            z["in_ready"].record(s_in)
+
+    def compute(i):
+        z = sets[i % 2]
+        vs = z["vs"]
         vs.Kc, vs.Vc = st["caches"][i % st["n_rot"]]
-        for k, t in h_in.items():
-            getattr(vs, k).copy_(t, non_blocking=True)
-        d_k.copy_(h_k, non_blocking=True)
-        d_v.copy_(h_v, non_blocking=True)
-        for b in range(B):                                   # the projection's write of the tree K/V rows
-            vs.Kc[b, :, seq[b]:seq[b] + T].copy_(d_k[b])
-            vs.Vc[b, :, seq[b]:seq[b] + T].copy_(d_v[b])
+        s_cmp.wait_event(z["in_ready"])
+        s_cmp.wait_event(z["out_done"])                      # the results of step i-2 have left this set
+        if same_len:                                         # the projection's write of the tree K/V rows
+            vs.Kc[:, :, seq[0]:seq[0] + T].copy_(z["d_k"])
+            vs.Vc[:, :, seq[0]:seq[0] + T].copy_(z["d_v"])
+        else:
+            for b in range(B):
+                vs.Kc[b, :, seq[b]:seq[b] + T].copy_(z["d_k"][b])
+                vs.Vc[b, :, seq[b]:seq[b] + T].copy_(z["d_v"][b])
         vs.build()
         vs.attn(variant)
         vs.accept()
         vs.compact()
-        for k, t in h_out.items():
-            t.copy_(getattr(vs, k), non_blocking=True)
-        torch.cuda.synchronize()                             # the caller reads the result every step
+        z["cmp_done"].record(s_cmp)
 
-    for i in range(warmup):
-        one(i)
-    t0, t1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    def copy_out(i):
+        z = sets[i % 2]
+        s_out.wait_event(z["cmp_done"])
+        with torch.cuda.stream(s_out):
+            z["h_out"].copy_(z["d_out"], non_blocking=True)
+            z["out_done"].record(s_out)
+
+    def run(n):
+        copy_in(0)
+        for i in range(n):
+            if i + 1 < n:
+                copy_in(i + 1)
+            compute(i)
+            copy_out(i)
+            if i > 0:
+                sets[(i - 1) % 2]["out_done"].synchronize()      # the caller reads the results of step i-1
+        sets[(n - 1) % 2]["out_done"].synchronize()
+
+    run(max(warmup, 2))
     torch.cuda.synchronize()
+    t0, t1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     t0.record()
-    for i in range(steps):
-        one(i)
+    run(steps)
+    torch.cuda.synchronize()
     t1.record()
     torch.cuda.synchronize()
+    # the two buffer sets hold the results of two consecutive steps on the same inputs: they must agree (bit for bit
+    # when the steps also saw the same cache), or the overlap of copies and kernels broke something
+    for k in out_names:
+        if k == "O" and st["n_rot"] > 1:                     # consecutive steps saw different caches
+            continue
+        if not torch.equal(sets[0]["hv_out"][k], sets[1]["hv_out"][k]):
+            raise RuntimeError("end-to-end run: the two buffer sets disagree on " + k)
     return t0.elapsed_time(t1) / steps, h2d, d2h
 
 
@@ -549,7 +617,9 @@ def main():
                      "algorithmic_bytes": kvb + qob, "traffic": TRAFFIC.get(args.workload)},
         "e2e": {"value": kvb * world / (e2e_ms * 1e-3) / 1e9, "unit": "GB/s", "ms_per_step": e2e_ms,
                 "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
-                "note": "cached prefix resident; step inputs (draft arrays, Q, tree K/V rows, target ids) from pinned host"},
+                "note": "cached prefix resident; step inputs (draft arrays, Q, tree K/V rows, target ids) from pinned host and "
+                        "results (O, n_acc, path, bonus, new_seq_len) read back every step; two buffer sets in flight: the copies "
+                        "of steps i+1 and i-1 overlap the kernels of step i"},
         "gpu_launches": 5 * args.steps,
         "clocks": clocks, "device_flags": flags,
     }
