@@ -8,6 +8,7 @@
 namespace {
 
 __global__ void __launch_bounds__(128) accept_kernel(graft_accept_params a, unsigned* status) {
+    graft_wait_for_stream();
     const int lane = threadIdx.x & 31;
     const int b = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
     if (b >= a.B) return;
@@ -76,7 +77,6 @@ extern "C" int graft_accept(graft_ctx* ctx, const graft_accept_params* p, void* 
         !p->path || !p->best_node || !p->bonus)
         return GRAFT_ERR_INVALID_ARG;
     const int warps = 4;
-    accept_kernel<<<(p->B + warps - 1) / warps, warps * 32, 0, (cudaStream_t)stream>>>(*p, ctx->status);
-    GRAFT_CHECK_CUDA(cudaGetLastError());
+    GRAFT_CHECK_CUDA(graft_launch(accept_kernel, dim3((p->B + warps - 1) / warps), dim3(warps * 32), 0, (cudaStream_t)stream, *p, ctx->status));
     return GRAFT_OK;
 }

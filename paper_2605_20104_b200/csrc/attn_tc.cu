@@ -582,6 +582,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap kmap, const __grid_constant__
                 tma_load_5d(sQ + blk * TILE_BYTES + half * HALF_BYTES, &qmap, half * 64, 0, (row0 + blk * 128) / G, sg.h, sg.b, bar(BAR_Q));
     };
 
+    asm volatile("griddepcontrol.wait;" ::: "memory");       // launched as a programmatic dependent: the kernel before this one is complete from here on
     a.epoch = next_call_no(a);
     if (warp == 0) plan_first(a, G, (int)blockIdx.x, (int)gridDim.x, blockIdx.x == 0, true, s_plan);
     if (threadIdx.x == 0) s_abort = 0;
@@ -1474,6 +1475,7 @@ attn_tc_pair_kernel(const __grid_constant__ CUtensorMap kmap, const __grid_const
     const uint32_t rank = cluster_ctarank();          // 0: leader (issues the MMAs), 1: peer
     const int worker = (int)(blockIdx.x >> 1), nworkers = (int)(gridDim.x >> 1);
 
+    asm volatile("griddepcontrol.wait;" ::: "memory");       // launched as a programmatic dependent: the kernel before this one is complete from here on
     a.epoch = next_call_no(a);
     if ((smem_u32(smem_raw) & 1023u) != 0) {          // the tiles would miss their alignment: refuse to run (both CTAs alike)
         if (threadIdx.x == 0) { atomicOr(status, (unsigned)GRAFT_FLAG_INTERNAL); cta_leaves(a); }
@@ -1710,6 +1712,7 @@ attn_tc_rb_kernel(const __grid_constant__ CUtensorMap kmap, const __grid_constan
     const int rank = a.single ? 0 : (int)(blockIdx.x & 1);           // which 128-row block of an item
     const int worker = a.single ? (int)blockIdx.x : (int)(blockIdx.x >> 1), nworkers = a.single ? (int)gridDim.x : (int)(gridDim.x >> 1);
 
+    asm volatile("griddepcontrol.wait;" ::: "memory");       // launched as a programmatic dependent: the kernel before this one is complete from here on
     a.epoch = next_call_no(a);
     if ((smem_u32(smem_raw) & 1023u) != 0) {          // the tiles would miss their alignment: refuse to run
         if (threadIdx.x == 0) { atomicOr(status, (unsigned)GRAFT_FLAG_INTERNAL); cta_leaves(a); }
@@ -1948,6 +1951,7 @@ constexpr int kMergeWarps = 8;       // warps per CTA; rows per CTA is a launch 
 
 __global__ void __launch_bounds__(kMergeWarps * 32, 4) merge_streamk_kernel(TcArgs a, int rows_per_cta, unsigned* status) {
     asm volatile("griddepcontrol.wait;" ::: "memory");      // launched early: nothing is read before the attention kernel is complete
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
     a.epoch = __ldcg(a.call_no);                            // the call the attention kernel just finished
     const graft_attn_params& p = a.p;
     const int G = a.G;
@@ -2216,14 +2220,14 @@ int graft_attn_tc_launch(graft_ctx* ctx, const graft_attn_params* p, cudaStream_
     if (use_pair) {
         int pairs = pair_clusters();
         if (pairs > ctx->num_sms / 2) pairs = ctx->num_sms / 2;       // the workspace has two slots per SM
-        if (p->block_table) attn_tc_pair_kernel<true><<<2 * pairs, P_NTHREADS, P_SMEM_DYN, stream>>>(kmap, vmap, qmap, a, ctx->status);
-        else attn_tc_pair_kernel<false><<<2 * pairs, P_NTHREADS, P_SMEM_DYN, stream>>>(kmap, vmap, qmap, a, ctx->status);
+        GRAFT_CHECK_CUDA(graft_launch(p->block_table ? attn_tc_pair_kernel<true> : attn_tc_pair_kernel<false>, dim3(2 * pairs),
+                                      dim3(P_NTHREADS), P_SMEM_DYN, stream, kmap, vmap, qmap, a, ctx->status));
     } else if (use_rb) {
         const int rb_grid = a.single ? ctx->num_sms : ctx->num_sms & ~1;
-        if (p->block_table) attn_tc_rb_kernel<true><<<rb_grid, R_NTHREADS, R_SMEM_DYN, stream>>>(kmap, vmap, qmap, a, ctx->status);
-        else attn_tc_rb_kernel<false><<<rb_grid, R_NTHREADS, R_SMEM_DYN, stream>>>(kmap, vmap, qmap, a, ctx->status);
+        GRAFT_CHECK_CUDA(graft_launch(p->block_table ? attn_tc_rb_kernel<true> : attn_tc_rb_kernel<false>, dim3(rb_grid),
+                                      dim3(R_NTHREADS), R_SMEM_DYN, stream, kmap, vmap, qmap, a, ctx->status));
     } else
-    attn_tc_kernel<<<grid, NTHREADS, SMEM_DYN, stream>>>(kmap, vmap, qmap, a, ctx->status);
+    GRAFT_CHECK_CUDA(graft_launch(attn_tc_kernel, dim3(grid), dim3(NTHREADS), SMEM_DYN, stream, kmap, vmap, qmap, a, ctx->status));
     GRAFT_CHECK_CUDA(cudaGetLastError());
     if (a.inkernel) return GRAFT_OK;               // merged in place: the last part of an item to finish combined them
     // few rows: one row per warp (the merge is latency-bound); many rows: four, to keep the CTA count down

@@ -45,6 +45,7 @@ __device__ __forceinline__ unsigned long long block_ballot(bool pred, unsigned* 
 }
 
 __global__ void __launch_bounds__(kThreads) build_tree_kernel(graft_build_params a, unsigned* status) {
+    graft_wait_for_stream();
     const int b = blockIdx.x, i = threadIdx.x;
     __shared__ int s_par[64], s_depth[64], s_sel[64], s_new[64];
     __shared__ int s_tok[64], s_opar[64];
@@ -253,7 +254,6 @@ extern "C" int graft_build_tree(graft_ctx* ctx, const graft_build_params* p, voi
     if (p->mode == GRAFT_PRUNE_GATED &&
         (p->n_ckpt > 0 && (!p->ckpt_depth || !p->ckpt_keep || !p->ckpt_log_tau || !p->tmpl_offset)))
         return GRAFT_ERR_INVALID_ARG;
-    build_tree_kernel<<<p->B, kThreads, 0, (cudaStream_t)stream>>>(*p, ctx->status);
-    GRAFT_CHECK_CUDA(cudaGetLastError());
+    GRAFT_CHECK_CUDA(graft_launch(build_tree_kernel, dim3(p->B), dim3(kThreads), 0, (cudaStream_t)stream, *p, ctx->status));
     return GRAFT_OK;
 }

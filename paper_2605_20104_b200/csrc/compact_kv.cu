@@ -10,6 +10,7 @@ namespace {
 constexpr int kThreads = 256;
 
 __global__ void __launch_bounds__(kThreads) compact_kernel(graft_compact_params a, unsigned* status) {
+    graft_wait_for_stream();
     extern __shared__ uint4 stage[];            // [n_acc][d/8] 16-byte chunks
     __shared__ int s_path[64];
     __shared__ int s_ok;
@@ -88,7 +89,6 @@ extern "C" int graft_compact_kv(graft_ctx* ctx, const graft_compact_params* p, v
     const long long ctas = 2ll * p->B * p->Hkv * p->n_layers;
     if (ctas > 0x7fffffffll) return GRAFT_ERR_UNSUPPORTED;
     const size_t smem = (size_t)p->T_max * (p->d / 8) * sizeof(uint4);     // <= 32 KB
-    compact_kernel<<<(unsigned)ctas, kThreads, smem, (cudaStream_t)stream>>>(*p, ctx->status);
-    GRAFT_CHECK_CUDA(cudaGetLastError());
+    GRAFT_CHECK_CUDA(graft_launch(compact_kernel, dim3((unsigned)ctas), dim3(kThreads), smem, (cudaStream_t)stream, *p, ctx->status));
     return GRAFT_OK;
 }

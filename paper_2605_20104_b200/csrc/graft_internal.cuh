@@ -23,6 +23,32 @@ struct graft_ctx {
 
 static inline bool graft_aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 
+// Every kernel of the library is launched as a programmatic dependent of the kernel before it in the stream: its CTAs
+// may be set up while that kernel still runs, and they wait (graft_wait_for_stream, the first statement of every
+// kernel) until it has completed and its writes are visible, so stream order holds for every input whatever kernel
+// produced it.  What is saved is the launch gap between the small kernels of a step.
+#ifdef __CUDACC__
+template <typename... KArgs, typename... Args>
+static inline cudaError_t graft_launch(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t stream, Args&&... args) {
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = grid;
+    cfg.blockDim = block;
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = stream;
+    cudaLaunchAttribute attr;
+    attr.id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr.val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = &attr;
+    cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...);
+}
+// first statement of a kernel: wait for the kernel before it in the stream, then let the one after it be set up
+__device__ __forceinline__ void graft_wait_for_stream() {
+    asm volatile("griddepcontrol.wait;" ::: "memory");
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+}
+#endif
+
 // attention launchers (one per kernel family); both return GRAFT_OK or an error code
 int graft_attn_mma_init();   // per device, called by graft_create with the device current
 int graft_attn_tc_init();
