@@ -1941,15 +1941,26 @@ attn_tc_rb_kernel(const __grid_constant__ CUtensorMap kmap, const __grid_constan
 }
 
 // ---------------------------------------------------------------------------------------------------
-// merge: one warp per output row of the padded [T_max * G] row space of a (b, h_kv)
+// merge: half a warp per output row of the padded [T_max * G] row space of a (b, h_kv)
 // ---------------------------------------------------------------------------------------------------
 // Rows of an item that was cut across CTAs are merged with  M = max m_i, w_i = 2^(m_i - M),
 // O = sum w_i O_i / sum w_i l_i;  rows of padding nodes are zeroed (LSE -inf); rows of items that one CTA
 // finished alone were already final.  The set of CTAs that hold a piece of an item follows from the
 // same cut as in the attention kernel.
-constexpr int kMergeWarps = 8;       // warps per CTA; rows per CTA is a launch parameter (8: one per warp, or 32)
+// The kernel is a chain of dependent round trips to L2 (the recorded cut, the partial slots' descriptors with
+// the parts' maxima and sums, the partial rows) and every row walks it once; what it costs is the number of
+// links times the number of rows a warp takes one after the other.  So a row belongs to sixteen lanes (eight
+// columns each) with lane i of them looking after part i, all rows of a launch are in flight at once as long as
+// the batch allows it, and the maximum and sum of both slots of a candidate CTA are requested together with
+// its descriptors instead of after them.  Items cut into many parts (few sequences on many SMs) take a whole
+// warp per row instead (LPR = 32): four columns per lane and eight parts' rows in flight rather than four.
+constexpr int kMergeWarps = 8;       // warps per CTA; rows per CTA is a launch parameter (one or four passes)
 
+template <int LPR>                   // lanes per row: 16 or 32
 __global__ void __launch_bounds__(kMergeWarps * 32, 4) merge_streamk_kernel(TcArgs a, int rows_per_cta, unsigned* status) {
+    constexpr int kRows = kMergeWarps * (32 / LPR);        // rows of a CTA in flight
+    constexpr int NL = 128 / LPR / 4;                      // 16-byte loads per lane and partial row
+    constexpr int PF = 8 / NL;                             // partial rows in flight per round
     asm volatile("griddepcontrol.wait;" ::: "memory");      // launched early: nothing is read before the attention kernel is complete
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
     a.epoch = __ldcg(a.call_no);                            // the call the attention kernel just finished
@@ -1981,14 +1992,17 @@ __global__ void __launch_bounds__(kMergeWarps * 32, 4) merge_streamk_kernel(TcAr
     const long long per = s_per;
     const bool pieces = s_pieces != 0;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    for (int r = grp * rows_per_cta + warp; r < min(rows_pad, (grp + 1) * rows_per_cta); r += kMergeWarps) {
+    const int hw = lane / LPR, hl = lane % LPR;             // which of the warp's rows, lane among the row's lanes
+    const unsigned hmask = LPR == 32 ? 0xffffffffu : 0xffffu << (16 * hw);      // the two halves of a warp go their own ways
+    for (int r = grp * rows_per_cta + (32 / LPR) * warp + hw; r < min(rows_pad, (grp + 1) * rows_per_cta); r += kRows) {
     const int t = r / G, g = r % G;
     __nv_bfloat16* orow = reinterpret_cast<__nv_bfloat16*>(p.O) + (size_t)b * p.o_stride_b + (size_t)t * p.o_stride_t +
-                          (size_t)(h * G + g) * p.o_stride_h + lane * 4;
+                          (size_t)(h * G + g) * p.o_stride_h + hl * (4 * NL);
     float* lse = p.LSE ? p.LSE + ((size_t)b * p.Hq + h * G + g) * p.T_max + t : nullptr;
     if (t >= si.T) {                       // padding node: zero row
-        *reinterpret_cast<uint2*>(orow) = make_uint2(0u, 0u);
-        if (lse && lane == 0) *lse = -CUDART_INF_F;
+        if (NL == 2) *reinterpret_cast<uint4*>(orow) = make_uint4(0u, 0u, 0u, 0u);
+        else *reinterpret_cast<uint2*>(orow) = make_uint2(0u, 0u);
+        if (lse && hl == 0) *lse = -CUDART_INF_F;
         continue;
     }
     const int rb = r / BR, rl = r % BR;
@@ -2009,59 +2023,83 @@ __global__ void __launch_bounds__(kMergeWarps * 32, 4) merge_streamk_kernel(TcAr
         nparts = (int)(last / per) - c_first + 1;
     }
     if (nparts <= 1) continue;             // one CTA had the whole item and wrote the final rows
-    // stream-K: part i lives in CTA c_first + i, in the slot whose descriptor names this item (none if
-    // that CTA's range held no tile of the item)
-    auto part_base = [&](int i) -> const float* {
-        int slot;
+    // Part i: its slot (-1: that CTA's range held no tile of the item), maximum and sum of this row.  Stream-K: part i
+    // lives in CTA c_first + i, in the slot whose descriptor names this item; both slots' values are requested at once.
+    auto part = [&](int i, int& slot, float& m, float& l) {
         if (pieces) {
             slot = 2 * (piece_cta0 + i);
+            const float* ml = a.partial + (size_t)slot * SLOT_FLOATS + BR * D + rl;
+            m = __ldcg(ml);
+            l = __ldcg(ml + BR);
         } else {
             const int c = c_first + i;
-            slot = a.desc[2 * c] == id ? 2 * c : (a.desc[2 * c + 1] == id ? 2 * c + 1 : -1);
+            const float* ml0 = a.partial + (size_t)(2 * c) * SLOT_FLOATS + BR * D + rl;
+            const int d0 = __ldcg(a.desc + 2 * c), d1 = __ldcg(a.desc + 2 * c + 1);
+            const float m0 = __ldcg(ml0), l0 = __ldcg(ml0 + BR), m1 = __ldcg(ml0 + SLOT_FLOATS), l1 = __ldcg(ml0 + SLOT_FLOATS + BR);
+            slot = d0 == id ? 2 * c : (d1 == id ? 2 * c + 1 : -1);
+            m = d0 == id ? m0 : m1;
+            l = d0 == id ? l0 : l1;
         }
-        return slot < 0 ? nullptr : a.partial + (size_t)slot * SLOT_FLOATS;
+        if (slot < 0) { m = -CUDART_INF_F; l = 0.f; }
     };
-    float acc[4] = {0.f, 0.f, 0.f, 0.f};
-    float den = 0.f, M = -CUDART_INF_F;
-    for (int i = lane; i < nparts; i += 32) {
-        const float* pb = part_base(i);
-        if (pb) M = fmaxf(M, pb[BR * D + rl]);
+    // lane hl keeps part hl (the first LPR); items cut into more parts than that walk the rest in rounds of LPR
+    int slot0 = -1;
+    float m0 = -CUDART_INF_F, l0 = 0.f;
+    if (hl < nparts) part(hl, slot0, m0, l0);
+    float M = m0;
+    for (int i = LPR + hl; i < nparts; i += LPR) {
+        int sl;
+        float m, l;
+        part(i, sl, m, l);
+        M = fmaxf(M, m);
     }
 #pragma unroll
-    for (int o = 16; o; o >>= 1) M = fmaxf(M, __shfl_xor_sync(0xffffffffu, M, o));
-    for (int i0 = 0; i0 < nparts; i0 += 32) {
-        float wgt = 0.f, l = 0.f;
-        const float* my_pb = i0 + lane < nparts ? part_base(i0 + lane) : nullptr;
-        if (my_pb) {
-            const float m = my_pb[BR * D + rl];
-            l = my_pb[BR * D + BR + rl];
-            wgt = (m == -CUDART_INF_F || M == -CUDART_INF_F) ? 0.f : exp2f(m - M);
-        }
-        den += wgt * l;
-        const int cnt = min(32, nparts - i0);
-        for (int j0 = 0; j0 < cnt; j0 += 8) {       // 8 partial rows in flight per round and four CTAs per SM: the kernel is bound by
-            float4 x[8];                              // the memory round trips in flight (two CTAs of 123 registers: +4 us on four 64K sequences)
+    for (int o = LPR / 2; o; o >>= 1) M = fmaxf(M, __shfl_xor_sync(hmask, M, o));
+    float acc[4 * NL];
 #pragma unroll
-            for (int j = 0; j < 8; ++j)
+    for (int q = 0; q < 4 * NL; ++q) acc[q] = 0.f;
+    float den = 0.f;
+    for (int i0 = 0; i0 < nparts; i0 += LPR) {
+        int slot = slot0;
+        float m = m0, l = l0;
+        if (i0 > 0) {
+            slot = -1; m = -CUDART_INF_F; l = 0.f;
+            if (i0 + hl < nparts) part(i0 + hl, slot, m, l);
+        }
+        const float wgt = (m == -CUDART_INF_F || M == -CUDART_INF_F) ? 0.f : exp2f(m - M);
+        den += wgt * l;
+        const int cnt = min(LPR, nparts - i0);
+        for (int j0 = 0; j0 < cnt; j0 += PF) {       // eight 16-byte loads in flight per round
+            float4 x[PF][NL];
+#pragma unroll
+            for (int j = 0; j < PF; ++j)
                 if (j0 + j < cnt) {
                     // the owner lane of part j0 + j knows whether it exists; a missing part has weight 0
-                    const unsigned long long pbj = __shfl_sync(0xffffffffu, (unsigned long long)my_pb, j0 + j);
-                    x[j] = pbj ? *reinterpret_cast<const float4*>(reinterpret_cast<const float*>(pbj) + (size_t)rl * D + lane * 4)
-                               : make_float4(0.f, 0.f, 0.f, 0.f);
+                    const int sj = __shfl_sync(hmask, slot, j0 + j, LPR);
+                    const float4* src = reinterpret_cast<const float4*>(a.partial + (size_t)(sj < 0 ? 0 : sj) * SLOT_FLOATS + (size_t)rl * D) + hl * NL;
+#pragma unroll
+                    for (int q = 0; q < NL; ++q) x[j][q] = sj >= 0 ? __ldcg(src + q) : make_float4(0.f, 0.f, 0.f, 0.f);
                 }
 #pragma unroll
-            for (int j = 0; j < 8; ++j)
+            for (int j = 0; j < PF; ++j)
                 if (j0 + j < cnt) {
-                    const float wj = __shfl_sync(0xffffffffu, wgt, j0 + j);
-                    acc[0] += wj * x[j].x; acc[1] += wj * x[j].y; acc[2] += wj * x[j].z; acc[3] += wj * x[j].w;
+                    const float wj = __shfl_sync(hmask, wgt, j0 + j, LPR);
+#pragma unroll
+                    for (int q = 0; q < NL; ++q) {
+                        acc[4 * q] += wj * x[j][q].x; acc[4 * q + 1] += wj * x[j][q].y; acc[4 * q + 2] += wj * x[j][q].z; acc[4 * q + 3] += wj * x[j][q].w;
+                    }
                 }
         }
     }
 #pragma unroll
-    for (int o = 16; o; o >>= 1) den += __shfl_xor_sync(0xffffffffu, den, o);
+    for (int o = LPR / 2; o; o >>= 1) den += __shfl_xor_sync(hmask, den, o);
     const float inv = den > 0.f ? 1.f / den : 0.f;
-    *reinterpret_cast<uint2*>(orow) = make_uint2(pack_bf16(acc[0] * inv, acc[1] * inv), pack_bf16(acc[2] * inv, acc[3] * inv));
-    if (lse && lane == 0) *lse = den > 0.f ? (M + log2f(den)) * kLn2 : -CUDART_INF_F;
+    if (NL == 2)
+        *reinterpret_cast<uint4*>(orow) = make_uint4(pack_bf16(acc[0] * inv, acc[1] * inv), pack_bf16(acc[2] * inv, acc[3] * inv),
+                                                     pack_bf16(acc[4 * NL - 4] * inv, acc[4 * NL - 3] * inv), pack_bf16(acc[4 * NL - 2] * inv, acc[4 * NL - 1] * inv));
+    else
+        *reinterpret_cast<uint2*>(orow) = make_uint2(pack_bf16(acc[0] * inv, acc[1] * inv), pack_bf16(acc[2] * inv, acc[3] * inv));
+    if (lse && hl == 0) *lse = den > 0.f ? (M + log2f(den)) * kLn2 : -CUDART_INF_F;
     }
 }
 
@@ -2230,9 +2268,12 @@ int graft_attn_tc_launch(graft_ctx* ctx, const graft_attn_params* p, cudaStream_
     GRAFT_CHECK_CUDA(graft_launch(attn_tc_kernel, dim3(grid), dim3(NTHREADS), SMEM_DYN, stream, kmap, vmap, qmap, a, ctx->status));
     GRAFT_CHECK_CUDA(cudaGetLastError());
     if (a.inkernel) return GRAFT_OK;               // merged in place: the last part of an item to finish combined them
-    // few rows: one row per warp (the merge is latency-bound); many rows: four, to keep the CTA count down
+    // Items in about four parts or fewer: half a warp per row; more: a warp per row.  Few rows: all of them in flight at
+    // once (the merge is latency-bound); many rows: four passes, to keep the CTA count down
     const int rows_pad = p->T_max * a.G;
-    const int rows_per_cta = (long long)p->B * p->Hkv * rows_pad >= 32768 ? 32 : 8;
+    const bool half_warp = 2 * (long long)workers <= 7 * (long long)p->B * p->Hkv;        // workers / items + 1 <= 4.5 parts
+    const int rows_flight = kMergeWarps * (half_warp ? 2 : 1);
+    const int rows_per_cta = (long long)p->B * p->Hkv * rows_pad >= 65536 ? 4 * rows_flight : rows_flight;
     const int groups = (rows_pad + rows_per_cta - 1) / rows_per_cta;
     // programmatic dependent launch: the merge CTAs are set up while the attention kernel still runs and wait
     // (griddepcontrol.wait) until it has completed and its writes are visible
@@ -2246,6 +2287,6 @@ int graft_attn_tc_launch(graft_ctx* ctx, const graft_attn_params* p, cudaStream_
     attr.val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = &attr;
     cfg.numAttrs = 1;
-    GRAFT_CHECK_CUDA(cudaLaunchKernelEx(&cfg, merge_streamk_kernel, a, rows_per_cta, ctx->status));
+    GRAFT_CHECK_CUDA(cudaLaunchKernelEx(&cfg, half_warp ? merge_streamk_kernel<16> : merge_streamk_kernel<32>, a, rows_per_cta, ctx->status));
     return GRAFT_OK;
 }
