@@ -2237,16 +2237,19 @@ int graft_attn_tc_launch(graft_ctx* ctx, const graft_attn_params* p, cudaStream_
     a.partial = reinterpret_cast<float*>(reinterpret_cast<char*>(ctx->ws) + GRAFT_WS_HEADER + kDescBytes + cut_bytes(p->B) + counter_bytes(p->B, p->Hkv));
     a.epoch = 0u;
     a.call_no = ctx->status + 4;            // two words of the workspace header
-    // Merge in the kernel (by the last part of an item to arrive) when items are cut into two or three parts: that CTA
-    // reads all parts of its 128 rows alone, which then beats a second launch (measured: -15 % on a batch of eight 4K
-    // contexts, -10 % on the ragged batch of sixteen; but +2 % on four 64K sequences cut into five parts each and
-    // +70 % on a single sequence cut into nine).  The host only knows the shapes: an item is about one KV head of one
-    // sequence, so there are about workers / (B * H_kv) + 1 parts per item; the kernel merges when that is below 2.5.
+    // Merge in the kernel (by the last part of an item to arrive) only for short calls whose items are cut into two or
+    // three parts: there the second launch costs more than one CTA reading all parts of its 128 rows alone.  The host
+    // only knows the shapes: an item is about one KV head of one sequence, so there are about workers / (B * H_kv) + 1
+    // parts per item.  Measured (Qwen3-14B heads, 74 workers, in-kernel against the merge kernel): 8 x 4K -5 us of 60,
+    // 8 x 8K -5 of 91, 5 x 8K -3 of 87, the ragged batch of sixteen -3 of 173; but 16 x 4K +3, 12 x 8K +1, and from 16K
+    // context on, where an early part has left L2 by the time the last one arrives, +15 to +17 us (5, 6, 8 x 16K;
+    // 5, 6 x 32K), +11 on 5 x 64K; a single sequence cut into nine +70 %.
     a.G = G;
     a.q_tma = q_tma ? 1 : 0;
     a.single = use_rb && p->T_max * G <= 128 ? 1 : 0;
     const int workers = a.single ? ctx->num_sms : ctx->num_sms / 2;
-    a.inkernel = (use_pair || use_rb) && workers <= 2 * (long long)p->B * p->Hkv ? 1 : 0;
+    const long long heads = (long long)p->B * p->Hkv;
+    a.inkernel = (use_pair || use_rb) && workers <= 2 * heads && heads <= workers && p->S_cap <= 12288 ? 1 : 0;
     a.prof_cta = 0;
 #ifdef GRAFT_TC_EXPERIMENTS
     if (getenv("GRAFT_TC_PROF_CTA")) a.prof_cta = atoi(getenv("GRAFT_TC_PROF_CTA"));
