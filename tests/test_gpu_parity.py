@@ -327,14 +327,16 @@ def test_many_short_sequences(orc, G, Step):
     full_case(orc, G, Step, w, "auto")
 
 
+@pytest.mark.parametrize("L0", [9000, 20000])
 @pytest.mark.parametrize("variant", ["mma", "one", "auto", "pair", "l2pair"])
-def test_one_long_sequence_among_short_ones(orc, G, Step, variant):
+def test_one_long_sequence_among_short_ones(orc, G, Step, variant, L0):
     """Enough (sequence, KV head) items that the kernels merge the parts of an item themselves, and one item that is
-    cut across most of the workers: its last part merges dozens of partials."""
+    cut across most of the workers: its last part merges dozens of partials.  With the longer context the merge
+    kernel runs instead, half a warp per row, and walks an item of more than sixteen parts in rounds."""
     rng = np.random.default_rng(27)
     B = 12
     parents = [W.random_tree_parents(rng, int(rng.integers(8, 33))) for _ in range(B)]
-    L = [9000] + [int(x) for x in rng.integers(50, 400, size=B - 1)]
+    L = [L0] + [int(x) for x in rng.integers(50, 400, size=B - 1)]
     w = W.custom(parents, Hq=16, Hkv=4, d=128, L=L, T_max=32, seed=27)
     rows = sample_rows(np.random.default_rng(127), orc.build_tree(w)["tree_size"], w.Hq, 400)
     full_case(orc, G, Step, w, variant, rows=rows)
