@@ -55,6 +55,40 @@ def measured_peaks():
     return 6650.0, "fallback"
 
 
+def tensor_peaks_tflops():
+    """Dense bf16 throughput, (burst, sustained under the power cap): measured, or the fallback figures."""
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(p):
+        d = json.load(open(p))
+        return float(d.get("bf16_tflops", 1590.0)), float(d.get("bf16_tflops_sustained", 1400.0))
+    return 1590.0, 1400.0
+
+
+EXP_PER_SECOND = 16 * 148 * 1.965e9      # exponential unit: 16 results per clock and SM, 148 SMs at the maximum SM clock
+
+
+def three_bounds(w, tree_size, attn_seconds, hbm_gbs):
+    """The attention call against each unit it needs (scores of R = T G rows per KV head against every visible key):
+    HBM time of the K/V, Q and O bytes, tensor time of 4 d R (L + T) flops per (sequence, KV head), exponential-unit
+    time of R (L + T) exponentials.  The slowest of the three is the binding bound of the shape.  The tensor time uses
+    the burst figure (these runs stay far below the power cap, at the maximum SM clock); the fraction of the sustained
+    figure is printed beside it."""
+    G = w.Hq // w.Hkv
+    keys = [int(w.seq_len[b]) + int(tree_size[b]) for b in range(w.B)]
+    rows = [int(tree_size[b]) * G for b in range(w.B)]
+    flops = sum(w.Hkv * 4 * w.d * r * k for r, k in zip(rows, keys))
+    exps = sum(w.Hkv * r * k for r, k in zip(rows, keys))
+    kv, qo = kv_bytes(w, tree_size)
+    burst, sustained = tensor_peaks_tflops()
+    t = {"hbm": (kv + qo) / (hbm_gbs * 1e9), "tensor": flops / (burst * 1e12), "exp": exps / EXP_PER_SECOND}
+    binding = max(t, key=t.get)
+    return {"useful_tflops": flops / attn_seconds / 1e12, "frac_of_bf16_burst": t["tensor"] / attn_seconds,
+            "frac_of_bf16_sustained": flops / (sustained * 1e12) / attn_seconds,
+            "frac_of_exp_unit": t["exp"] / attn_seconds, "frac_of_hbm": t["hbm"] / attn_seconds,
+            "binding": binding, "frac_of_binding": t[binding] / attn_seconds,
+            "floor_us": {k: v * 1e6 for k, v in t.items()}}
+
+
 def kv_bytes(w, tree_size):
     """Algorithmic bytes of one attention call: every visible K and V row once, plus Q and O."""
     kv = sum(w.Hkv * (int(w.seq_len[b]) + int(tree_size[b])) * w.d * 2 * 2 for b in range(w.B))
@@ -614,7 +648,8 @@ def main():
                      "frac": achieved / peak, "frac_of_8TBps_nominal": achieved / 8000.0,
                      "us_per_call": attn_ms * 1e3, "us_per_call_min": attn_ms_min * 1e3,
                      "us_per_call_series": st.get("attn_series"),
-                     "algorithmic_bytes": kvb + qob, "traffic": TRAFFIC.get(args.workload)},
+                     "algorithmic_bytes": kvb + qob, "traffic": TRAFFIC.get(args.workload),
+                     "units": three_bounds(w, st["tree"]["tree_size"], attn_ms * 1e-3, peak)},
         "e2e": {"value": kvb * world / (e2e_ms * 1e-3) / 1e9, "unit": "GB/s", "ms_per_step": e2e_ms,
                 "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
                 "note": "cached prefix resident; step inputs (draft arrays, Q, tree K/V rows, target ids) from pinned host and "
@@ -645,6 +680,8 @@ def main():
             extra.append({"workload": name, "us_per_step": ms2 * 1e3, "attn_us": a2 * 1e3, "attn_us_min": a2min * 1e3,
                           "attn_GBps": (kv2 + qo2) / (a2 * 1e-3) / 1e9,
                           "attn_frac_of_" + peak_kind: (kv2 + qo2) / (a2 * 1e-3) / 1e9 / peak,
+                          "attn_frac_of_8TBps_nominal": (kv2 + qo2) / (a2 * 1e-3) / 1e9 / 8000.0,
+                          "units": three_bounds(s2["w"], s2["tree"]["tree_size"], a2 * 1e-3, peak),
                           "kv_bytes": kv2, "l2": "larger than L2" if s2["n_rot"] == 1 else "rotating %d caches" % s2["n_rot"]})
             del s2
             torch.cuda.empty_cache()
