@@ -12,6 +12,8 @@
 namespace {
 
 constexpr int kThreads = 64;
+constexpr int kTmplCache = 128;     // template nodes and checkpoints kept in shared memory (larger inputs are read in place)
+constexpr int kCkptCache = 8;
 
 __device__ __forceinline__ bool better(float sa, int a, float sb, int b) {
     // order of "keep the top K draft nodes by cumulative path score": score desc, index asc
@@ -53,6 +55,9 @@ __global__ void __launch_bounds__(kThreads) build_tree_kernel(graft_build_params
     __shared__ float s_f2[2];
     __shared__ int s_i2[2];
     __shared__ unsigned s_u2[2];
+    __shared__ int s_tp[kTmplCache], s_tr[kTmplCache], s_te[kTmplCache];      // template parents, ranks, envelope indices
+    __shared__ int s_cd[kCkptCache], s_ck[kCkptCache], s_to[kCkptCache + 1];  // checkpoint depths, keep counts, template offsets
+    __shared__ float s_ct[kCkptCache];                                        // checkpoint thresholds
 
     int32_t* o_tok = a.tree_token + (size_t)b * a.T_max;
     int32_t* o_par = a.tree_parent + (size_t)b * a.T_max;
@@ -61,9 +66,30 @@ __global__ void __launch_bounds__(kThreads) build_tree_kernel(graft_build_params
     uint64_t* o_anc = a.tree_anc + (size_t)b * a.T_max;
     unsigned flags = 0;
 
+    // Every input that does not depend on another one is requested here, in one round trip to memory: the kernel is
+    // a chain of dependent loads (about 0.7 us each) and little else.
     const int n = a.n_draft[b];
     const int budget = a.k_max ? a.k_max[b] : a.K_max;
     const int L = a.seq_len[b];
+    int tok = -1, par = -1;
+    float sc = -CUDART_INF_F;
+    if (i < a.N_max) {
+        tok = a.draft_token[(size_t)b * a.N_max + i];
+        par = a.draft_parent[(size_t)b * a.N_max + i];
+        sc = a.draft_score[(size_t)b * a.N_max + i];
+    }
+    const int keep_count = a.mode == GRAFT_PRUNE_TOPK ? a.keep_count[b] : 0;
+    const bool tmpl_cached = a.N_tmpl <= kTmplCache, ckpt_cached = a.n_ckpt <= kCkptCache;
+    if (a.mode != GRAFT_PRUNE_NONE && tmpl_cached)
+        for (int u = i; u < a.N_tmpl; u += kThreads) {
+            s_tp[u] = a.tmpl_parent[u];
+            s_tr[u] = a.tmpl_rank[u];
+            s_te[u] = a.env_token ? a.tmpl_env[u] : 0;
+        }
+    if (a.mode == GRAFT_PRUNE_GATED && ckpt_cached) {
+        if (i < a.n_ckpt) { s_cd[i] = a.ckpt_depth[i]; s_ck[i] = a.ckpt_keep[i]; s_ct[i] = a.ckpt_log_tau[i]; }
+        if (i <= a.n_ckpt && a.n_ckpt > 0) s_to[i] = a.tmpl_offset[i];
+    }
     if (n < 1 || n > a.N_max || budget < 1 || budget > a.T_max || L < 0 ||
         (long long)L + a.T_max > (long long)a.S_cap) {
         if (i < a.T_max) { o_tok[i] = -1; o_par[i] = -1; o_pos[i] = 0; o_src[i] = INT_MIN; o_anc[i] = 0; }
@@ -72,12 +98,8 @@ __global__ void __launch_bounds__(kThreads) build_tree_kernel(graft_build_params
     }
 
     // ---- 1. load, depth and validity by climbing the parent chain (strictly decreasing indices)
-    int tok = -1, par = -1;
-    float sc = -CUDART_INF_F;
+    if (i >= n) { tok = -1; par = -1; sc = -CUDART_INF_F; }
     if (i < n) {
-        tok = a.draft_token[(size_t)b * a.N_max + i];
-        par = a.draft_parent[(size_t)b * a.N_max + i];
-        sc = a.draft_score[(size_t)b * a.N_max + i];
         if (sc != sc) { sc = -CUDART_INF_F; if (i > 0) flags |= GRAFT_FLAG_NAN_SCORE; }
         if (i > 0 && (par < 0 || par >= i)) flags |= GRAFT_FLAG_BAD_PARENT;
     }
@@ -106,20 +128,20 @@ __global__ void __launch_bounds__(kThreads) build_tree_kernel(graft_build_params
     } else if (a.mode == GRAFT_PRUNE_TOPK || a.mode == GRAFT_PRUNE_GATED) {
         int K_draft = n, max_depth = INT_MAX;
         if (a.mode == GRAFT_PRUNE_TOPK) {
-            K_draft = a.keep_count[b];
+            K_draft = keep_count;
         } else {
             int stage = -1;
             for (int c = 0; c < a.n_ckpt && stage < 0; ++c) {
-                const int D = a.ckpt_depth[c];
+                const int D = ckpt_cached ? s_cd[c] : a.ckpt_depth[c];
                 float smax = block_max((valid && i > 0 && depth == D) ? sc : -CUDART_INF_F, s_f2);
-                if (smax <= a.ckpt_log_tau[c]) stage = c;     // c_d <= tau_d: gate closed, prune here
+                if (smax <= (ckpt_cached ? s_ct[c] : a.ckpt_log_tau[c])) stage = c;     // c_d <= tau_d: gate closed, prune here
             }
             if (stage < 0) graft = false;
             else {
-                K_draft = a.ckpt_keep[stage];
-                max_depth = a.ckpt_depth[stage];
-                t_lo = a.tmpl_offset[stage];
-                t_hi = a.tmpl_offset[stage + 1];
+                K_draft = ckpt_cached ? s_ck[stage] : a.ckpt_keep[stage];
+                max_depth = ckpt_cached ? s_cd[stage] : a.ckpt_depth[stage];
+                t_lo = ckpt_cached ? s_to[stage] : a.tmpl_offset[stage];
+                t_hi = ckpt_cached ? s_to[stage + 1] : a.tmpl_offset[stage + 1];
             }
         }
         if (graft) {
@@ -169,14 +191,15 @@ __global__ void __launch_bounds__(kThreads) build_tree_kernel(graft_build_params
     int T = K_kept;
     if (graft) {
         const int K_ret = max(0, min(t_hi - t_lo, budget - K_kept));
+        const bool from_cache = tmpl_cached && t_lo >= 0 && t_hi <= a.N_tmpl;
         const int attach = a.attach_tail && K_kept > 0 ? K_kept - 1 : 0;      // where template nodes without a template parent hang
         T += K_ret;
         const int u = i;
         int tp = -1, r = 0, du = 0;
         bool ok = true;
         if (u < K_ret) {
-            tp = a.tmpl_parent[t_lo + u];
-            r = a.tmpl_rank[t_lo + u];
+            tp = from_cache ? s_tp[t_lo + u] : a.tmpl_parent[t_lo + u];
+            r = from_cache ? s_tr[t_lo + u] : a.tmpl_rank[t_lo + u];
             if (tp < -1 || tp >= u || r < 0 || r >= a.k) { ok = false; tp = -1; flags |= GRAFT_FLAG_BAD_TEMPLATE; }
         }
         s_par[i] = tp;                       // template-local parents (draft parents no longer needed)
@@ -194,7 +217,7 @@ __global__ void __launch_bounds__(kThreads) build_tree_kernel(graft_build_params
             // the envelope holds the token of every rank path already: one independent load per node
             if (u < K_ret) {
                 int x = -1;
-                const int e = a.tmpl_env[t_lo + u];
+                const int e = from_cache ? s_te[t_lo + u] : a.tmpl_env[t_lo + u];
                 if (e < 0 || e >= a.N_env) flags |= GRAFT_FLAG_BAD_TEMPLATE;
                 else if (ok) {
                     x = a.env_token[(size_t)b * a.N_env + e];
