@@ -13,7 +13,22 @@ __global__ void __launch_bounds__(128) accept_kernel(graft_accept_params a, unsi
     const int b = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
     if (b >= a.B) return;
     const size_t row = (size_t)b * a.T_max;
+    // every input is requested at once (the arrays are [B, T_max] whatever the tree's size): the kernel is one round
+    // trip to memory, a few ballots and shuffles, and the stores
     const int T = a.tree_size[b];
+    unsigned long long anc_in[2];
+    int tok_in[2], par_in[2], next_in[2];
+#pragma unroll
+    for (int s = 0; s < 2; ++s) {
+        const int i = lane + 32 * s;
+        anc_in[s] = 0; tok_in[s] = -1; par_in[s] = -1; next_in[s] = -1;
+        if (i < a.T_max) {
+            anc_in[s] = a.tree_anc[row + i];
+            tok_in[s] = a.tree_token[row + i];
+            par_in[s] = a.tree_parent[row + i];
+            next_in[s] = a.target_next[row + i];
+        }
+    }
     int32_t* path = a.path + row;
     if (T < 1 || T > a.T_max) {
         for (int j = lane; j < a.T_max; j += 32) path[j] = -1;
@@ -25,16 +40,13 @@ __global__ void __launch_bounds__(128) accept_kernel(graft_accept_params a, unsi
 #pragma unroll
     for (int s = 0; s < 2; ++s) {
         const int i = lane + 32 * s;
-        anc[s] = 0;
-        match[s] = false;
-        if (i < T) {
-            anc[s] = a.tree_anc[row + i];
-            if (i == 0) match[s] = true;
-            else {
-                const int tok = a.tree_token[row + i], p = a.tree_parent[row + i];
-                if (p >= 0 && p < i) match[s] = tok >= 0 && tok == a.target_next[row + p];
-            }
-        }
+        anc[s] = i < T ? anc_in[s] : 0;
+        // the target's id at the parent sits in lane parent % 32
+        const int tok = tok_in[s], p = par_in[s];
+        const int pc = (p >= 0 && p < 64) ? p : 0;
+        const int n0 = __shfl_sync(0xffffffffu, next_in[0], pc & 31), n1 = __shfl_sync(0xffffffffu, next_in[1], pc & 31);
+        const int next_p = pc < 32 ? n0 : n1;
+        match[s] = i < T && (i == 0 || (p >= 0 && p < i && tok >= 0 && tok == next_p));
     }
     const unsigned long long matched =
         (unsigned long long)__ballot_sync(0xffffffffu, match[0]) | ((unsigned long long)__ballot_sync(0xffffffffu, match[1]) << 32);
@@ -60,10 +72,11 @@ __global__ void __launch_bounds__(128) accept_kernel(graft_accept_params a, unsi
         const int i = lane + 32 * s;
         if ((banc >> i) & 1ull) path[__popcll(banc & ((1ull << i) - 1ull))] = i;
     }
+    const int bonus = __shfl_sync(0xffffffffu, best < 32 ? next_in[0] : next_in[1], owner);
     if (lane == 0) {
         a.n_acc[b] = n;
         a.best_node[b] = best;
-        a.bonus[b] = a.target_next[row + best];
+        a.bonus[b] = bonus;
     }
 }
 

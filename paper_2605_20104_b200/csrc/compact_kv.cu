@@ -21,13 +21,15 @@ __global__ void __launch_bounds__(kThreads) compact_kernel(graft_compact_params 
     const int layer = idx / a.B;
     const int L = a.seq_len[b];
     const int n = a.n_acc[b];
+    // asked for together with the two above (the array is [B, T_max] whatever n_acc says): one round trip less
+    const int path_in = (int)threadIdx.x < a.T_max ? a.path[(size_t)b * a.T_max + threadIdx.x] : -1;
     const int chunks = a.d / 8;
 
     if (threadIdx.x == 0) s_ok = 1;
     __syncthreads();
     bool bad = n < 0 || n > a.T_max || L < 0;
     if (!bad && threadIdx.x < n) {
-        const int pj = a.path[(size_t)b * a.T_max + threadIdx.x];
+        const int pj = path_in;
         s_path[threadIdx.x] = pj;
         if (pj < (int)threadIdx.x || pj >= a.T_max || (long long)L + pj >= a.S_cap) bad = true;
     }
