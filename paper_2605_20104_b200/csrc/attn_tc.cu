@@ -105,6 +105,12 @@ struct SeqInfo {
     bool found;
 };
 
+// Quotient of two non-negative 64-bit numbers; nearly always both fit 32 bits, and the 64-bit division is a routine of
+// a hundred-odd instructions on the one thread that plans.
+__device__ __forceinline__ long long udiv(long long a, long long b) {
+    if ((((unsigned long long)a | (unsigned long long)b) >> 32) == 0) return (long long)((unsigned)a / (unsigned)b);
+    return a / b;
+}
 __device__ __forceinline__ void seq_shape(const graft_attn_params& p, int G, int b, int& L, int& T, int& nrb, int& ntiles, int& wlast) {
     L = p.seq_len[b];
     T = p.tree_size[b];
@@ -122,9 +128,9 @@ __device__ __forceinline__ long long head_units(int ntiles, int nrb, int wlast) 
 __device__ __forceinline__ void piece_shape(int ntiles, long long per, int& nsplit, int& plen) {
     nsplit = plen = 0;
     if (ntiles <= 0) return;
-    long long want = ntiles / per;
+    long long want = udiv(ntiles, per);
     if (want < 1) want = 1;
-    plen = (int)((ntiles + want - 1) / want);
+    plen = (int)udiv(ntiles + want - 1, want);
     nsplit = (ntiles + plen - 1) / plen;
 }
 
@@ -192,9 +198,9 @@ __device__ __forceinline__ void choose_cut(const graft_attn_params& p, int G, in
     SeqEntry* table = record ? reinterpret_cast<SeqEntry*>(record + 1) : nullptr;
     long long tiles;
     (void)scan_sequences(p, G, 0, -1, total, tiles, 0, table);
-    const long long per_tiles = (tiles + grid - 1) / grid > 0 ? (tiles + grid - 1) / grid : 1;
+    const long long per_tiles = udiv(tiles + grid - 1, grid) > 0 ? udiv(tiles + grid - 1, grid) : 1;
     pieces = false;
-    per = (total + grid - 1) / grid;
+    per = udiv(total + grid - 1, grid);
     if (per < kW2) per = kW2;   // a range never shorter than the heaviest tile, so every CTA inside an item's span owns a tile
     if (per_tiles < kStreamMinTiles) {
         long long units, dummy;
@@ -218,7 +224,7 @@ __device__ __forceinline__ void item_span(const SeqInfo& si, int h, int rb, long
 __device__ __forceinline__ long long tiles_below(long long g, long long U, int w) {
     if (g <= U) return 0;
     const long long a = g - U - kOvh;
-    const long long c = a > 0 ? (a + w - 1) / w : 0;
+    const long long c = a > 0 ? udiv(a + w - 1, w) : 0;
     return c < 1 ? 1 : c;
 }
 __device__ __forceinline__ int item_id(const graft_attn_params& p, int b, int h, int rb) { return ((b * p.Hkv + h) << 3) | rb; }
@@ -274,9 +280,9 @@ __device__ __forceinline__ void plan_round(const TcArgs& a, int G, int worker, b
         const long long hu = head_units(si.ntiles, si.nrb, si.wlast);
         const long long seq_end = si.base + (long long)p.Hkv * hu;
         // walk the items of this sequence from the one that holds unit g
-        int h = (int)((g - si.base) / hu);
-        const long long rem = (g - si.base) % hu;
-        int rb = (int)(rem / ((long long)si.ntiles * kW2 + kOvh));
+        int h = (int)udiv(g - si.base, hu);
+        const long long rem = (g - si.base) - (long long)h * hu;
+        int rb = (int)udiv(rem, (long long)si.ntiles * kW2 + kOvh);
         if (rb > si.nrb - 1) rb = si.nrb - 1;
         while (g < g_hi && g < seq_end && n < MAXSEG) {
             long long U;
@@ -300,8 +306,8 @@ __device__ __forceinline__ void plan_round(const TcArgs& a, int G, int worker, b
                     // the workers whose ranges hold a tile of this item
                     const long long per = pl.per;
                     const long long last = si.ntiles > 1 ? U + kOvh + (long long)(si.ntiles - 1) * w : U;
-                    sg.c_first = (int)(U / per);
-                    sg.c_span = (int)(last / per) - sg.c_first + 1;
+                    sg.c_first = (int)udiv(U, per);
+                    sg.c_span = (int)udiv(last, per) - sg.c_first + 1;
                     sg.nparts = 0;
                     for (int c = sg.c_first; a.inkernel && c < sg.c_first + sg.c_span; ++c) {
                         long long lo = tiles_below(c * per, U, w), hi = tiles_below((c + 1) * per, U, w);
@@ -2018,9 +2024,9 @@ __global__ void __launch_bounds__(kMergeWarps * 32, 4) merge_streamk_kernel(TcAr
         long long U;
         int w;
         item_span(si, h, rb, U, w);
-        c_first = (int)(U / per);
+        c_first = (int)udiv(U, per);
         const long long last = si.ntiles > 1 ? U + kOvh + (long long)(si.ntiles - 1) * w : U;      // first unit of the last tile
-        nparts = (int)(last / per) - c_first + 1;
+        nparts = (int)udiv(last, per) - c_first + 1;
     }
     if (nparts <= 1) continue;             // one CTA had the whole item and wrote the final rows
     // Part i: its slot (-1: that CTA's range held no tile of the item), maximum and sum of this row.  Stream-K: part i
