@@ -45,6 +45,7 @@ __global__ void __launch_bounds__(UT, 2) update_kernel(graft_update_params p, un
     __shared__ float s_cv[UCAP];
     __shared__ int s_ci[UCAP];
     __shared__ float s_wtop[UT / 32][UK];
+    __shared__ int s_rank[(UT / 32) * UK];
     __shared__ int s_hot[UT];
     __shared__ int s_cnt, s_nhot, s_min, s_dup;
     __shared__ float s_tau;
@@ -97,30 +98,30 @@ __global__ void __launch_bounds__(UT, 2) update_kernel(graft_update_params p, un
             x = up ? fmaxf(x, y) : fminf(x, y);
         }
     if (lane < UK) s_wtop[warp][lane] = x;
+    if (tid < (UT / 32) * UK) s_rank[tid] = 0;
     __syncthreads();
-    if (warp == 0) {
-        float c[(UT / 32) * UK / 32];               // 8 values per lane
-#pragma unroll
-        for (int q = 0; q < (UT / 32) * UK / 32; ++q) c[q] = (&s_wtop[0][0])[q * 32 + lane];
-        float tau = -CUDART_INF_F;
-        for (int j = 0; j < k; ++j) {
-            float best = -CUDART_INF_F;
-            int at = 0;
-#pragma unroll
-            for (int q = 0; q < (UT / 32) * UK / 32; ++q)
-                if (c[q] > best) { best = c[q]; at = q; }
-            float wbest = best;
-#pragma unroll
-            for (int o = 16; o; o >>= 1) wbest = fmaxf(wbest, __shfl_xor_sync(0xffffffffu, wbest, o));
-            tau = wbest;
-            const unsigned who = __ballot_sync(0xffffffffu, best == wbest);
-            if (lane == __ffs(who) - 1) {            // remove one occurrence
-#pragma unroll
-                for (int q = 0; q < (UT / 32) * UK / 32; ++q)
-                    if (q == at) c[q] = -CUDART_INF_F;
+    // The k largest of a warp are the only ones of its 32 that can be among the k largest of all: (UT / 32) * k
+    // candidates.  Every candidate counts how many candidates come before it (larger, or equal with a lower index), a few
+    // threads per candidate sharing the count; the one with k - 1 before it is the k-th largest.
+    {
+        const int nc = (UT / 32) * k;                 // <= 256
+        const int parts = UT / nc;                    // >= 2 threads per candidate
+        const int c = tid % nc, part = tid / nc;
+        if (part < parts) {
+            const float v = s_wtop[c / k][c % k];
+            const int per = (nc + parts - 1) / parts;
+            const int lo = part * per, hi = min(nc, lo + per);
+            int ahead = 0;
+            int w = lo / k, jj = lo % k;                // candidate j = w * k + jj, walked without a division per step
+            for (int j = lo; j < hi; ++j) {
+                const float u = s_wtop[w][jj];
+                ahead += (u > v || (u == v && j < c)) ? 1 : 0;
+                if (++jj == k) { jj = 0; ++w; }
             }
+            if (ahead) atomicAdd(&s_rank[c], ahead);
         }
-        if (lane == 0) s_tau = tau;
+        __syncthreads();
+        if (tid < nc && s_rank[tid] == k - 1) s_tau = s_wtop[tid / k][tid % k];
     }
     __syncthreads();
     const float tau = s_tau;
@@ -209,7 +210,16 @@ __global__ void __launch_bounds__(UT, 2) update_kernel(graft_update_params p, un
 
     // ---- the k best of the list (warp 0)
     int n_sel = 0;
-    if (warp == 0) {
+    if (n_gt <= UT) {
+        // the usual, short list: every entry counts the entries that come before it and takes that place
+        if (tid < n_gt) {
+            const float v = s_cv[tid];
+            const int id = s_ci[tid];
+            int ahead = 0;
+            for (int e = 0; e < n_gt; ++e) ahead += before(s_cv[e], s_ci[e], v, id) ? 1 : 0;
+            if (ahead < k) s_top[ahead] = id;
+        }
+    } else if (warp == 0) {
         for (int j = 0; j < k && j < n_gt; ++j) {
             float bv = -CUDART_INF_F;
             int bi = 0x7fffffff, be = -1;
