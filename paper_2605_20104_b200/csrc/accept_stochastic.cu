@@ -51,6 +51,7 @@ __device__ __forceinline__ void scaled8(const __nv_bfloat16* row, int v0, int V,
 // One CTA per tree node; a warp takes a step of 256 ids at a time (four in flight), leaves the step's
 // (max, sum of exponentials relative to it) and folds it into its running pair.
 __global__ void __launch_bounds__(ST, 2) softmax_stats_kernel(graft_accept_stochastic_params p) {
+    graft_wait_for_stream();
     __shared__ float s_m[ST / 32], s_s[ST / 32];
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int r = blockIdx.x, b = r / p.T_max, i = r % p.T_max;
@@ -132,6 +133,7 @@ __global__ void __launch_bounds__(ST, 2) softmax_stats_kernel(graft_accept_stoch
 }
 
 __global__ void __launch_bounds__(WT) accept_walk_kernel(graft_accept_stochastic_params p, unsigned* status) {
+    graft_wait_for_stream();
     constexpr int NW = WT / 32;
     __shared__ int s_par[64], s_tok[64];
     __shared__ float s_w[64];                 // weight exp(z - m) of node i's token in its parent's row
@@ -302,9 +304,8 @@ extern "C" int graft_accept_stochastic(graft_ctx* ctx, const graft_accept_stocha
         return GRAFT_ERR_INVALID_ARG;
     if (!graft_aligned16(p->logits) || p->logits_stride_row < p->V || p->logits_stride_row % 8 != 0) return GRAFT_ERR_INVALID_ARG;
     cudaStream_t s = static_cast<cudaStream_t>(stream);
-    softmax_stats_kernel<<<p->B * p->T_max, ST, 0, s>>>(*p);
-    GRAFT_CHECK_CUDA(cudaGetLastError());
-    accept_walk_kernel<<<p->B, WT, 0, s>>>(*p, ctx->status);
-    GRAFT_CHECK_CUDA(cudaGetLastError());
+    // both kernels are programmatic dependents of the kernel before them: the walk's CTAs are set up while the statistics drain
+    GRAFT_CHECK_CUDA(graft_launch(softmax_stats_kernel, dim3(p->B * p->T_max), dim3(ST), 0, s, *p));
+    GRAFT_CHECK_CUDA(graft_launch(accept_walk_kernel, dim3(p->B), dim3(WT), 0, s, *p, ctx->status));
     return GRAFT_OK;
 }

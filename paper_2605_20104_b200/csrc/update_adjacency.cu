@@ -51,6 +51,7 @@ __global__ void __launch_bounds__(UT, 2) update_kernel(graft_update_params p, un
     __shared__ float s_tau;
     __shared__ int s_top[UK];
 
+    graft_wait_for_stream();
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int r = blockIdx.x, b = r / p.T_max, i = r % p.T_max;
     int T = p.tree_size[b];
@@ -300,7 +301,6 @@ extern "C" int graft_update_adjacency(graft_ctx* ctx, const graft_update_params*
     // the candidate list holds what k-1 threads can contribute
     const long long per_thread = (((long long)(p->V >> 3) + UT - 1) / UT) * 8 + 1;
     if ((p->k - 1) * per_thread > UCAP) return GRAFT_ERR_UNSUPPORTED;
-    update_kernel<<<p->B * p->T_max, UT, 0, static_cast<cudaStream_t>(stream)>>>(*p, ctx->status);
-    GRAFT_CHECK_CUDA(cudaGetLastError());
+    GRAFT_CHECK_CUDA(graft_launch(update_kernel, dim3(p->B * p->T_max), dim3(UT), 0, static_cast<cudaStream_t>(stream), *p, ctx->status));
     return GRAFT_OK;
 }
