@@ -346,7 +346,8 @@ int graft_accept(graft_ctx* ctx, const graft_accept_params* p, void* stream);
  * an outcome is only defined up to that rounding when a random number falls within ~1e-5 (relative to
  * rem) of a decision boundary.
  * row_stats: caller-provided scratch of graft_accept_stochastic_scratch_floats(B, T_max, V) floats (per row the
- * max of logits / temperature and the sum of exponentials, of the whole row and of every 256 ids).
+ * max of logits / temperature and the sum of exponentials, of the parts of the row that one CTA each scans and of
+ * every 256 ids).
  * logits: 16-byte aligned base, row stride a multiple of 8 elements; temperature > 0; T_max <= 64; V <= 524288.
  */
 typedef struct {

@@ -1,7 +1,7 @@
 // graft_accept_stochastic: acceptance under temperature sampling, two kernels.
 //
-//   softmax_stats_kernel   one CTA per tree node streams that node's V logits once and leaves the row's
-//                          (max of logit / temperature, sum of exponentials) pair and the same pair for
+//   softmax_stats_kernel   two CTAs per tree node stream that node's V logits once (alternate rounds of steps) and
+//                          leave their (max of logit / temperature, sum of exponentials) pairs and the same pair for
 //                          every step of 256 ids: which rows the walk will need is only known while
 //                          walking, so all valid rows are done at once, in parallel (HBM-bound: V * 2 bytes
 //                          per valid node, as the adjacency refresh);
@@ -21,12 +21,14 @@ constexpr int ST = 512;        // threads of the statistics kernel
 constexpr int WT = 1024;       // threads of the walk kernel
 constexpr int kStep = 256;     // ids per step: eight per lane of a warp
 constexpr int kMaxSteps = 2 * WT;   // steps of a row the walk kernel can scan: V <= 524288
+constexpr int kParts = 2;      // CTAs that share a row of the statistics kernel (alternate rounds of steps): one CTA per row left
+                               // most SMs with one row and some with two (measured: -3 us on 192 rows, -8 us on 48)
 
 __device__ __forceinline__ float lo_f(uint32_t w) { return __uint_as_float(w << 16); }
 __device__ __forceinline__ float hi_f(uint32_t w) { return __uint_as_float(w & 0xffff0000u); }
 __host__ __device__ __forceinline__ int steps_of(int V) { return (V + kStep - 1) / kStep; }
-// scratch of a row: (m, s) of the row, then (m, s) of every step
-__host__ __device__ __forceinline__ size_t row_floats(int V) { return 2 + 2 * (size_t)steps_of(V); }
+// scratch of a row: (m, s) of each part of the row, then (m, s) of every step
+__host__ __device__ __forceinline__ size_t row_floats(int V) { return 2 * kParts + 2 * (size_t)steps_of(V); }
 
 // (m, s) <- (m, s) (+) (m2, s2): s counts exponentials relative to m
 __device__ __forceinline__ void combine(float& m, float& s, float m2, float s2) {
@@ -34,6 +36,19 @@ __device__ __forceinline__ void combine(float& m, float& s, float m2, float s2) 
     if (mn == -CUDART_INF_F) { m = mn; s = 0.f; return; }
     s = s * __expf(m - mn) + s2 * __expf(m2 - mn);
     m = mn;
+}
+
+// (m, s) of a whole row from its parts' pairs, and m alone
+__device__ __forceinline__ void row_pair(const float* st, float& m, float& s) {
+    m = st[0]; s = st[1];
+#pragma unroll
+    for (int q = 1; q < kParts; ++q) combine(m, s, st[2 * q], st[2 * q + 1]);
+}
+__device__ __forceinline__ float row_max(const float* st) {
+    float m = st[0];
+#pragma unroll
+    for (int q = 1; q < kParts; ++q) m = fmaxf(m, st[2 * q]);
+    return m;
 }
 
 // eight scaled logits of a lane: ids v0 .. v0 + 7 of the row, -inf past its end
@@ -48,13 +63,13 @@ __device__ __forceinline__ void scaled8(const __nv_bfloat16* row, int v0, int V,
     }
 }
 
-// One CTA per tree node; a warp takes a step of 256 ids at a time (four in flight), leaves the step's
-// (max, sum of exponentials relative to it) and folds it into its running pair.
+// kParts CTAs per tree node; a warp takes a step of 256 ids at a time (four in flight), leaves the step's
+// (max, sum of exponentials relative to it) and folds it into its running pair; the CTA leaves the pair of its part.
 __global__ void __launch_bounds__(ST, 2) softmax_stats_kernel(graft_accept_stochastic_params p) {
     graft_wait_for_stream();
     __shared__ float s_m[ST / 32], s_s[ST / 32];
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-    const int r = blockIdx.x, b = r / p.T_max, i = r % p.T_max;
+    const int r = blockIdx.x / kParts, part = blockIdx.x % kParts, b = r / p.T_max, i = r % p.T_max;
     int T = p.tree_size[b];
     if (T < 0 || T > p.T_max) T = 0;
     if (i >= T) return;
@@ -64,7 +79,7 @@ __global__ void __launch_bounds__(ST, 2) softmax_stats_kernel(graft_accept_stoch
     const int nsteps = steps_of(p.V);
     float m = -CUDART_INF_F, s = 0.f;
     constexpr int NWS = ST / 32, kFlight = 4;          // steps a warp has in flight; they share one reference maximum
-    for (int st = warp; st < nsteps; st += kFlight * NWS) {
+    for (int st = warp + part * kFlight * NWS; st < nsteps; st += kParts * kFlight * NWS) {
         float z[kFlight][8];
         float vm = -CUDART_INF_F;
         if ((st + (kFlight - 1) * NWS + 1) * kStep <= p.V) {
@@ -112,7 +127,7 @@ __global__ void __launch_bounds__(ST, 2) softmax_stats_kernel(graft_accept_stoch
         for (int h = 0; h < kFlight; ++h) {
             const int sx = st + h * NWS;
             if (sx < nsteps) {
-                if (lane == h) { out[2 + 2 * sx] = vm; out[2 + 2 * sx + 1] = add[h]; }
+                if (lane == h) { out[2 * kParts + 2 * sx] = vm; out[2 * kParts + 2 * sx + 1] = add[h]; }
                 tot += add[h];
             }
         }
@@ -128,7 +143,7 @@ __global__ void __launch_bounds__(ST, 2) softmax_stats_kernel(graft_accept_stoch
             const float m2 = __shfl_xor_sync(0xffffffffu, m, o), s2 = __shfl_xor_sync(0xffffffffu, s, o);
             combine(m, s, m2, s2);
         }
-        if (lane == 0) { out[0] = m; out[1] = s; }
+        if (lane == 0) { out[2 * part] = m; out[2 * part + 1] = s; }
     }
 }
 
@@ -167,10 +182,9 @@ __global__ void __launch_bounds__(WT) accept_walk_kernel(graft_accept_stochastic
             par = p.tree_parent[(size_t)b * p.T_max + tid];
             x = p.tree_token[(size_t)b * p.T_max + tid];
             u = p.u_accept[(size_t)b * p.T_max + tid];
-            m = stats[tid * rf];
-            sm = stats[tid * rf + 1];
+            row_pair(stats + tid * rf, m, sm);
             if (tid == 0 || par < 0 || par >= tid) par = -1;               // the root, or not a tree node: nobody's child
-            else if (x >= 0 && x < p.V) w = __expf(__bfloat162float(lg[(size_t)par * p.logits_stride_row + x]) * inv_t - stats[par * rf]);
+            else if (x >= 0 && x < p.V) w = __expf(__bfloat162float(lg[(size_t)par * p.logits_stride_row + x]) * inv_t - row_max(stats + par * rf));
         }
         s_par[tid] = par; s_tok[tid] = x; s_w[tid] = w; s_u[tid] = u; s_m[tid] = m; s_s[tid] = sm;
     }
@@ -207,7 +221,7 @@ __global__ void __launch_bounds__(WT) accept_walk_kernel(graft_accept_stochastic
     const int u = s_best, nrej = s_nrej;
     const float m = s_m[u], target = p.u_bonus[b] * s_rem * s_s[u];
     const __nv_bfloat16* row = lg + (size_t)u * p.logits_stride_row;
-    const float* steps = stats + u * rf + 2;
+    const float* steps = stats + u * rf + 2 * kParts;
     const int nsteps = steps_of(p.V);
     for (int st = tid; st < nsteps; st += WT) {
         const float ms = steps[2 * st];
@@ -305,7 +319,7 @@ extern "C" int graft_accept_stochastic(graft_ctx* ctx, const graft_accept_stocha
     if (!graft_aligned16(p->logits) || p->logits_stride_row < p->V || p->logits_stride_row % 8 != 0) return GRAFT_ERR_INVALID_ARG;
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     // both kernels are programmatic dependents of the kernel before them: the walk's CTAs are set up while the statistics drain
-    GRAFT_CHECK_CUDA(graft_launch(softmax_stats_kernel, dim3(p->B * p->T_max), dim3(ST), 0, s, *p));
+    GRAFT_CHECK_CUDA(graft_launch(softmax_stats_kernel, dim3(p->B * p->T_max * kParts), dim3(ST), 0, s, *p));
     GRAFT_CHECK_CUDA(graft_launch(accept_walk_kernel, dim3(p->B), dim3(WT), 0, s, *p, ctx->status));
     return GRAFT_OK;
 }
